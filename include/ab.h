@@ -1,0 +1,150 @@
+/*
+ * libab: the per-GPU hot path of AB-Training on NVIDIA B200 (sm_100a).
+ *
+ * Notation (the paper's Eq. 3, with its k written r): a layer weight W (m x n,
+ * out-features x in-features) is held as W = A B with A (m x r) and B (r x n).
+ * Activations x are N x n, outputs y and upstream gradients dY are N x m,
+ * T = x B^T and dT = dY A are N x r.  Every matrix is row-major.
+ *
+ * Conventions for every call
+ *  - Pointers are DEVICE pointers owned by the caller unless a parameter says "host".
+ *    The library allocates no device memory and keeps no state between calls; scratch
+ *    space is passed in as `ws` (size from ab_workspace_bytes, 256-byte aligned).
+ *  - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
+ *    default stream).  Buffers must stay valid until the stream has run the call.
+ *  - Arguments that can be checked on the host (NULL, non-positive sizes, r > min(m,n),
+ *    a short workspace, a misaligned pointer) are rejected with a negative status and
+ *    nothing is launched.  Conditions only the device can see (an iteration that did not
+ *    converge, a bounded wait that ran out) are written to a device status word and never
+ *    trap; the context stays usable.
+ *  - There is no CPU fallback: without a CUDA device every compute call returns AB_ERR_CUDA.
+ *  - bf16 storage always means fp32 accumulation.  dA, dB, sigma are always fp32.
+ */
+#ifndef AB_H_
+#define AB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  AB_OK = 0,
+  AB_ERR_INVALID_ARG = -1,   /* NULL pointer, non-positive size, r > min(m,n), bad leading dimension */
+  AB_ERR_UNSUPPORTED = -2,   /* a size beyond what the kernels handle (stated per call) */
+  AB_ERR_WORKSPACE = -3,     /* ws NULL, misaligned or smaller than ab_workspace_bytes says */
+  AB_ERR_NOT_CONVERGED = -4, /* device status: Jacobi sweep cap reached */
+  AB_ERR_TIMEOUT = -5,       /* device status: a bounded on-chip wait expired */
+  AB_ERR_CUDA = -6           /* a CUDA runtime call failed (no device, launch error) */
+} ab_status;
+
+typedef enum { AB_F32 = 0, AB_BF16 = 1 } ab_dtype;
+
+typedef enum {
+  AB_OP_LAYER_FORWARD = 0,
+  AB_OP_LAYER_BACKWARD = 1,
+  AB_OP_GROUP_AVERAGE = 2,
+  AB_OP_RECOMBINE = 3,
+  AB_OP_SVD_SPLIT = 4
+} ab_op;
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* ab_status_string(int status);
+
+/* Library version, "major.minor". */
+const char* ab_version(void);
+
+/*
+ * Scratch bytes a call needs (0 if none).  Arguments a given op does not use are ignored
+ * (pass 0).  For AB_OP_SVD_SPLIT, r is r_max.  Returns 0 for unknown ops or bad sizes.
+ */
+size_t ab_workspace_bytes(int op, int64_t N, int m, int n, int r, int K, int dt);
+
+/*
+ * Forward of the factorised layer (Eq. 3 used as a linear map): y = (x B^T) A^T.
+ *   x [N,n], A [m,r] (row stride ldA >= r), B [r,n] (row stride ldB >= n), y [N,m], all of
+ *   storage type dt.  T_save: NULL, or [N,r] of type dt that receives T = x B^T for the
+ *   backward call.  The rank-r intermediate stays on chip when dt = AB_BF16, r is a
+ *   multiple of 16 with 16 <= r <= 256 and m, n are multiples of 8; other shapes take a
+ *   slower general kernel (same results to rounding).  N = 0 is a no-op.
+ */
+int ab_layer_forward(const void* x, const void* A, const void* B, void* y, void* T_save,
+                     int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
+                     void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Backward of the factorised layer (chain rule through T):
+ *   dT = dY A, dX = dT B, dA = dY^T T, dB = dT^T x.
+ *   dX [N,n] of type dt; dA [m,r] and dB [r,n] are fp32 and dense (row strides r and n).
+ *   Any of dX, dA, dB may be NULL (not wanted: groups that train only A or only B).
+ *   T_saved: the T written by ab_layer_forward, or NULL to recompute it from x.
+ *   Sums over N are taken in a fixed order: two runs give identical bits.
+ */
+int ab_layer_backward(const void* x, const void* dY, const void* A, const void* B,
+                      const void* T_saved, void* dX, float* dA, float* dB,
+                      int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
+                      void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Mean of K group copies (Algorithm 1: A <- allReduce(A / worldSize), likewise B), the K
+ * workers being K arenas in one device's memory: copy k starts at base + k*stride_elems
+ * (elements of in_dt).  In fp32 and in a fixed order:
+ *   out[i] = fl( (((c0[i] + c1[i]) + c2[i]) + ...) * fl(1/K) ),   i < count.
+ * For K a power of two this equals the paper's divide-then-sum bit for bit.
+ * out has type out_dt (fp32 -> bf16 rounds to nearest even).  1 <= K <= 64.
+ */
+int ab_group_average(const void* base, int64_t stride_elems, int K, int64_t count,
+                     int in_dt, int out_dt, void* out, void* cuda_stream);
+
+/*
+ * Recombination (Algorithm 1: W <- A B): W [m,n] fp32 (dense) = Abar [m,r] Bbar [r,n],
+ * factors of type dt, product accumulated in fp32 without reduced-precision passes.
+ */
+int ab_recombine(const void* Abar, const void* Bbar, float* W, int m, int n, int r,
+                 int ldA, int ldB, int dt, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Truncated SVD and split (Eq. 3 with the rank rule of the AB-decomposition phase):
+ *   W = U S V^T;  r' = #{ i < r_cap : s_i >= sigma_cutoff * s_0 }, at least 1, where
+ *   r_cap = min(r_max, m, n);  A = U_r' S_r'^(1/2),  B = S_r'^(1/2) V_r'^T.
+ *   W [m,n] dense of type w_dt.  A [m,r_max] (row stride r_max) and B [r_max,n] of type
+ *   out_dt; columns of A and rows of B with index >= r' are zero.  sigma [r_cap] fp32,
+ *   descending up to rounding; r_out: device int that receives r'; dev_status: device
+ *   int that receives AB_OK or AB_ERR_NOT_CONVERGED.  sigma_cutoff = 0 keeps r_cap.
+ *   The decomposition works on the Gram matrix of the shorter side in fp32; singular
+ *   values below about 2% of the largest lose relative accuracy (they keep absolute
+ *   accuracy 1e-6 * s_0).  min(m,n) <= 3072.
+ */
+int ab_svd_split(const void* W, int m, int n, int r_max, float sigma_cutoff,
+                 void* A, void* B, float* sigma, int* r_out, int* dev_status,
+                 int w_dt, int out_dt, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* One matrix of a batched group synchronisation.  All pointers are device pointers. */
+typedef struct {
+  const void* A_copies;   /* K copies of A [m,r], copy k at A_copies + k*strideA elements */
+  const void* B_copies;   /* K copies of B [r,n] */
+  int64_t strideA, strideB;
+  int m, n, r;            /* r = rank of the incoming factors = r_max of the outgoing ones */
+  void* A_out;            /* [m,r] */
+  void* B_out;            /* [r,n] */
+  float* sigma;           /* [min(r,m,n)] */
+  int* r_out;             /* device int */
+} ab_sync_desc;
+
+/*
+ * Group synchronisation of a whole model (Algorithm 1 from the two all-reduces to the next
+ * decomposition): for each of the L matrices, mean of the K copies of A and of B, W = Abar
+ * Bbar, then the split of W as in ab_svd_split.  descs: HOST array of L descriptors (read
+ * before the call returns).  Factor storage dt on both sides.  dev_status: device int[L].
+ * Workspace: ab_sync_workspace_bytes.
+ */
+int ab_group_sync(const ab_sync_desc* descs, int L, int K, float sigma_cutoff, int dt,
+                  int* dev_status, void* ws, size_t ws_bytes, void* cuda_stream);
+size_t ab_sync_workspace_bytes(const ab_sync_desc* descs, int L, int K, int dt);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AB_H_ */

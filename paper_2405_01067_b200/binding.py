@@ -1,0 +1,239 @@
+"""ctypes binding of libab.so: same names as the C entry points (include/ab.h), argument
+marshalling only.  Tensors are torch CUDA tensors (torch supplies device memory and streams);
+every step of the computation runs in the library's kernels.  There is no CPU path: loading
+fails loudly when the library has not been built, and every call raises on a negative status.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_char_p, c_float, c_int, c_int64, c_size_t, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libab.so")
+
+AB_F32, AB_BF16 = 0, 1
+AB_OP_LAYER_FORWARD, AB_OP_LAYER_BACKWARD, AB_OP_GROUP_AVERAGE, AB_OP_RECOMBINE, AB_OP_SVD_SPLIT = range(5)
+AB_OK = 0
+AB_ERR_INVALID_ARG, AB_ERR_UNSUPPORTED, AB_ERR_WORKSPACE = -1, -2, -3
+AB_ERR_NOT_CONVERGED, AB_ERR_TIMEOUT, AB_ERR_CUDA = -4, -5, -6
+
+EXPORTS = ["ab_status_string", "ab_version", "ab_workspace_bytes", "ab_layer_forward", "ab_layer_backward",
+           "ab_group_average", "ab_recombine", "ab_svd_split", "ab_group_sync", "ab_sync_workspace_bytes"]
+
+
+class AbError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+class ab_sync_desc(ctypes.Structure):
+    _fields_ = [("A_copies", c_void_p), ("B_copies", c_void_p), ("strideA", c_int64), ("strideB", c_int64),
+                ("m", c_int), ("n", c_int), ("r", c_int), ("A_out", c_void_p), ("B_out", c_void_p),
+                ("sigma", c_void_p), ("r_out", c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded library.  Raises if it has not been built (python -m paper_2405_01067_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python paper_2405_01067_b200/build.py`; "
+                           "there is no fallback path")
+    L = ctypes.CDLL(LIB_PATH)
+    L.ab_status_string.restype = c_char_p
+    L.ab_status_string.argtypes = [c_int]
+    L.ab_version.restype = c_char_p
+    L.ab_workspace_bytes.restype = c_size_t
+    L.ab_workspace_bytes.argtypes = [c_int, c_int64, c_int, c_int, c_int, c_int, c_int]
+    L.ab_layer_forward.restype = c_int
+    L.ab_layer_forward.argtypes = [c_void_p] * 5 + [c_int64] + [c_int] * 6 + [c_void_p, c_size_t, c_void_p]
+    L.ab_layer_backward.restype = c_int
+    L.ab_layer_backward.argtypes = [c_void_p] * 8 + [c_int64] + [c_int] * 6 + [c_void_p, c_size_t, c_void_p]
+    L.ab_group_average.restype = c_int
+    L.ab_group_average.argtypes = [c_void_p, c_int64, c_int, c_int64, c_int, c_int, c_void_p, c_void_p]
+    L.ab_recombine.restype = c_int
+    L.ab_recombine.argtypes = [c_void_p, c_void_p, c_void_p] + [c_int] * 6 + [c_void_p, c_size_t, c_void_p]
+    L.ab_svd_split.restype = c_int
+    L.ab_svd_split.argtypes = [c_void_p, c_int, c_int, c_int, c_float] + [c_void_p] * 5 + [c_int, c_int,
+                                                                                         c_void_p, c_size_t, c_void_p]
+    L.ab_group_sync.restype = c_int
+    L.ab_group_sync.argtypes = [ctypes.POINTER(ab_sync_desc), c_int, c_int, c_float, c_int, c_void_p, c_void_p,
+                                c_size_t, c_void_p]
+    L.ab_sync_workspace_bytes.restype = c_size_t
+    L.ab_sync_workspace_bytes.argtypes = [ctypes.POINTER(ab_sync_desc), c_int, c_int, c_int]
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().ab_status_string(int(status)).decode()
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return AB_F32
+    if t.dtype == torch.bfloat16:
+        return AB_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return c_void_p(s.cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != AB_OK:
+        raise AbError(status, where)
+
+
+def _dev_ok(*ts):
+    for t in ts:
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("tensors must be contiguous CUDA tensors")
+
+
+def workspace(nbytes: int, device) -> torch.Tensor:
+    """A 256-byte aligned scratch buffer of at least nbytes (torch's allocator aligns to 512)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def ab_workspace_bytes(op: int, N: int, m: int, n: int, r: int, K: int = 1, dt: int = AB_F32) -> int:
+    return int(lib().ab_workspace_bytes(op, N, m, n, r, K, dt))
+
+
+def ab_layer_forward(x, A, B, y=None, T_save=None, ws=None, stream=None, save_T=False):
+    """y = (x B^T) A^T.  Returns (y, T_save or None)."""
+    _dev_ok(x, A, B, y, T_save)
+    N, n = x.shape
+    m, r = A.shape
+    dt = _dt(x)
+    if y is None:
+        y = torch.empty((N, m), dtype=x.dtype, device=x.device)
+    if save_T and T_save is None:
+        T_save = torch.empty((N, r), dtype=x.dtype, device=x.device)
+    if ws is None:
+        ws = workspace(ab_workspace_bytes(AB_OP_LAYER_FORWARD, N, m, n, r, 1, dt), x.device)
+    st = lib().ab_layer_forward(_ptr(x), _ptr(A), _ptr(B), _ptr(y), _ptr(T_save), N, m, n, r,
+                                A.stride(0), B.stride(0), dt, _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "ab_layer_forward")
+    return y, T_save
+
+
+def ab_layer_backward(x, dY, A, B, T_saved=None, want=("dX", "dA", "dB"), dX=None, dA=None, dB=None,
+                      ws=None, stream=None):
+    """dX = (dY A) B, dA = dY^T T, dB = (dY A)^T x.  Returns (dX, dA, dB); entries not in `want` are None."""
+    _dev_ok(x, dY, A, B, T_saved, dX, dA, dB)
+    N, n = x.shape
+    m, r = A.shape
+    dt = _dt(x)
+    if "dX" in want and dX is None:
+        dX = torch.empty((N, n), dtype=x.dtype, device=x.device)
+    if "dA" in want and dA is None:
+        dA = torch.empty((m, r), dtype=torch.float32, device=x.device)
+    if "dB" in want and dB is None:
+        dB = torch.empty((r, n), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = workspace(ab_workspace_bytes(AB_OP_LAYER_BACKWARD, N, m, n, r, 1, dt), x.device)
+    st = lib().ab_layer_backward(_ptr(x), _ptr(dY), _ptr(A), _ptr(B), _ptr(T_saved), _ptr(dX), _ptr(dA), _ptr(dB),
+                                 N, m, n, r, A.stride(0), B.stride(0), dt, _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "ab_layer_backward")
+    return dX, dA, dB
+
+
+def ab_group_average(copies, out=None, out_dtype=None, stream=None):
+    """Mean over the leading axis of a (K, ...) tensor, fp32 sum in ascending k."""
+    _dev_ok(copies, out)
+    K = copies.shape[0]
+    count = copies[0].numel()
+    if out is None:
+        out = torch.empty(copies.shape[1:], dtype=out_dtype or torch.float32, device=copies.device)
+    st = lib().ab_group_average(_ptr(copies), copies.stride(0) if K > 1 else count, K, count, _dt(copies), _dt(out),
+                                _ptr(out), _stream(stream))
+    _check(st, "ab_group_average")
+    return out
+
+
+def ab_recombine(Abar, Bbar, W=None, stream=None):
+    """W = Abar Bbar in fp32."""
+    _dev_ok(Abar, Bbar, W)
+    m, r = Abar.shape
+    n = Bbar.shape[1]
+    if W is None:
+        W = torch.empty((m, n), dtype=torch.float32, device=Abar.device)
+    st = lib().ab_recombine(_ptr(Abar), _ptr(Bbar), _ptr(W), m, n, r, Abar.stride(0), Bbar.stride(0), _dt(Abar),
+                            None, 0, _stream(stream))
+    _check(st, "ab_recombine")
+    return W
+
+
+def ab_svd_split(W, r_max, sigma_cutoff=0.0, out_dtype=None, ws=None, stream=None):
+    """A = U_r' S^(1/2), B = S^(1/2) V_r'^T under the rank rule.  Returns (A, B, sigma, r_out, dev_status);
+    r_out and dev_status are device int tensors (read them after synchronising)."""
+    _dev_ok(W)
+    m, n = W.shape
+    od = out_dtype or W.dtype
+    r_cap = min(r_max, m, n)
+    A = torch.empty((m, r_max), dtype=od, device=W.device)
+    B = torch.empty((r_max, n), dtype=od, device=W.device)
+    sigma = torch.empty((r_cap,), dtype=torch.float32, device=W.device)
+    r_out = torch.zeros((1,), dtype=torch.int32, device=W.device)
+    status = torch.zeros((1,), dtype=torch.int32, device=W.device)
+    if ws is None:
+        ws = workspace(ab_workspace_bytes(AB_OP_SVD_SPLIT, 0, m, n, r_max, 1, _dt(W)), W.device)
+    st = lib().ab_svd_split(_ptr(W), m, n, r_max, float(sigma_cutoff), _ptr(A), _ptr(B), _ptr(sigma), _ptr(r_out),
+                            _ptr(status), _dt(W), AB_BF16 if od == torch.bfloat16 else AB_F32, _ptr(ws), ws.numel(),
+                            _stream(stream))
+    _check(st, "ab_svd_split")
+    return A, B, sigma, r_out, status
+
+
+class SyncPlan:
+    """Buffers and descriptors of one model's group synchronisation (ab_group_sync)."""
+
+    def __init__(self, A_copies, B_copies, sigma_cutoff):
+        self.A_copies, self.B_copies = list(A_copies), list(B_copies)
+        self.L = len(self.A_copies)
+        self.K = self.A_copies[0].shape[0]
+        self.cutoff = float(sigma_cutoff)
+        dev = self.A_copies[0].device
+        self.dt = _dt(self.A_copies[0])
+        self.A_out, self.B_out, self.sigma = [], [], []
+        self.r_out = torch.zeros((self.L,), dtype=torch.int32, device=dev)
+        self.status = torch.zeros((self.L,), dtype=torch.int32, device=dev)
+        self.descs = (ab_sync_desc * self.L)()
+        for i, (Ak, Bk) in enumerate(zip(self.A_copies, self.B_copies)):
+            _dev_ok(Ak, Bk)
+            K, m, r = Ak.shape
+            n = Bk.shape[2]
+            self.A_out.append(torch.empty((m, r), dtype=Ak.dtype, device=dev))
+            self.B_out.append(torch.empty((r, n), dtype=Ak.dtype, device=dev))
+            self.sigma.append(torch.empty((min(r, m, n),), dtype=torch.float32, device=dev))
+            d = self.descs[i]
+            d.A_copies, d.B_copies = Ak.data_ptr(), Bk.data_ptr()
+            d.strideA, d.strideB = (Ak.stride(0), Bk.stride(0)) if K > 1 else (m * r, r * n)
+            d.m, d.n, d.r = m, n, r
+            d.A_out, d.B_out = self.A_out[i].data_ptr(), self.B_out[i].data_ptr()
+            d.sigma = self.sigma[i].data_ptr()
+            d.r_out = self.r_out.data_ptr() + 4 * i
+        self.ws = workspace(lib().ab_sync_workspace_bytes(self.descs, self.L, self.K, self.dt), dev)
+
+
+def ab_group_sync(plan: SyncPlan, stream=None):
+    """Mean of K copies -> W = Abar Bbar -> split under the rank rule, for every matrix of the plan."""
+    st = lib().ab_group_sync(plan.descs, plan.L, plan.K, plan.cutoff, plan.dt, _ptr(plan.status), _ptr(plan.ws),
+                             plan.ws.numel(), _stream(stream))
+    _check(st, "ab_group_sync")
+    return plan.A_out, plan.B_out, plan.sigma, plan.r_out, plan.status

@@ -1,0 +1,250 @@
+// C-ABI entry points: argument checks, workspace carving, dispatch.  See include/ab.h.
+#include <vector>
+#include <string.h>
+
+#include "ab_common.cuh"
+
+namespace ab {
+namespace {
+
+template <typename TI, typename TO>
+__global__ void cast_kernel(const TI* __restrict__ in, TO* __restrict__ out, int64_t count) {
+  const int64_t step = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += step) from_f32(out[i], to_f32(in[i]));
+}
+
+int cast_f32_to(const float* in, void* out, int dt, int64_t count, cudaStream_t st) {
+  if (count == 0) return AB_OK;
+  unsigned grid = (unsigned)((count + 255) / 256 < 148 * 8 ? (count + 255) / 256 : 148 * 8);
+  if (dt == AB_F32) cast_kernel<float, float><<<grid, 256, 0, st>>>(in, static_cast<float*>(out), count);
+  else cast_kernel<float, bf16><<<grid, 256, 0, st>>>(in, static_cast<bf16*>(out), count);
+  AB_LAUNCH_OK();
+  return AB_OK;
+}
+
+bool have_device() {
+  int n = 0;
+  return cudaGetDeviceCount(&n) == cudaSuccess && n > 0;
+}
+
+int check_layer_args(const void* x, const void* A, const void* B, int64_t N, int m, int n, int r,
+                     int ldA, int ldB, int dt) {
+  if (!dtype_ok(dt)) return AB_ERR_INVALID_ARG;
+  if (N < 0 || m <= 0 || n <= 0 || r <= 0) return AB_ERR_INVALID_ARG;
+  if (r > m || r > n) return AB_ERR_INVALID_ARG;
+  if (ldA < r || ldB < n) return AB_ERR_INVALID_ARG;
+  if (!x || !A || !B) return AB_ERR_INVALID_ARG;
+  return AB_OK;
+}
+
+// general path: every product is one strided GEMM on the fp32 pipes, T and dT live in the workspace
+size_t general_forward_ws(int64_t N, int r) { return align_up((size_t)N * r * sizeof(float), 256); }
+size_t general_backward_ws(int64_t N, int r) { return 2 * align_up((size_t)N * r * sizeof(float), 256); }
+
+int general_forward(const void* x, const void* A, const void* B, void* y, void* T_save,
+                    int64_t N, int m, int n, int r, int ldA, int ldB, int dt, void* ws, size_t ws_bytes,
+                    cudaStream_t st) {
+  Arena ar(ws, ws_bytes);
+  float* T = ar.take_n<float>((size_t)N * r);
+  if (!ws || !ar.fits()) return AB_ERR_WORKSPACE;
+  AB_TRY(gemm_simt(x, dt, n, 1, B, dt, 1, ldB, T, AB_F32, r, N, r, n, st));        // T = x B^T
+  if (T_save) AB_TRY(cast_f32_to(T, T_save, dt, N * r, st));
+  AB_TRY(gemm_simt(T, AB_F32, r, 1, A, dt, 1, ldA, y, dt, m, N, m, r, st));         // y = T A^T
+  return AB_OK;
+}
+
+int general_backward(const void* x, const void* dY, const void* A, const void* B, const void* T_saved,
+                     void* dX, float* dA, float* dB, int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
+                     void* ws, size_t ws_bytes, cudaStream_t st) {
+  Arena ar(ws, ws_bytes);
+  float* T = ar.take_n<float>((size_t)N * r);
+  float* dT = ar.take_n<float>((size_t)N * r);
+  if (!ws || !ar.fits()) return AB_ERR_WORKSPACE;
+  AB_TRY(gemm_simt(dY, dt, m, 1, A, dt, ldA, 1, dT, AB_F32, r, N, r, m, st));      // dT = dY A
+  if (dX) AB_TRY(gemm_simt(dT, AB_F32, r, 1, B, dt, ldB, 1, dX, dt, n, N, n, r, st));   // dX = dT B
+  if (dA) {
+    const void* Tsrc = T_saved;
+    int t_dt = dt;
+    if (!Tsrc) {
+      AB_TRY(gemm_simt(x, dt, n, 1, B, dt, 1, ldB, T, AB_F32, r, N, r, n, st));
+      Tsrc = T;
+      t_dt = AB_F32;
+    }
+    AB_TRY(gemm_simt(dY, dt, 1, m, Tsrc, t_dt, r, 1, dA, AB_F32, r, m, r, N, st));  // dA = dY^T T
+  }
+  if (dB) AB_TRY(gemm_simt(dT, AB_F32, 1, r, x, dt, n, 1, dB, AB_F32, n, r, n, N, st));  // dB = dT^T x
+  return AB_OK;
+}
+
+}  // namespace
+}  // namespace ab
+
+using namespace ab;
+
+extern "C" {
+
+const char* ab_status_string(int s) {
+  switch (s) {
+    case AB_OK: return "ok";
+    case AB_ERR_INVALID_ARG: return "invalid argument";
+    case AB_ERR_UNSUPPORTED: return "unsupported size";
+    case AB_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case AB_ERR_NOT_CONVERGED: return "iteration did not converge";
+    case AB_ERR_TIMEOUT: return "bounded device wait expired";
+    case AB_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown status";
+  }
+}
+
+const char* ab_version(void) { return "0.1"; }
+
+size_t ab_workspace_bytes(int op, int64_t N, int m, int n, int r, int K, int dt) {
+  (void)K;
+  if (m <= 0 || n <= 0 || r <= 0 || N < 0) return 0;
+  switch (op) {
+    case AB_OP_LAYER_FORWARD: {
+      size_t g = general_forward_ws(N, r), t = chain_tc_forward_ws(N, m, n, r);
+      return (g > t ? g : t) + 256;
+    }
+    case AB_OP_LAYER_BACKWARD: {
+      size_t g = general_backward_ws(N, r), t = chain_tc_backward_ws(N, m, n, r);
+      return (g > t ? g : t) + 256;
+    }
+    case AB_OP_SVD_SPLIT: {
+      SvdItem it;
+      memset(&it, 0, sizeof(it));
+      it.m = m; it.n = n; it.r_max = r; it.w_dt = dt; it.out_dt = dt;
+      return svd_batch_ws(&it, 1) + 256;
+    }
+    default: return 0;
+  }
+}
+
+int ab_layer_forward(const void* x, const void* A, const void* B, void* y, void* T_save,
+                     int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
+                     void* ws, size_t ws_bytes, void* cuda_stream) {
+  AB_TRY(check_layer_args(x, A, B, N, m, n, r, ldA, ldB, dt));
+  if (!y) return AB_ERR_INVALID_ARG;
+  if (!have_device()) return AB_ERR_CUDA;
+  if (N == 0) return AB_OK;
+  if (ws && !aligned(ws, 256)) return AB_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (chain_tc_supported(N, m, n, r, ldA, ldB, dt, x, A, B, y))
+    return chain_tc_forward(x, A, B, y, T_save, N, m, n, r, ldA, ldB, ws, ws_bytes, st);
+  return general_forward(x, A, B, y, T_save, N, m, n, r, ldA, ldB, dt, ws, ws_bytes, st);
+}
+
+int ab_layer_backward(const void* x, const void* dY, const void* A, const void* B,
+                      const void* T_saved, void* dX, float* dA, float* dB,
+                      int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
+                      void* ws, size_t ws_bytes, void* cuda_stream) {
+  AB_TRY(check_layer_args(x, A, B, N, m, n, r, ldA, ldB, dt));
+  if (!dY) return AB_ERR_INVALID_ARG;
+  if (!have_device()) return AB_ERR_CUDA;
+  if (ws && !aligned(ws, 256)) return AB_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (N == 0) {   // empty batch: the sums over N are empty
+    if (dA) AB_CUDA_OK(cudaMemsetAsync(dA, 0, (size_t)m * r * sizeof(float), st));
+    if (dB) AB_CUDA_OK(cudaMemsetAsync(dB, 0, (size_t)r * n * sizeof(float), st));
+    return AB_OK;
+  }
+  if (chain_tc_supported(N, m, n, r, ldA, ldB, dt, x, A, B, dY))
+    return chain_tc_backward(x, dY, A, B, T_saved, dX, dA, dB, N, m, n, r, ldA, ldB, ws, ws_bytes, st);
+  return general_backward(x, dY, A, B, T_saved, dX, dA, dB, N, m, n, r, ldA, ldB, dt, ws, ws_bytes, st);
+}
+
+int ab_group_average(const void* base, int64_t stride_elems, int K, int64_t count,
+                     int in_dt, int out_dt, void* out, void* cuda_stream) {
+  if (!dtype_ok(in_dt) || !dtype_ok(out_dt)) return AB_ERR_INVALID_ARG;
+  if (K < 1 || count < 0) return AB_ERR_INVALID_ARG;
+  if (K > 64) return AB_ERR_UNSUPPORTED;
+  if (count > 0 && (!base || !out)) return AB_ERR_INVALID_ARG;
+  if (K > 1 && stride_elems < count) return AB_ERR_INVALID_ARG;   // copies would overlap
+  if (!aligned(base, dtype_size(in_dt)) || !aligned(out, dtype_size(out_dt))) return AB_ERR_INVALID_ARG;
+  if (!have_device()) return AB_ERR_CUDA;
+  return group_average(base, stride_elems, K, count, in_dt, out_dt, out, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ab_recombine(const void* Abar, const void* Bbar, float* W, int m, int n, int r,
+                 int ldA, int ldB, int dt, void* ws, size_t ws_bytes, void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  if (!dtype_ok(dt) || m <= 0 || n <= 0 || r <= 0 || ldA < r || ldB < n) return AB_ERR_INVALID_ARG;
+  if (!Abar || !Bbar || !W) return AB_ERR_INVALID_ARG;
+  if (!have_device()) return AB_ERR_CUDA;
+  return gemm_simt(Abar, dt, ldA, 1, Bbar, dt, ldB, 1, W, AB_F32, n, m, n, r, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ab_svd_split(const void* W, int m, int n, int r_max, float sigma_cutoff,
+                 void* A, void* B, float* sigma, int* r_out, int* dev_status,
+                 int w_dt, int out_dt, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (!dtype_ok(w_dt) || !dtype_ok(out_dt)) return AB_ERR_INVALID_ARG;
+  if (m <= 0 || n <= 0 || r_max <= 0 || !(sigma_cutoff >= 0.f)) return AB_ERR_INVALID_ARG;
+  if (!W || !A || !B || !sigma || !r_out) return AB_ERR_INVALID_ARG;
+  if ((m < n ? m : n) > 3072) return AB_ERR_UNSUPPORTED;
+  if (!ws || !aligned(ws, 256)) return AB_ERR_WORKSPACE;
+  if (!have_device()) return AB_ERR_CUDA;
+  SvdItem it;
+  it.W = W; it.w_dt = w_dt; it.m = m; it.n = n; it.r_max = r_max; it.A = A; it.B = B; it.out_dt = out_dt;
+  it.sigma = sigma; it.r_out = r_out; it.dev_status = dev_status;
+  return svd_batch(&it, 1, sigma_cutoff, ws, ws_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// Workspace of ab_group_sync: per matrix Abar, Bbar (fp32) and W (fp32), then the SVD batch.
+static size_t sync_layout(const ab_sync_desc* d, int L, int dt, void* ws, std::vector<float*>* Ab,
+                          std::vector<float*>* Bb, std::vector<float*>* Wd, std::vector<SvdItem>* items, void** svd_ws) {
+  Arena ar(ws, 0);
+  std::vector<SvdItem> loc(L);
+  for (int i = 0; i < L; ++i) {
+    float* a = ar.take_n<float>((size_t)d[i].m * d[i].r);
+    float* b = ar.take_n<float>((size_t)d[i].r * d[i].n);
+    float* w = ar.take_n<float>((size_t)d[i].m * d[i].n);
+    if (Ab) { (*Ab)[i] = a; (*Bb)[i] = b; (*Wd)[i] = w; }
+    SvdItem& it = loc[i];
+    it.W = w; it.w_dt = AB_F32; it.m = d[i].m; it.n = d[i].n; it.r_max = d[i].r;
+    it.A = d[i].A_out; it.B = d[i].B_out; it.out_dt = dt; it.sigma = d[i].sigma; it.r_out = d[i].r_out;
+    it.dev_status = nullptr;
+  }
+  void* sw = ar.take(0);
+  size_t svd_bytes = svd_batch_ws(loc.data(), L);
+  if (svd_ws) *svd_ws = sw;
+  if (items) *items = loc;
+  return align_up(ar.used, 256) + svd_bytes;
+}
+
+size_t ab_sync_workspace_bytes(const ab_sync_desc* descs, int L, int K, int dt) {
+  (void)K;
+  if (!descs || L <= 0) return 0;
+  return sync_layout(descs, L, dt, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr) + 256;
+}
+
+int ab_group_sync(const ab_sync_desc* descs, int L, int K, float sigma_cutoff, int dt,
+                  int* dev_status, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (!descs || L <= 0 || K < 1 || !dtype_ok(dt) || !(sigma_cutoff >= 0.f)) return AB_ERR_INVALID_ARG;
+  if (K > 64) return AB_ERR_UNSUPPORTED;
+  for (int i = 0; i < L; ++i) {
+    const ab_sync_desc& d = descs[i];
+    if (d.m <= 0 || d.n <= 0 || d.r <= 0 || d.r > d.m || d.r > d.n) return AB_ERR_INVALID_ARG;
+    if (!d.A_copies || !d.B_copies || !d.A_out || !d.B_out || !d.sigma || !d.r_out) return AB_ERR_INVALID_ARG;
+    if (K > 1 && (d.strideA < (int64_t)d.m * d.r || d.strideB < (int64_t)d.r * d.n)) return AB_ERR_INVALID_ARG;
+    if ((d.m < d.n ? d.m : d.n) > 3072) return AB_ERR_UNSUPPORTED;
+  }
+  if (!ws || !aligned(ws, 256)) return AB_ERR_WORKSPACE;
+  if (!have_device()) return AB_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  std::vector<float*> Ab(L), Bb(L), Wd(L);
+  std::vector<SvdItem> items;
+  void* svd_ws = nullptr;
+  size_t need = sync_layout(descs, L, dt, ws, &Ab, &Bb, &Wd, &items, &svd_ws);
+  if (need > ws_bytes) return AB_ERR_WORKSPACE;
+  for (int i = 0; i < L; ++i) {
+    const ab_sync_desc& d = descs[i];
+    AB_TRY(group_average(d.A_copies, d.strideA, K, (int64_t)d.m * d.r, dt, AB_F32, Ab[i], st));
+    AB_TRY(group_average(d.B_copies, d.strideB, K, (int64_t)d.r * d.n, dt, AB_F32, Bb[i], st));
+    AB_TRY(gemm_simt(Ab[i], AB_F32, d.r, 1, Bb[i], AB_F32, d.n, 1, Wd[i], AB_F32, d.n, d.m, d.n, d.r, st));
+    items[i].dev_status = dev_status ? dev_status + i : nullptr;
+  }
+  size_t used = static_cast<char*>(svd_ws) - static_cast<char*>(ws);
+  return svd_batch(items.data(), L, sigma_cutoff, svd_ws, ws_bytes - used, st);
+}
+
+}  // extern "C"

@@ -1,0 +1,131 @@
+// Group mean of K factor copies held in one device's memory: a pure HBM stream.
+// Each thread owns 16 input bytes per copy (4 fp32 or 8 bf16 values), keeps up to four copies'
+// loads in flight, adds them in fp32 in ascending k and scales by fl(1/K).  The sum order is
+// part of the contract (results are compared bit for bit).
+#include "ab_common.cuh"
+
+namespace ab {
+namespace {
+
+template <typename T> struct Vec;
+template <> struct Vec<float> {
+  static constexpr int N = 4;
+  __device__ static void load(const float* p, float (&v)[4]) {
+    float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  }
+};
+template <> struct Vec<bf16> {
+  static constexpr int N = 8;
+  __device__ static void load(const bf16* p, float (&v)[8]) {
+    uint4 t = __ldcs(reinterpret_cast<const uint4*>(p));
+    uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {   // a bf16 is the high half of the fp32 with the same value
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+};
+
+template <int N>
+__device__ __forceinline__ void store_vec(float* p, const float (&v)[N]) {
+#pragma unroll
+  for (int i = 0; i < N; i += 4) __stcs(reinterpret_cast<float4*>(p + i), make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
+}
+template <int N>
+__device__ __forceinline__ void store_vec(bf16* p, const float (&v)[N]) {
+  uint32_t w[N / 2];
+#pragma unroll
+  for (int i = 0; i < N / 2; ++i) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    w[i] = *reinterpret_cast<uint32_t*>(&h);
+  }
+  if constexpr (N == 8) __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
+  else __stcs(reinterpret_cast<uint2*>(p), make_uint2(w[0], w[1]));
+}
+
+template <typename TIn, typename TOut>
+__global__ void __launch_bounds__(256)
+average_vec_kernel(const TIn* __restrict__ base, int64_t stride, int K, int64_t nvec, float inv,
+                   TOut* __restrict__ out) {
+  constexpr int V = Vec<TIn>::N;
+  const int64_t step = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step) {
+    const TIn* p = base + i * V;
+    float s[V];
+    Vec<TIn>::load(p, s);
+    int k = 1;
+    for (; k + 3 <= K; k += 3) {       // three more copies in flight, added in ascending k
+      float a[V], b[V], c[V];
+      Vec<TIn>::load(p + (int64_t)k * stride, a);
+      Vec<TIn>::load(p + (int64_t)(k + 1) * stride, b);
+      Vec<TIn>::load(p + (int64_t)(k + 2) * stride, c);
+#pragma unroll
+      for (int j = 0; j < V; ++j) s[j] = __fadd_rn(__fadd_rn(__fadd_rn(s[j], a[j]), b[j]), c[j]);
+    }
+    for (; k < K; ++k) {
+      float a[V];
+      Vec<TIn>::load(p + (int64_t)k * stride, a);
+#pragma unroll
+      for (int j = 0; j < V; ++j) s[j] = __fadd_rn(s[j], a[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < V; ++j) s[j] = __fmul_rn(s[j], inv);
+    store_vec<V>(out + i * V, s);
+  }
+}
+
+// Any alignment, any count: one element per thread (also handles the ragged tail).
+template <typename TIn, typename TOut>
+__global__ void __launch_bounds__(256)
+average_scalar_kernel(const TIn* __restrict__ base, int64_t stride, int K, int64_t first, int64_t count,
+                      float inv, TOut* __restrict__ out) {
+  const int64_t step = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = first + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += step) {
+    float s = to_f32(base[i]);
+    for (int k = 1; k < K; ++k) s = __fadd_rn(s, to_f32(base[i + (int64_t)k * stride]));
+    from_f32(out[i], __fmul_rn(s, inv));
+  }
+}
+
+template <typename TIn, typename TOut>
+int run(const void* base_, int64_t stride, int K, int64_t count, void* out_, cudaStream_t st) {
+  const TIn* base = static_cast<const TIn*>(base_);
+  TOut* out = static_cast<TOut*>(out_);
+  constexpr int V = Vec<TIn>::N;
+  const float inv = 1.0f / (float)K;
+  const bool vec_ok = aligned(base, 16) && aligned(out, 16) && (stride % V == 0);
+  int64_t nvec = vec_ok ? count / V : 0;
+  int sms = 148;
+  if (nvec > 0) {
+    int64_t blocks = (nvec + 255) / 256;
+    int64_t cap = (int64_t)sms * 8;
+    unsigned grid = (unsigned)(blocks < cap ? blocks : cap);
+    average_vec_kernel<TIn, TOut><<<grid, 256, 0, st>>>(base, stride, K, nvec, inv, out);
+    AB_LAUNCH_OK();
+  }
+  int64_t first = nvec * V;
+  if (first < count) {
+    int64_t rest = count - first;
+    int64_t blocks = (rest + 255) / 256;
+    int64_t cap = (int64_t)sms * 8;
+    unsigned grid = (unsigned)(blocks < cap ? blocks : cap);
+    average_scalar_kernel<TIn, TOut><<<grid, 256, 0, st>>>(base, stride, K, first, count, inv, out);
+    AB_LAUNCH_OK();
+  }
+  return AB_OK;
+}
+
+}  // namespace
+
+int group_average(const void* base, int64_t stride_elems, int K, int64_t count,
+                  int in_dt, int out_dt, void* out, cudaStream_t st) {
+  if (count == 0) return AB_OK;
+  if (in_dt == AB_F32 && out_dt == AB_F32) return run<float, float>(base, stride_elems, K, count, out, st);
+  if (in_dt == AB_F32 && out_dt == AB_BF16) return run<float, bf16>(base, stride_elems, K, count, out, st);
+  if (in_dt == AB_BF16 && out_dt == AB_F32) return run<bf16, float>(base, stride_elems, K, count, out, st);
+  return run<bf16, bf16>(base, stride_elems, K, count, out, st);
+}
+
+}  // namespace ab

@@ -1,0 +1,101 @@
+// Shared declarations of the library's translation units (internal; the public surface is include/ab.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "ab.h"
+
+namespace ab {
+
+typedef __nv_bfloat16 bf16;
+
+#define AB_CUDA_OK(expr)                                   \
+  do {                                                     \
+    cudaError_t _e = (expr);                               \
+    if (_e != cudaSuccess) return AB_ERR_CUDA;             \
+  } while (0)
+
+#define AB_LAUNCH_OK()                                     \
+  do {                                                     \
+    if (cudaPeekAtLastError() != cudaSuccess) {            \
+      cudaGetLastError();                                  \
+      return AB_ERR_CUDA;                                  \
+    }                                                      \
+  } while (0)
+
+#define AB_TRY(expr)                                       \
+  do {                                                     \
+    int _s = (expr);                                       \
+    if (_s != AB_OK) return _s;                            \
+  } while (0)
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline size_t dtype_size(int dt) { return dt == AB_BF16 ? 2 : 4; }
+static inline bool dtype_ok(int dt) { return dt == AB_F32 || dt == AB_BF16; }
+static inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Carves 256-byte aligned pieces out of the caller's workspace.
+struct Arena {
+  char* base;
+  size_t used;
+  size_t cap;
+  Arena(void* p, size_t bytes) : base(static_cast<char*>(p)), used(0), cap(bytes) {}
+  void* take(size_t bytes) {
+    size_t off = align_up(used, 256);
+    used = off + bytes;
+    return base ? base + off : nullptr;
+  }
+  template <typename T> T* take_n(size_t n) { return static_cast<T*>(take(n * sizeof(T))); }
+  bool fits() const { return used <= cap; }
+};
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ void from_f32(float& d, float v) { d = v; }
+__device__ __forceinline__ void from_f32(bf16& d, float v) { d = __float2bfloat16_rn(v); }
+
+// ---- general strided GEMM on the plain fp32 pipes (ab_gemm_simt.cu) ----------------------------
+// C[i,j] = sum_k A(i,k) * B(k,j), A(i,k) at A + i*sAm + k*sAk, B(k,j) at B + k*sBk + j*sBn,
+// C row-major with row stride ldc.  fp32 accumulation, k ascending inside a thread: results
+// do not depend on the launch.  a_dt/b_dt/c_dt are ab_dtype values.
+int gemm_simt(const void* A, int a_dt, int64_t sAm, int64_t sAk,
+              const void* B, int b_dt, int64_t sBk, int64_t sBn,
+              void* C, int c_dt, int64_t ldc,
+              int64_t M, int64_t N, int64_t K, cudaStream_t st);
+
+// ---- fused tensor-core chain (ab_chain_tc.cu) --------------------------------------------------
+bool chain_tc_supported(int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
+                        const void* x, const void* A, const void* B, const void* y);
+size_t chain_tc_forward_ws(int64_t N, int m, int n, int r);
+size_t chain_tc_backward_ws(int64_t N, int m, int n, int r);
+int chain_tc_forward(const void* x, const void* A, const void* B, void* y, void* T_save,
+                     int64_t N, int m, int n, int r, int ldA, int ldB,
+                     void* ws, size_t ws_bytes, cudaStream_t st);
+int chain_tc_backward(const void* x, const void* dY, const void* A, const void* B,
+                      const void* T_saved, void* dX, float* dA, float* dB,
+                      int64_t N, int m, int n, int r, int ldA, int ldB,
+                      void* ws, size_t ws_bytes, cudaStream_t st);
+
+// ---- SVD pipeline (ab_svd.cu) ------------------------------------------------------------------
+struct SvdItem {
+  const void* W;     // dense m x n
+  int w_dt;
+  int m, n, r_max;
+  void* A;           // m x r_max
+  void* B;           // r_max x n
+  int out_dt;
+  float* sigma;
+  int* r_out;
+  int* dev_status;
+};
+size_t svd_batch_ws(const SvdItem* items, int L);
+int svd_batch(const SvdItem* items, int L, float sigma_cutoff, void* ws, size_t ws_bytes, cudaStream_t st);
+
+// ---- group mean (ab_average.cu) ----------------------------------------------------------------
+int group_average(const void* base, int64_t stride_elems, int K, int64_t count,
+                  int in_dt, int out_dt, void* out, cudaStream_t st);
+
+}  // namespace ab

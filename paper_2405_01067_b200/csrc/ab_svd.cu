@@ -1,0 +1,557 @@
+// Truncated SVD and sqrt-sigma split (Eq. 3 with the rank rule), batched over matrices.
+//
+// Route: Gram matrix of the shorter side, G = W^T W (m >= n) or W W^T (m < n) -- the paper's
+// "transpose when n > m" is this choice of side -- then a block one-sided Jacobi eigensolve on
+// X = G with the rotations accumulated in V^T, all in fp32:
+//   * vectors are stored as ROWS (X is s x s, V^T is s x s), split into blocks of b rows;
+//   * a sweep is nb-1 rounds of disjoint block pairs (round-robin); one CTA per pair keeps the
+//     2b x s panel in shared memory, forms its 2b x 2b Gram matrix M, diagonalises M with a
+//     parallel two-sided cyclic Jacobi (M, Q in shared memory), applies Q^T to the panel and
+//     to the matching panel of V^T;
+//   * sweeps repeat until no pair of rows has |x_i.x_j| > tol |x_i||x_j| (a device flag; the
+//     host enqueues a fixed number of sweeps and converged matrices return at once).
+// At convergence the rows of V^T are eigenvectors of G (singular vectors of the short side)
+// and |x_i| = sigma_i^2.  The long-side factor is W V_r (or V_r^T W) by a GEMM; sigma_i is
+// re-measured as the norm of that product, which makes A^T A = B B^T = diag(sigma) hold by
+// construction.  No wait in these kernels can spin: every loop has a fixed trip count.
+#include <vector>
+#include <algorithm>
+#include <map>
+
+#include "ab_common.cuh"
+
+namespace ab {
+namespace {
+
+struct JState {
+  int done;            // 1 once converged (or sweep cap reached)
+  unsigned off_bits;   // max relative off-orthogonality seen in the running sweep (float bits)
+  int sweeps;
+  unsigned maxn2_bits;      // largest squared row norm of the previous sweep (float bits)
+  unsigned next_maxn2_bits; // the same, being collected in the running sweep
+  int status;
+};
+
+constexpr int kMaxSweeps = 14;
+constexpr int kInnerSweeps = 10;
+constexpr float kDeadRel2 = 1e-12f;   // rows below 1e-6 of the largest norm count as zero
+
+__host__ __device__ inline float jacobi_tol(int s) {
+  float t = 2e-7f * sqrtf((float)s);
+  return t < 2e-6f ? 2e-6f : t;
+}
+
+__global__ void init_state_kernel(float* __restrict__ Vt, JState* __restrict__ st, int s, int count) {
+  const int mat = blockIdx.y;
+  float* V = Vt + (size_t)mat * s * s;
+  const size_t total = (size_t)s * s;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x)
+    V[i] = (i / s == i % s) ? 1.f : 0.f;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    JState z;
+    z.done = 0; z.off_bits = 0; z.sweeps = 0; z.maxn2_bits = 0; z.next_maxn2_bits = 0; z.status = AB_OK;
+    st[mat] = z;
+  }
+}
+
+__global__ void sweep_end_kernel(JState* __restrict__ st, int count, float tol) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  JState z = st[i];
+  if (z.done) return;
+  z.sweeps += 1;
+  if (__uint_as_float(z.off_bits) <= tol) z.done = 1;
+  else if (z.sweeps >= kMaxSweeps) { z.done = 1; z.status = AB_ERR_NOT_CONVERGED; }
+  z.off_bits = 0;
+  if (z.next_maxn2_bits) z.maxn2_bits = z.next_maxn2_bits;
+  z.next_maxn2_bits = 0;
+  st[i] = z;
+}
+
+// Index pair k of round t in a round-robin over an even number `ne` of players.
+__device__ __forceinline__ void rr_pair(int ne, int t, int k, int& p, int& q) {
+  const int n1 = ne - 1;
+  if (k == 0) { p = n1; q = t % n1; }
+  else { p = (t + k) % n1; q = (t - k + n1) % n1; }
+  if (p > q) { int tmp = p; p = q; q = tmp; }
+}
+
+template <int PB>
+__global__ void __launch_bounds__(256)
+jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, int nb, int round,
+                   float tol, JState* __restrict__ states) {
+  constexpr int HB = PB / 2;          // rows per block
+  constexpr int RT = PB / 16;         // register tile of the panel Gram
+  constexpr int LDM = PB + 1;
+  extern __shared__ __align__(16) float smem[];
+  const int mat = blockIdx.y;
+  JState* st = states + mat;
+  if (st->done) return;
+  const int nbe = nb + (nb & 1);
+  int bi, bj;
+  rr_pair(nbe, round, blockIdx.x, bi, bj);
+  if (bj >= nb && nb > 1) return;     // this block sits the round out
+  const int ldp = ((s + 3) & ~3) + 4;
+  float* P = smem;                    // PB x ldp
+  float* Ms = P + (size_t)PB * ldp;   // PB x LDM
+  float* Qt = Ms + PB * LDM;          // PB x PB, Qt[c][i] = Q[i][c]
+  float* cs = Qt + PB * PB;           // HB
+  float* sn = cs + HB;                // HB
+  int* pq = reinterpret_cast<int*>(sn + HB);   // 2*HB
+  __shared__ int any_rot;
+  const int tid = threadIdx.x;
+  float* X = Xall + (size_t)mat * s * s;
+  float* V = Vall + (size_t)mat * s * s;
+  const float maxn2 = __uint_as_float(st->maxn2_bits);
+  const float dead2 = kDeadRel2 * maxn2;
+
+  auto grow = [&](int lr) -> int {    // local panel row -> global row (or -1)
+    int g = (lr < HB) ? bi * HB + lr : bj * HB + (lr - HB);
+    if (lr >= HB && bj >= nb) return -1;
+    return g < s ? g : -1;
+  };
+  auto load_panel = [&](const float* src) {
+    const int s4 = ldp - 4;           // padded row length handled, multiple of 4
+    for (int idx = tid; idx < PB * s4; idx += 256) {
+      int lr = idx / s4, k = idx - lr * s4;
+      int g = grow(lr);
+      P[(size_t)lr * ldp + k] = (g >= 0 && k < s) ? src[(size_t)g * s + k] : 0.f;
+    }
+  };
+  auto store_panel = [&](float* dst) {
+    for (int idx = tid; idx < PB * s; idx += 256) {
+      int lr = idx / s, k = idx - lr * s;
+      int g = grow(lr);
+      if (g >= 0) dst[(size_t)g * s + k] = P[(size_t)lr * ldp + k];
+    }
+  };
+  auto apply_q = [&]() {              // P <- Q^T P, one panel column per thread at a time
+    for (int k = tid; k < s; k += 256) {
+      float col[PB];
+#pragma unroll
+      for (int j = 0; j < PB; ++j) col[j] = P[(size_t)j * ldp + k];
+      for (int i = 0; i < PB; ++i) {
+        const float4* qrow = reinterpret_cast<const float4*>(Qt + i * PB);
+        float acc = 0.f;
+#pragma unroll
+        for (int j4 = 0; j4 < PB / 4; ++j4) {
+          float4 q4 = qrow[j4];
+          acc = fmaf(q4.x, col[4 * j4], acc);
+          acc = fmaf(q4.y, col[4 * j4 + 1], acc);
+          acc = fmaf(q4.z, col[4 * j4 + 2], acc);
+          acc = fmaf(q4.w, col[4 * j4 + 3], acc);
+        }
+        P[(size_t)i * ldp + k] = acc;
+      }
+    }
+  };
+
+  load_panel(X);
+  for (int idx = tid; idx < PB * PB; idx += 256) Qt[idx] = (idx / PB == idx % PB) ? 1.f : 0.f;
+  if (tid == 0) any_rot = 0;
+  __syncthreads();
+
+  // ---- M = P P^T
+  {
+    const int tx = tid & 15, ty = tid >> 4;
+    float acc[RT][RT];
+#pragma unroll
+    for (int i = 0; i < RT; ++i)
+#pragma unroll
+      for (int j = 0; j < RT; ++j) acc[i][j] = 0.f;
+    const int s4 = ldp - 4;
+    for (int k = 0; k < s4; k += 4) {
+      float4 a[RT], b[RT];
+#pragma unroll
+      for (int i = 0; i < RT; ++i) a[i] = *reinterpret_cast<const float4*>(P + (size_t)(ty + 16 * i) * ldp + k);
+#pragma unroll
+      for (int j = 0; j < RT; ++j) b[j] = *reinterpret_cast<const float4*>(P + (size_t)(tx + 16 * j) * ldp + k);
+#pragma unroll
+      for (int i = 0; i < RT; ++i)
+#pragma unroll
+        for (int j = 0; j < RT; ++j) {
+          acc[i][j] = fmaf(a[i].x, b[j].x, acc[i][j]);
+          acc[i][j] = fmaf(a[i].y, b[j].y, acc[i][j]);
+          acc[i][j] = fmaf(a[i].z, b[j].z, acc[i][j]);
+          acc[i][j] = fmaf(a[i].w, b[j].w, acc[i][j]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < RT; ++i)
+#pragma unroll
+      for (int j = 0; j < RT; ++j) Ms[(ty + 16 * i) * LDM + tx + 16 * j] = acc[i][j];
+  }
+  __syncthreads();
+
+  // ---- how far from orthogonal is this panel?  (also collects the largest squared norm)
+  {
+    float worst = 0.f, big = 0.f;
+    for (int idx = tid; idx < PB * PB; idx += 256) {
+      int i = idx / PB, j = idx - i * PB;
+      float mii = Ms[i * LDM + i], mjj = Ms[j * LDM + j];
+      if (i == j) { big = fmaxf(big, mii); continue; }
+      if (i < j && mii > dead2 && mjj > dead2 && mii > 0.f && mjj > 0.f) {
+        float rel = fabsf(Ms[i * LDM + j]) / (sqrtf(mii) * sqrtf(mjj));
+        worst = fmaxf(worst, rel);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      worst = fmaxf(worst, __shfl_xor_sync(0xffffffffu, worst, o));
+      big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, o));
+    }
+    if ((tid & 31) == 0) {
+      atomicMax(&st->off_bits, __float_as_uint(worst));
+      atomicMax(&st->next_maxn2_bits, __float_as_uint(big));
+      if (worst > tol) atomicExch(&any_rot, 1);
+    }
+  }
+  __syncthreads();
+  if (!any_rot) return;               // panel already orthogonal: nothing to write
+  __syncthreads();
+
+  // ---- diagonalise M: parallel cyclic two-sided Jacobi, HB disjoint rotations per step
+  for (int sweep = 0; sweep < kInnerSweeps; ++sweep) {
+    if (tid == 0) any_rot = 0;
+    __syncthreads();
+    for (int t = 0; t < PB - 1; ++t) {
+      if (tid < HB) {
+        int p, q;
+        rr_pair(PB, t, tid, p, q);
+        float app = Ms[p * LDM + p], aqq = Ms[q * LDM + q], apq = Ms[p * LDM + q];
+        float c = 1.f, sv = 0.f;
+        if (app > dead2 && aqq > dead2 && app > 0.f && aqq > 0.f &&
+            fabsf(apq) > 0.25f * tol * sqrtf(app) * sqrtf(aqq)) {
+          float zeta = (aqq - app) / (2.f * apq);
+          float tt = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
+          c = rsqrtf(1.f + tt * tt);
+          sv = c * tt;
+          any_rot = 1;
+        }
+        cs[tid] = c; sn[tid] = sv; pq[2 * tid] = p; pq[2 * tid + 1] = q;
+      }
+      __syncthreads();
+      // 2x2 blocks of M (rows of pair a, columns of pair b), then rows of Qt
+      for (int task = tid; task < HB * HB + PB * HB; task += 256) {
+        if (task < HB * HB) {
+          int a = task / HB, b = task - a * HB;
+          int pa = pq[2 * a], qa = pq[2 * a + 1], pb = pq[2 * b], qb = pq[2 * b + 1];
+          float ca = cs[a], sa = sn[a], cb = cs[b], sb = sn[b];
+          float m00 = Ms[pa * LDM + pb], m01 = Ms[pa * LDM + qb];
+          float m10 = Ms[qa * LDM + pb], m11 = Ms[qa * LDM + qb];
+          float n00 = cb * m00 - sb * m01, n01 = sb * m00 + cb * m01;
+          float n10 = cb * m10 - sb * m11, n11 = sb * m10 + cb * m11;
+          float r00 = ca * n00 - sa * n10, r10 = sa * n00 + ca * n10;
+          float r01 = ca * n01 - sa * n11, r11 = sa * n01 + ca * n11;
+          if (a == b && sa != 0.f) { r01 = 0.f; r10 = 0.f; }
+          Ms[pa * LDM + pb] = r00; Ms[pa * LDM + qb] = r01;
+          Ms[qa * LDM + pb] = r10; Ms[qa * LDM + qb] = r11;
+        } else {
+          int u = task - HB * HB;
+          int b = u / PB, i = u - b * PB;
+          int pb = pq[2 * b], qb = pq[2 * b + 1];
+          float cb = cs[b], sb = sn[b];
+          float q0 = Qt[pb * PB + i], q1 = Qt[qb * PB + i];
+          Qt[pb * PB + i] = cb * q0 - sb * q1;
+          Qt[qb * PB + i] = sb * q0 + cb * q1;
+        }
+      }
+      __syncthreads();
+    }
+    if (!any_rot) break;              // uniform: read after the step's barrier
+    __syncthreads();
+  }
+
+  // ---- rotate the panel of X, then the same rows of V^T
+  apply_q();
+  __syncthreads();
+  store_panel(X);
+  __syncthreads();
+  load_panel(V);
+  __syncthreads();
+  apply_q();
+  __syncthreads();
+  store_panel(V);
+}
+
+template <int PB>
+size_t jacobi_smem_bytes(int s) {
+  const int ldp = ((s + 3) & ~3) + 4;
+  return sizeof(float) * ((size_t)PB * ldp + (size_t)PB * (PB + 1) + (size_t)PB * PB + PB) + sizeof(int) * PB;
+}
+
+// lam[i] = |row i of X|, perm = indices by descending lam (ties by index).  One CTA per matrix.
+__global__ void __launch_bounds__(256)
+norms_sort_kernel(const float* __restrict__ Xall, int s, float* __restrict__ lam_all, int* __restrict__ perm_all) {
+  extern __shared__ float lam_s[];
+  const int mat = blockIdx.x;
+  const float* X = Xall + (size_t)mat * s * s;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int i = warp; i < s; i += 8) {
+    double acc = 0.0;
+    for (int k = lane; k < s; k += 32) { float v = X[(size_t)i * s + k]; acc += (double)v * v; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) lam_s[i] = (float)sqrt(acc);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < s; i += 256) {
+    float li = lam_s[i];
+    int rank = 0;
+    for (int j = 0; j < s; ++j) {
+      float lj = lam_s[j];
+      rank += (lj > li) || (lj == li && j < i);
+    }
+    perm_all[(size_t)mat * s + rank] = i;
+    lam_all[(size_t)mat * s + i] = li;
+  }
+}
+
+// Vr[k][:] = Vt[perm[k]][:], k < r_cap
+__global__ void gather_rows_kernel(const float* __restrict__ Vt, const int* __restrict__ perm, int s, int r_cap,
+                                   float* __restrict__ Vr) {
+  const int k = blockIdx.x;
+  if (k >= r_cap) return;
+  const float* src = Vt + (size_t)perm[k] * s;
+  for (int u = threadIdx.x; u < s; u += blockDim.x) Vr[(size_t)k * s + u] = src[u];
+}
+
+// sigma[k] = norm over t of Ylong(k,t), Ylong(k,t) = Y[t*st_ + k*sk].  32 values of k per CTA.
+__global__ void __launch_bounds__(256)
+long_norms_kernel(const float* __restrict__ Y, int64_t st_, int64_t sk, int L, int r_cap, float* __restrict__ sigma) {
+  __shared__ double red[8][33];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (sk == 1) {                      // neighbouring k adjacent in memory: lane = k, warps stride over t
+    const int k = blockIdx.x * 32 + lane;
+    double acc = 0.0;
+    if (k < r_cap)
+      for (int t = warp; t < L; t += 8) { float v = Y[(int64_t)t * st_ + k]; acc += (double)v * v; }
+    red[warp][lane] = acc;
+    __syncthreads();
+    if (warp == 0 && k < r_cap) {
+      double t = 0.0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t += red[i][lane];
+      sigma[k] = (float)sqrt(t);
+    }
+  } else {                            // neighbouring t adjacent: one warp walks one k
+    for (int kk = warp; kk < 32; kk += 8) {
+      const int k = blockIdx.x * 32 + kk;
+      if (k >= r_cap) continue;
+      double acc = 0.0;
+      for (int t = lane; t < L; t += 32) { float v = Y[(int64_t)t * st_ + (int64_t)k * sk]; acc += (double)v * v; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (lane == 0) sigma[k] = (float)sqrt(acc);
+    }
+  }
+}
+
+__global__ void rank_rule_kernel(const float* __restrict__ sigma, int r_cap, float cutoff, int* __restrict__ r_out,
+                                 const JState* __restrict__ st, int* __restrict__ dev_status) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  float top = 0.f;
+  for (int k = 0; k < r_cap; ++k) top = fmaxf(top, sigma[k]);
+  const float thr = cutoff * top;
+  int keep = 0;
+  for (int k = 0; k < r_cap; ++k) keep += (sigma[k] >= thr) ? 1 : 0;
+  if (keep < 1) keep = 1;
+  *r_out = keep;
+  if (dev_status) *dev_status = st->status;
+}
+
+// long factor: F(t,k) = Ylong(k,t) / sqrt(sigma_k); short factor: F(k,u) = sqrt(sigma_k) Vr[k][u].
+// Columns/rows k >= r' (and k >= r_cap) are written as zero.
+template <typename TO>
+__global__ void write_factors_kernel(const float* __restrict__ Y, int64_t yt, int64_t yk,
+                                     const float* __restrict__ Vr, const float* __restrict__ sigma,
+                                     const int* __restrict__ r_out, int L, int s, int r_cap, int r_max,
+                                     TO* __restrict__ Flong, int64_t lt, int64_t lk,
+                                     TO* __restrict__ Fshort, int64_t sk_, int64_t su) {
+  const int rk = *r_out;
+  const int64_t nlong = (int64_t)L * r_max, nshort = (int64_t)s * r_max;
+  const int64_t step = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < nlong + nshort; idx += step) {
+    if (idx < nlong) {
+      // walk the long factor in its own memory order
+      int64_t t, k;
+      if (lk == 1) { t = idx / r_max; k = idx - t * r_max; } else { k = idx / L; t = idx - k * L; }
+      float v = 0.f;
+      if (k < rk && k < r_cap) {
+        float sg = sigma[k];
+        v = sg > 0.f ? Y[t * yt + k * yk] * rsqrtf(sg) : 0.f;
+      }
+      from_f32(Flong[t * lt + k * lk], v);
+    } else {
+      int64_t j = idx - nlong, k, u;
+      if (su == 1) { k = j / s; u = j - k * s; } else { u = j / r_max; k = j - u * r_max; }
+      float v = 0.f;
+      if (k < rk && k < r_cap) v = sqrtf(sigma[k]) * Vr[k * (int64_t)s + u];
+      from_f32(Fshort[k * sk_ + u * su], v);
+    }
+  }
+}
+
+struct Plan {
+  int s, L, r_cap, pb, nb;
+  bool tall;           // m >= n
+};
+
+Plan make_plan(const SvdItem& it) {
+  Plan p;
+  p.tall = it.m >= it.n;
+  p.s = p.tall ? it.n : it.m;
+  p.L = p.tall ? it.m : it.n;
+  p.r_cap = std::min(it.r_max, p.s);
+  p.pb = p.s <= 768 ? 64 : (p.s <= 1536 ? 32 : 16);
+  int hb = p.pb / 2;
+  p.nb = (p.s + hb - 1) / hb;
+  return p;
+}
+
+struct ItemWs {
+  float *lam, *Vr, *Y, *Wf;
+  int* perm;
+};
+
+// Lays out the workspace: per group (equal s) X, Vt and states; per item the rest.
+struct Layout {
+  std::map<int, std::vector<int>> groups;     // s -> item indices
+  std::map<int, float*> X, Vt;
+  std::map<int, JState*> st;
+  std::vector<ItemWs> item;
+  size_t bytes;
+};
+
+Layout make_layout(const SvdItem* items, int L, void* ws) {
+  Layout lo;
+  Arena ar(ws, 0);
+  for (int i = 0; i < L; ++i) lo.groups[make_plan(items[i]).s].push_back(i);
+  for (auto& g : lo.groups) {
+    size_t s = (size_t)g.first, cnt = g.second.size();
+    lo.X[g.first] = ar.take_n<float>(cnt * s * s);
+    lo.Vt[g.first] = ar.take_n<float>(cnt * s * s);
+    lo.st[g.first] = ar.take_n<JState>(cnt);
+  }
+  lo.item.resize(L);
+  for (int i = 0; i < L; ++i) {
+    Plan p = make_plan(items[i]);
+    lo.item[i].lam = nullptr;
+    lo.item[i].perm = nullptr;
+    lo.item[i].Vr = ar.take_n<float>((size_t)p.r_cap * p.s);
+    lo.item[i].Y = ar.take_n<float>((size_t)p.L * p.r_cap);
+    lo.item[i].Wf = nullptr;
+  }
+  for (auto& g : lo.groups) {   // lam/perm are group-contiguous (one sort launch per group)
+    size_t s = (size_t)g.first, cnt = g.second.size();
+    float* lam = ar.take_n<float>(cnt * s);
+    int* perm = ar.take_n<int>(cnt * s);
+    for (size_t j = 0; j < cnt; ++j) {
+      lo.item[g.second[j]].lam = lam ? lam + j * s : nullptr;
+      lo.item[g.second[j]].perm = perm ? perm + j * s : nullptr;
+    }
+  }
+  lo.bytes = align_up(ar.used, 256);
+  return lo;
+}
+
+template <int PB>
+int run_jacobi(float* X, float* Vt, JState* st, int s, int nb, int count, cudaStream_t stream) {
+  const size_t smem = jacobi_smem_bytes<PB>(s);
+  if (smem > 227 * 1024) return AB_ERR_UNSUPPORTED;
+  AB_CUDA_OK(cudaFuncSetAttribute(jacobi_pair_kernel<PB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const int nbe = nb + (nb & 1);
+  const int rounds = nbe > 2 ? nbe - 1 : 1;
+  const float tol = jacobi_tol(s);
+  dim3 grid((unsigned)(nbe / 2), (unsigned)count);
+  for (int sw = 0; sw < kMaxSweeps; ++sw) {
+    for (int r = 0; r < rounds; ++r) {
+      jacobi_pair_kernel<PB><<<grid, 256, smem, stream>>>(X, Vt, s, nb, r, tol, st);
+    }
+    sweep_end_kernel<<<(count + 127) / 128, 128, 0, stream>>>(st, count, tol);
+  }
+  AB_LAUNCH_OK();
+  return AB_OK;
+}
+
+}  // namespace
+
+size_t svd_batch_ws(const SvdItem* items, int L) {
+  return make_layout(items, L, nullptr).bytes;
+}
+
+int svd_batch(const SvdItem* items, int L, float sigma_cutoff, void* ws, size_t ws_bytes, cudaStream_t stream) {
+  Layout lo = make_layout(items, L, ws);
+  if (lo.bytes > ws_bytes) return AB_ERR_WORKSPACE;
+  // 1. Gram matrices into X
+  for (auto& g : lo.groups) {
+    const int s = g.first;
+    for (size_t j = 0; j < g.second.size(); ++j) {
+      const SvdItem& it = items[g.second[j]];
+      float* G = lo.X[s] + j * (size_t)s * s;
+      if (it.m >= it.n)   // G = W^T W
+        AB_TRY(gemm_simt(it.W, it.w_dt, 1, it.n, it.W, it.w_dt, it.n, 1, G, AB_F32, s, s, s, it.m, stream));
+      else                // G = W W^T
+        AB_TRY(gemm_simt(it.W, it.w_dt, it.n, 1, it.W, it.w_dt, 1, it.n, G, AB_F32, s, s, s, it.n, stream));
+    }
+  }
+  // 2. eigen-decomposition of every group
+  for (auto& g : lo.groups) {
+    const int s = g.first, count = (int)g.second.size();
+    Plan p = make_plan(items[g.second[0]]);
+    dim3 ig(64, (unsigned)count);
+    init_state_kernel<<<ig, 256, 0, stream>>>(lo.Vt[s], lo.st[s], s, count);
+    AB_LAUNCH_OK();
+    int rc;
+    if (p.pb == 64) rc = run_jacobi<64>(lo.X[s], lo.Vt[s], lo.st[s], s, p.nb, count, stream);
+    else if (p.pb == 32) rc = run_jacobi<32>(lo.X[s], lo.Vt[s], lo.st[s], s, p.nb, count, stream);
+    else rc = run_jacobi<16>(lo.X[s], lo.Vt[s], lo.st[s], s, p.nb, count, stream);
+    AB_TRY(rc);
+    norms_sort_kernel<<<count, 256, (size_t)s * sizeof(float), stream>>>(
+        lo.X[s], s, lo.item[g.second[0]].lam, lo.item[g.second[0]].perm);
+    AB_LAUNCH_OK();
+  }
+  // 3. per matrix: leading vectors, long-side product, sigma, rank rule, factors
+  for (auto& g : lo.groups) {
+    const int s = g.first;
+    for (size_t j = 0; j < g.second.size(); ++j) {
+      const int i = g.second[j];
+      const SvdItem& it = items[i];
+      Plan p = make_plan(it);
+      const ItemWs& w = lo.item[i];
+      const float* Vt = lo.Vt[s] + j * (size_t)s * s;
+      gather_rows_kernel<<<p.r_cap, 256, 0, stream>>>(Vt, w.perm, s, p.r_cap, w.Vr);
+      AB_LAUNCH_OK();
+      int64_t yt, yk;   // Ylong(k,t) = Y[t*yt + k*yk]
+      if (p.tall) {     // Y (m x r_cap) = W Vr^T
+        AB_TRY(gemm_simt(it.W, it.w_dt, it.n, 1, w.Vr, AB_F32, 1, s, w.Y, AB_F32, p.r_cap, it.m, p.r_cap, it.n, stream));
+        yt = p.r_cap; yk = 1;
+      } else {          // Y (r_cap x n) = Vr W
+        AB_TRY(gemm_simt(w.Vr, AB_F32, s, 1, it.W, it.w_dt, it.n, 1, w.Y, AB_F32, it.n, p.r_cap, it.n, it.m, stream));
+        yt = 1; yk = it.n;
+      }
+      long_norms_kernel<<<(p.r_cap + 31) / 32, 256, 0, stream>>>(w.Y, yt, yk, p.L, p.r_cap, it.sigma);
+      AB_LAUNCH_OK();
+      rank_rule_kernel<<<1, 32, 0, stream>>>(it.sigma, p.r_cap, sigma_cutoff, it.r_out, lo.st[s] + j, it.dev_status);
+      AB_LAUNCH_OK();
+      // tall: A is the long factor (A[t][k], strides r_max, 1), B the short one (B[k][u], strides n, 1)
+      // wide: B is the long factor (B[k][t], strides 1, n),     A the short one (A[u][k]: k stride 1, u stride r_max)
+      void* Fl = p.tall ? it.A : it.B;
+      void* Fs = p.tall ? it.B : it.A;
+      int64_t lt = p.tall ? it.r_max : 1, lk = p.tall ? 1 : it.n;
+      int64_t sk = p.tall ? it.n : 1, su = p.tall ? 1 : it.r_max;
+      int64_t total = (int64_t)(p.L + s) * it.r_max;
+      unsigned grid = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8);
+      if (it.out_dt == AB_F32)
+        write_factors_kernel<float><<<grid, 256, 0, stream>>>(w.Y, yt, yk, w.Vr, it.sigma, it.r_out, p.L, s, p.r_cap,
+                                                             it.r_max, (float*)Fl, lt, lk, (float*)Fs, sk, su);
+      else
+        write_factors_kernel<bf16><<<grid, 256, 0, stream>>>(w.Y, yt, yk, w.Vr, it.sigma, it.r_out, p.L, s, p.r_cap,
+                                                            it.r_max, (bf16*)Fl, lt, lk, (bf16*)Fs, sk, su);
+      AB_LAUNCH_OK();
+    }
+  }
+  return AB_OK;
+}
+
+}  // namespace ab

@@ -1,0 +1,321 @@
+"""CUDA path against the CPU checker on the same seeded inputs, through the C-ABI.
+
+Tolerances: bf16 storage / fp32 accumulation, relative Frobenius error <= 2e-2; fp32 paths
+<= 1e-4; singular values within 1e-4 relative; ||A B - W_r||_F / ||W||_F <= 1e-4 (sign
+invariant: factors are never compared element by element); the group mean bit for bit.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ab_oracle as orc
+from paper_2405_01067_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+TOL_F32 = 1e-4
+
+
+@pytest.fixture(scope="module")
+def ab():
+    from paper_2405_01067_b200 import binding
+    binding.lib()
+    return binding
+
+
+def dev(a, bf16=False):
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+    return t.to(torch.bfloat16) if bf16 else t
+
+
+def host(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def run_chain(ab, d, bf16, save_T):
+    x, dY, A, B = (dev(d[k], bf16) for k in ("x", "dY", "A", "B"))
+    y, T = ab.ab_layer_forward(x, A, B, save_T=save_T)
+    dX, dA, dB = ab.ab_layer_backward(x, dY, A, B, T_saved=T)
+    torch.cuda.synchronize()
+    return host(y), (host(T) if T is not None else None), host(dX), host(dA), host(dB)
+
+
+def check_chain(ab, d, bf16, save_T=False):
+    tol = TOL_BF16 if bf16 else TOL_F32
+    y, T, dX, dA, dB = run_chain(ab, d, bf16, save_T)
+    T_ref, y_ref = orc.forward(d["x"], d["A"], d["B"])
+    dX_ref, dA_ref, dB_ref, _ = orc.backward(d["x"], d["dY"], d["A"], d["B"])
+    errs = dict(y=orc.rel_frob(y, y_ref), dX=orc.rel_frob(dX, dX_ref), dA=orc.rel_frob(dA, dA_ref),
+                dB=orc.rel_frob(dB, dB_ref))
+    if T is not None:
+        errs["T"] = orc.rel_frob(T, T_ref)
+    for k, v in errs.items():
+        assert v <= tol, (k, v, errs)
+    return errs
+
+
+# ------------------------------------------------------------------ chain: small and ragged shapes
+
+@pytest.mark.parametrize("N,m,n,r", [(64, 256, 512, 32), (1, 1, 1, 1), (37, 19, 23, 5), (130, 70, 66, 33),
+                                     (200, 96, 160, 31), (129, 64, 64, 64)])
+@pytest.mark.parametrize("save_T", [False, True])
+def test_chain_fp32(ab, N, m, n, r, save_T):
+    d = synth.chain_case(100 + N + m, m, n, r, N, bf16=False)
+    check_chain(ab, d, False, save_T)
+
+
+@pytest.mark.parametrize("N,m,n,r", [(300, 256, 128, 32), (257, 384, 512, 192), (1000, 768, 256, 256),
+                                     (77, 40, 56, 8), (513, 136, 264, 48), (128, 128, 128, 16),
+                                     (640, 512, 1024, 64), (100, 50, 70, 7)])
+@pytest.mark.parametrize("save_T", [False, True])
+def test_chain_bf16(ab, N, m, n, r, save_T):
+    d = synth.chain_case(200 + N + r, m, n, r, N, bf16=True)
+    check_chain(ab, d, True, save_T)
+
+
+def test_chain_strided_factors(ab):
+    d = synth.chain_case(5, 96, 80, 24, 150, bf16=False)
+    Abig = torch.zeros((96, 40), device="cuda")
+    Bbig = torch.zeros((24, 100), device="cuda")
+    Abig[:, :24] = dev(d["A"])
+    Bbig[:, :80] = dev(d["B"])
+    x, dY = dev(d["x"]), dev(d["dY"])
+    L = ab.lib()
+    y = torch.empty((150, 96), device="cuda")
+    ws = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_FORWARD, 150, 96, 80, 24), "cuda")
+    st = L.ab_layer_forward(x.data_ptr(), Abig.data_ptr(), Bbig.data_ptr(), y.data_ptr(), None, 150, 96, 80, 24,
+                            40, 100, 0, ws.data_ptr(), ws.numel(), None)
+    assert st == 0
+    torch.cuda.synchronize()
+    assert orc.rel_frob(host(y), orc.forward(d["x"], d["A"], d["B"])[1]) <= TOL_F32
+
+
+def test_backward_optional_outputs_and_determinism(ab):
+    d = synth.chain_case(9, 256, 384, 64, 700, bf16=True)
+    x, dY, A, B = (dev(d[k], True) for k in ("x", "dY", "A", "B"))
+    full = ab.ab_layer_backward(x, dY, A, B)
+    only_b = ab.ab_layer_backward(x, dY, A, B, want=("dX", "dB"))
+    only_a = ab.ab_layer_backward(x, dY, A, B, want=("dA",))
+    again = ab.ab_layer_backward(x, dY, A, B)
+    torch.cuda.synchronize()
+    assert only_b[1] is None and only_a[0] is None and only_a[2] is None
+    assert torch.equal(full[0], only_b[0]) and torch.equal(full[2], only_b[2]) and torch.equal(full[1], only_a[1])
+    for a, b in zip(full, again):
+        assert torch.equal(a, b)       # fixed reduction order: identical bits
+
+
+def test_empty_batch(ab):
+    A = torch.randn(8, 2, device="cuda")
+    B = torch.randn(2, 6, device="cuda")
+    x = torch.empty((0, 6), device="cuda")
+    dY = torch.empty((0, 8), device="cuda")
+    y, _ = ab.ab_layer_forward(x, A, B)
+    dX, dA, dB = ab.ab_layer_backward(x, dY, A, B)
+    torch.cuda.synchronize()
+    assert y.shape == (0, 8) and dX.shape == (0, 6)
+    assert torch.count_nonzero(dA) == 0 and torch.count_nonzero(dB) == 0
+
+
+# ------------------------------------------------------------------ group mean: bit for bit
+
+@pytest.mark.parametrize("K", [1, 2, 3, 4, 8, 13])
+@pytest.mark.parametrize("count", [1, 7, 1024, 4096 + 5, 1 << 20])
+@pytest.mark.parametrize("in_bf16,out_bf16", [(False, False), (True, False), (True, True), (False, True)])
+def test_group_average_bit_exact(ab, K, count, in_bf16, out_bf16):
+    rng = np.random.default_rng(K * 1000 + count % 977)
+    c = rng.standard_normal((K, count)).astype(np.float32)
+    if in_bf16:
+        c = synth.bf16_round(c)
+    out = ab.ab_group_average(dev(c, in_bf16), out_dtype=torch.bfloat16 if out_bf16 else torch.float32)
+    torch.cuda.synchronize()
+    ref = orc.group_average_f32(c)
+    if out_bf16:
+        ref = synth.bf16_round(ref)
+    got = out.float().cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+
+
+def test_group_average_strided_and_unaligned(ab):
+    K, count = 4, 1003
+    rng = np.random.default_rng(3)
+    arena = torch.from_numpy(rng.standard_normal(K * 1100 + 16).astype(np.float32)).cuda()
+    L = ab.lib()
+    out = torch.empty(count + 1, device="cuda")
+    for off in (0, 1, 3):   # base not 16-byte aligned: the scalar kernel takes over
+        st = L.ab_group_average(arena.data_ptr() + 4 * off, 1100, K, count, 0, 0, out.data_ptr() + 4 * (off % 2), None)
+        assert st == 0
+        torch.cuda.synchronize()
+        h = arena.cpu().numpy()
+        c = np.stack([h[off + k * 1100: off + k * 1100 + count] for k in range(K)])
+        got = out.cpu().numpy()[off % 2: off % 2 + count]
+        assert np.array_equal(got.view(np.uint32), orc.group_average_f32(c).view(np.uint32))
+
+
+def test_group_average_empty(ab):
+    c = torch.empty((3, 0), device="cuda")
+    assert ab.ab_group_average(c).numel() == 0
+
+
+# ------------------------------------------------------------------ recombine
+
+@pytest.mark.parametrize("m,n,r", [(256, 512, 32), (1, 1, 1), (70, 130, 33), (768, 768, 192), (65, 63, 17)])
+def test_recombine(ab, m, n, r):
+    rng = np.random.default_rng(m + n + r)
+    A = rng.standard_normal((m, r)).astype(np.float32)
+    B = rng.standard_normal((r, n)).astype(np.float32)
+    W = ab.ab_recombine(dev(A), dev(B))
+    torch.cuda.synchronize()
+    assert orc.rel_frob(host(W), orc.recombine(A, B)) <= 1e-6
+
+
+def test_recombine_bf16_factors(ab):
+    rng = np.random.default_rng(1)
+    A = synth.bf16_round(rng.standard_normal((100, 24)).astype(np.float32))
+    B = synth.bf16_round(rng.standard_normal((24, 90)).astype(np.float32))
+    W = ab.ab_recombine(dev(A, True), dev(B, True))
+    torch.cuda.synchronize()
+    assert orc.rel_frob(host(W), orc.recombine(A, B)) <= 1e-6
+
+
+# ------------------------------------------------------------------ SVD split
+
+def check_split(ab, W, r_max, cutoff, out_bf16=False, s_ref=None):
+    """Compares sigma, the kept rank, the product A B (at the GPU's rank) and the balance
+    invariant with the checker.  Near the cutoff boundary ranks r' and r'+-1 are both valid."""
+    A, B, sigma, r_out, status = ab.ab_svd_split(dev(W), r_max, cutoff,
+                                                 out_dtype=torch.bfloat16 if out_bf16 else None)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    r_gpu = int(r_out.item())
+    m, n = W.shape
+    r_cap = min(r_max, m, n)
+    Wd = np.asarray(W, dtype=np.float64)
+    U, s, Vt, _ = orc.jacobi_svd(Wd)
+    r_ref = orc.rank_rule(s, cutoff, r_cap)
+    near = np.any(np.abs(s[:r_cap] - cutoff * s[0]) <= 1e-3 * s[0]) if cutoff > 0 else False
+    if near:
+        assert abs(r_gpu - r_ref) <= 1
+    else:
+        assert r_gpu == r_ref, (r_gpu, r_ref)
+    sg = host(sigma)
+    k = min(r_gpu, r_ref)
+    tol_s = 8e-3 if out_bf16 else 1e-4
+    assert np.all(np.abs(sg[:k] - s[:k]) <= 1e-4 * s[:k]), np.max(np.abs(sg[:k] - s[:k]) / s[:k])
+    Ah, Bh = host(A), host(B)
+    assert np.count_nonzero(Ah[:, r_gpu:]) == 0 and np.count_nonzero(Bh[r_gpu:]) == 0
+    Wr = (U[:, :r_gpu] * s[:r_gpu]) @ Vt[:r_gpu]
+    err = np.linalg.norm(Ah @ Bh - Wr) / np.linalg.norm(Wd)
+    assert err <= (tol_s if out_bf16 else 1e-4), err
+    if not out_bf16:
+        bal_a = np.linalg.norm(Ah[:, :r_gpu].T @ Ah[:, :r_gpu] - np.diag(sg[:r_gpu])) / s[0]
+        bal_b = np.linalg.norm(Bh[:r_gpu] @ Bh[:r_gpu].T - np.diag(sg[:r_gpu])) / s[0]
+        assert bal_a <= 1e-3 and bal_b <= 1e-3, (bal_a, bal_b)
+    return r_gpu, sg
+
+
+@pytest.mark.parametrize("m,n,r_max", [(256, 512, 32), (96, 64, 16), (64, 96, 16), (33, 47, 33), (130, 70, 20),
+                                       (200, 192, 192), (1, 5, 1), (7, 1, 1), (2, 2, 2), (320, 100, 100)])
+def test_svd_split_fixed_rank(ab, m, n, r_max):
+    rng = np.random.default_rng(m * 7 + n)
+    W = rng.standard_normal((m, n)).astype(np.float32) / np.sqrt(n)
+    check_split(ab, W, r_max, 0.0)
+
+
+def test_svd_split_planted_spectrum_rank_rule(ab):
+    rng = np.random.default_rng(12)
+    sig = np.exp(-np.arange(192) / 64.0)
+    W = synth.planted_matrix(rng, 384, 192, sig)
+    r, sg = check_split(ab, W, 192, 0.1)
+    assert r == 148
+    W2 = np.ascontiguousarray(W.T)
+    r2, _ = check_split(ab, W2, 192, 0.1)
+    assert r2 == 148
+
+
+def test_svd_split_exact_low_rank(ab):
+    rng = np.random.default_rng(13)
+    for (m, n, r) in [(160, 96, 24), (96, 160, 24)]:
+        W = (rng.standard_normal((m, r)) @ rng.standard_normal((r, n)) / np.sqrt(r)).astype(np.float32)
+        A, B, sigma, r_out, status = ab.ab_svd_split(dev(W), r, 0.0)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0 and int(r_out.item()) == r
+        assert orc.rel_frob(host(A) @ host(B), W) <= 1e-5     # exact recovery at rank <= r
+        # asking for more rank than W has must not add anything
+        A2, B2, _, r2, _ = ab.ab_svd_split(dev(W), r + 8, 0.0)
+        torch.cuda.synchronize()
+        assert int(r2.item()) == r + 8
+        assert orc.rel_frob(host(A2) @ host(B2), W) <= 1e-5
+
+
+def test_svd_split_bf16_output_and_cutoff_extremes(ab):
+    rng = np.random.default_rng(14)
+    W = rng.standard_normal((128, 80)).astype(np.float32)
+    check_split(ab, W, 40, 0.0, out_bf16=True)
+    A, B, sigma, r_out, _ = ab.ab_svd_split(dev(W), 40, 5.0)     # cutoff above 1: one value is kept
+    torch.cuda.synchronize()
+    assert int(r_out.item()) == 1
+    assert torch.count_nonzero(A[:, 1:]) == 0 and torch.count_nonzero(B[1:]) == 0
+
+
+def test_svd_split_zero_matrix(ab):
+    W = np.zeros((20, 12), dtype=np.float32)
+    A, B, sigma, r_out, status = ab.ab_svd_split(dev(W), 4, 0.0)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.count_nonzero(A) == 0 and torch.count_nonzero(B) == 0 and torch.count_nonzero(sigma) == 0
+
+
+# ------------------------------------------------------------------ the five workloads (scaled where needed)
+
+def test_workload_linear_fp32_full(ab):
+    """First workload at full size: forward, backward, mean, recombine, re-split, seed 0."""
+    d = synth.linear_fp32(0)
+    A, B, _, _ = orc.svd_split(d["W"], d["r"], 0.0)
+    d["A"], d["B"] = A.astype(np.float32), B.astype(np.float32)
+    check_chain(ab, d, False, save_T=True)
+    Ak = synth.group_copies(d["A"], d["noise_A"])
+    Bk = synth.group_copies(d["B"], d["noise_B"])
+    Abar = ab.ab_group_average(dev(Ak))
+    Bbar = ab.ab_group_average(dev(Bk))
+    W = ab.ab_recombine(Abar, Bbar)
+    torch.cuda.synchronize()
+    assert np.array_equal(Abar.cpu().numpy().view(np.uint32), orc.group_average_f32(Ak).view(np.uint32))
+    assert np.array_equal(Bbar.cpu().numpy().view(np.uint32), orc.group_average_f32(Bk).view(np.uint32))
+    W_ref = orc.recombine(orc.group_average_f32(Ak), orc.group_average_f32(Bk))
+    assert orc.rel_frob(host(W), W_ref) <= 1e-6
+    check_split(ab, W.cpu().numpy(), d["r"], 0.0)
+    check_split(ab, d["W"], d["r"], 0.0)          # the full-rank random W itself
+
+
+def test_workload_group_sync_scaled(ab):
+    """ViT-B/16 group sync recipe at 1/4 scale (six matrices of one block), K=8, cutoff 0.1."""
+    shapes = synth.VIT_BLOCK_SHAPES
+    ds = [synth.vit_sync_matrix(3, i, m, n, K=8, scale=4) for i, (m, n) in enumerate(shapes)]
+    Aks = [synth.group_copies(d["A"], d["noise_A"]) for d in ds]
+    Bks = [synth.group_copies(d["B"], d["noise_B"]) for d in ds]
+    plan = ab.SyncPlan([dev(a) for a in Aks], [dev(b) for b in Bks], 0.1)
+    A_out, B_out, sigma, r_out, status = ab.ab_group_sync(plan)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(status) == 0
+    for i, d in enumerate(ds):
+        ref = orc.group_sync(orc.group_average_f32(Aks[i])[None], orc.group_average_f32(Bks[i])[None], d["r"], 0.1)
+        s = ref["sigma"]
+        r_gpu = int(r_out[i].item())
+        near = np.any(np.abs(s[:d["r"]] - 0.1 * s[0]) <= 1e-3 * s[0])
+        assert abs(r_gpu - ref["r"]) <= (1 if near else 0), (i, r_gpu, ref["r"])
+        k = min(r_gpu, ref["r"])
+        sg = host(sigma[i])
+        assert np.all(np.abs(sg[:k] - s[:k]) <= 1e-4 * s[:k])
+        U, s2, Vt, _ = orc.jacobi_svd(ref["W"])
+        Wr = (U[:, :r_gpu] * s2[:r_gpu]) @ Vt[:r_gpu]
+        err = np.linalg.norm(host(A_out[i]) @ host(B_out[i]) - Wr) / np.linalg.norm(ref["W"])
+        assert err <= 1e-4, (i, err)
+
+
+def test_workload_resnet_and_vgg_scaled(ab):
+    d = synth.resnet_conv(2, N=1024)
+    check_chain(ab, d, True, save_T=True)
+    for r in (8, 16, 32, 64):
+        d = synth.vgg_conv(r, 4, N=512)
+        check_chain(ab, d, True)
