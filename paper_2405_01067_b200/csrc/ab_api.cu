@@ -33,7 +33,7 @@ int check_layer_args(const void* x, const void* A, const void* B, int64_t N, int
   if (N < 0 || m <= 0 || n <= 0 || r <= 0) return AB_ERR_INVALID_ARG;
   if (r > m || r > n) return AB_ERR_INVALID_ARG;
   if (ldA < r || ldB < n) return AB_ERR_INVALID_ARG;
-  if (!x || !A || !B) return AB_ERR_INVALID_ARG;
+  if (!A || !B || (N > 0 && !x)) return AB_ERR_INVALID_ARG;
   return AB_OK;
 }
 
@@ -124,7 +124,7 @@ int ab_layer_forward(const void* x, const void* A, const void* B, void* y, void*
                      int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
                      void* ws, size_t ws_bytes, void* cuda_stream) {
   AB_TRY(check_layer_args(x, A, B, N, m, n, r, ldA, ldB, dt));
-  if (!y) return AB_ERR_INVALID_ARG;
+  if (N > 0 && !y) return AB_ERR_INVALID_ARG;
   if (!have_device()) return AB_ERR_CUDA;
   if (N == 0) return AB_OK;
   if (ws && !aligned(ws, 256)) return AB_ERR_WORKSPACE;
@@ -139,7 +139,7 @@ int ab_layer_backward(const void* x, const void* dY, const void* A, const void* 
                       int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
                       void* ws, size_t ws_bytes, void* cuda_stream) {
   AB_TRY(check_layer_args(x, A, B, N, m, n, r, ldA, ldB, dt));
-  if (!dY) return AB_ERR_INVALID_ARG;
+  if (N > 0 && !dY) return AB_ERR_INVALID_ARG;
   if (!have_device()) return AB_ERR_CUDA;
   if (ws && !aligned(ws, 256)) return AB_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

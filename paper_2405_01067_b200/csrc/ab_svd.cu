@@ -224,7 +224,7 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
             fabsf(apq) > 0.25f * tol * sqrtf(app) * sqrtf(aqq)) {
           float zeta = (aqq - app) / (2.f * apq);
           float tt = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
-          c = rsqrtf(1.f + tt * tt);
+          c = 1.f / sqrtf(1.f + tt * tt);   // IEEE sqrt and divide: c^2 + s^2 = 1 to an ulp, no drift
           sv = c * tt;
           any_rot = 1;
         }
@@ -307,13 +307,26 @@ norms_sort_kernel(const float* __restrict__ Xall, int s, float* __restrict__ lam
   }
 }
 
-// Vr[k][:] = Vt[perm[k]][:], k < r_cap
-__global__ void gather_rows_kernel(const float* __restrict__ Vt, const int* __restrict__ perm, int s, int r_cap,
-                                   float* __restrict__ Vr) {
+// Vr[k][:] = Vt[perm[k]][:] scaled to unit length, k < r_cap (thousands of fp32 rotations leave
+// the rows orthogonal but let their norms wander by ~1e-6)
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const float* __restrict__ Vt, const int* __restrict__ perm, int s, int r_cap,
+                   float* __restrict__ Vr) {
+  __shared__ double red[8];
   const int k = blockIdx.x;
   if (k >= r_cap) return;
   const float* src = Vt + (size_t)perm[k] * s;
-  for (int u = threadIdx.x; u < s; u += blockDim.x) Vr[(size_t)k * s + u] = src[u];
+  double acc = 0.0;
+  for (int u = threadIdx.x; u < s; u += 256) { float v = src[u]; acc += (double)v * v; }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  double tot = 0.0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tot += red[i];
+  const float inv = tot > 0.0 ? (float)(1.0 / sqrt(tot)) : 0.f;
+  for (int u = threadIdx.x; u < s; u += 256) Vr[(size_t)k * s + u] = src[u] * inv;
 }
 
 // sigma[k] = norm over t of Ylong(k,t), Ylong(k,t) = Y[t*st_ + k*sk].  32 values of k per CTA.
