@@ -1,0 +1,317 @@
+#!/usr/bin/env python
+"""Benchmark of the AB-Training hot path on B200.
+
+A step is one pass of the whole path over one batch of synthetic input at the ViT-B/16 MLP
+shapes (W1 3072x768, W2 768x3072, rank 192, 50,432 token rows, bf16 storage / fp32
+accumulation, K = 4 group copies):
+  chain : ab_layer_forward + ab_layer_backward (dX, dA, dB) of both layers,
+  sync  : ab_group_sync of both layers (mean of the K copies, W = Abar Bbar, truncated-SVD split).
+`value` is the chain's algorithmic TFLOP/s, 6 N r (m+n) per layer, over the chain's share of
+the timed steps (CUDA events inside every step); the sync is reported beside it as ms per
+step.  `ms_per_step` covers both.  One process per GPU; ranks take independent batches (weak
+scaling, no collective on the data path).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--rows R]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "AB layer fwd+bwd TFLOP/s"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+R = 192
+LAYERS = ((3072, 768), (768, 3072))
+K_GROUPS = 4
+
+
+def chain_flops(N, layers=LAYERS, r=R):
+    return sum(6.0 * N * r * (m + n) for m, n in layers)
+
+
+def chain_bytes(N, layers=LAYERS):
+    # every activation once: x in forward and backward, y out, dY in, dX out (bf16)
+    return sum(2.0 * N * (3 * n + 2 * m) for m, n in layers)
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], tc_burst=d["bf16_tflops"], tc_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm=6650.0, tc_burst=1590.0, tc_sustained=1400.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.stop_flag, self.sm, self.reasons, self.max_sm = index, False, [], set(), None
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_sm = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+                     0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+            while not self.stop_flag:
+                self.sm.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                bits = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                for b, nm in names.items():
+                    if bits & b:
+                        self.reasons.add(nm)
+                time.sleep(0.05)
+        except Exception as e:  # clocks are evidence, not a dependency of the measurement
+            self.reasons.add(f"nvml_unavailable:{type(e).__name__}")
+
+    def summary(self):
+        return dict(sm_mhz=float(np.median(self.sm)) if self.sm else None, sm_max_mhz=self.max_sm,
+                    reasons=sorted(self.reasons), samples=len(self.sm))
+
+
+def make_inputs(rank, N):
+    """Host-side synthetic inputs of both layers for one rank (seed depends on the rank)."""
+    from paper_2405_01067_b200 import synth
+    out = []
+    for li in (1, 2):
+        d = synth.vit_mlp(li, seed=1 + 100 * rank, N=N, K=K_GROUPS)
+        d["A_copies"] = synth.group_copies(d["A"], d["noise_A"], bf16=True)
+        d["B_copies"] = synth.group_copies(d["B"], d["noise_B"], bf16=True)
+        out.append(d)
+    return out
+
+
+def cpu_baseline(inputs, rows, sync_scale=8):
+    """The CPU checker, as it stands, on a bounded sample: chain on the first `rows` rows of both
+    layers; the group sync of a 1/sync_scale-size copy of the recipe (timed separately)."""
+    from oracle import ab_oracle as orc
+    from paper_2405_01067_b200 import synth
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    t0 = time.perf_counter()
+    for d in inputs:
+        x, dY = d["x"][:rows], d["dY"][:rows]
+        orc.forward(x, d["A"], d["B"])
+        orc.backward(x, dY, d["A"], d["B"])
+    t_chain = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    for i, (m, n) in enumerate(LAYERS):
+        s = synth.vit_sync_matrix(1, i, m, n, K=K_GROUPS, scale=sync_scale)
+        orc.group_sync(synth.group_copies(s["A"], s["noise_A"]), synth.group_copies(s["B"], s["noise_B"]), s["r"], 0.0)
+    t_sync = time.perf_counter() - t0
+    return dict(value=chain_flops(rows) / t_chain / 1e12, unit=UNIT, cores=int(cores), kind="oracle",
+                sample=f"chain: first {rows} of 50432 rows of both layers, float64, {t_chain:.2f} s; "
+                       f"sync: both matrices at 1/{sync_scale} scale, own Jacobi SVD, {t_sync:.2f} s",
+                chain_s=t_chain, sync_sample_s=t_sync)
+
+
+def run_reference(args):
+    """--impl reference: the CPU checker timed on the host cores, same metric and config."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    rows = args.ref_rows
+    inputs = make_inputs(0, rows)
+    for _ in range(args.warmup):
+        cpu_baseline(inputs, min(rows, 512))
+    t0 = time.perf_counter()
+    last = None
+    for _ in range(args.steps):
+        last = cpu_baseline(inputs, rows)
+    dt = (time.perf_counter() - t0) / args.steps
+    chain_s = last["chain_s"]
+    v = chain_flops(rows) / chain_s / 1e12
+    line = dict(impl="reference", metric=METRIC, value=v, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=dt * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic",
+                config=dict(workload="vit_b16_mlp_pair_r192 (bounded sample)", rows=rows, K=K_GROUPS, r=R),
+                cpu_baseline=dict(value=v, unit=UNIT, cores=last["cores"], kind="oracle", sample=last["sample"]),
+                e2e=dict(value=v, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2405_01067_b200 import binding as ab
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    ab.lib()
+    N = args.rows
+    inputs = make_inputs(rank, N)
+    bf = torch.bfloat16
+
+    def pinned(a):
+        return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(bf).pin_memory()
+
+    layers = []
+    for d in inputs:
+        m, n = d["m"], d["n"]
+        h = {k: pinned(d[k]) for k in ("x", "dY", "A", "B", "A_copies", "B_copies")}
+        g = {k: v.cuda() for k, v in h.items()}
+        g.update(y=torch.empty((N, m), dtype=bf, device="cuda"), T=torch.empty((N, R), dtype=bf, device="cuda"),
+                 dX=torch.empty((N, n), dtype=bf, device="cuda"),
+                 dA=torch.empty((m, R), dtype=torch.float32, device="cuda"),
+                 dB=torch.empty((R, n), dtype=torch.float32, device="cuda"),
+                 ws_f=ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_FORWARD, N, m, n, R, 1, ab.AB_BF16), "cuda"),
+                 ws_b=ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_BACKWARD, N, m, n, R, 1, ab.AB_BF16), "cuda"))
+        hout = dict(dA=torch.empty((m, R), dtype=torch.float32).pin_memory(),
+                    dB=torch.empty((R, n), dtype=torch.float32).pin_memory(),
+                    A=torch.empty((m, R), dtype=bf).pin_memory(), B=torch.empty((R, n), dtype=bf).pin_memory(),
+                    sigma=torch.empty((R,), dtype=torch.float32).pin_memory())
+        layers.append(dict(m=m, n=n, h=h, g=g, hout=hout))
+    plan = ab.SyncPlan([L["g"]["A_copies"] for L in layers], [L["g"]["B_copies"] for L in layers], 0.0)
+
+    def chain():
+        for L in layers:
+            g = L["g"]
+            ab.ab_layer_forward(g["x"], g["A"], g["B"], y=g["y"], T_save=g["T"], ws=g["ws_f"])
+            ab.ab_layer_backward(g["x"], g["dY"], g["A"], g["B"], T_saved=g["T"], dX=g["dX"], dA=g["dA"], dB=g["dB"],
+                                 ws=g["ws_b"])
+
+    def step(marks=None):
+        if marks is not None:
+            marks[0].record()
+        chain()
+        if marks is not None:
+            marks[1].record()
+        ab.ab_group_sync(plan)
+        if marks is not None:
+            marks[2].record()
+
+    def e2e_step():
+        for L in layers:
+            L["g"]["x"].copy_(L["h"]["x"], non_blocking=True)
+            L["g"]["dY"].copy_(L["h"]["dY"], non_blocking=True)
+        step()
+        for i, L in enumerate(layers):
+            L["hout"]["dA"].copy_(L["g"]["dA"], non_blocking=True)
+            L["hout"]["dB"].copy_(L["g"]["dB"], non_blocking=True)
+            L["hout"]["A"].copy_(plan.A_out[i], non_blocking=True)
+            L["hout"]["B"].copy_(plan.B_out[i], non_blocking=True)
+            L["hout"]["sigma"].copy_(plan.sigma[i], non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    marks = [[ev(), ev(), ev()] for _ in range(args.steps)]
+    launches0 = ab.ab_launch_count()
+    t_begin, t_end = ev(), ev()
+    t_begin.record()
+    for i in range(args.steps):
+        step(marks[i])
+    t_end.record()
+    barrier()
+    sampler.stop_flag = True
+    launches = ab.ab_launch_count() - launches0
+    total_ms = t_begin.elapsed_time(t_end)
+    chain_ms = sum(mk[0].elapsed_time(mk[1]) for mk in marks)
+    sync_ms = sum(mk[1].elapsed_time(mk[2]) for mk in marks)
+    if int(plan.status.abs().sum().item()) != 0:
+        raise SystemExit("group sync reported a device-side error status")
+
+    # end to end: inputs start in pinned host memory, results end there
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e0, e1 = ev(), ev()
+    e0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    times = torch.tensor([total_ms, chain_ms, sync_ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, chain_ms, sync_ms, e2e_ms = [float(v) for v in times.tolist()]
+    sampler.join(timeout=2.0)
+    if rank == 0:
+        pk = measured_peaks()
+        K = args.steps
+        flops_step = chain_flops(N) * world
+        value = flops_step * K / (chain_ms * 1e-3) / 1e12
+        e2e_chain_share = e2e_ms - sync_ms   # same sync work; the rest is chain plus copies
+        e2e_value = flops_step * K / (max(e2e_chain_share, 1e-6) * 1e-3) / 1e12
+        h2d = sum(L["h"]["x"].numel() + L["h"]["dY"].numel() for L in layers) * 2
+        d2h = sum(sum(t.numel() * t.element_size() for t in L["hout"].values()) for L in layers)
+        per_gpu = value / world
+        roof = dict(bound="tensor", kernel="ab_layer_forward+ab_layer_backward (both layers)",
+                    achieved=per_gpu, peak=pk["tc_sustained"], unit="TFLOP/s", frac=per_gpu / pk["tc_sustained"],
+                    traffic=None, peak_source=f"bf16_tflops_sustained of {pk['source']}",
+                    frac_of_nominal_2250=per_gpu / NOMINAL_BF16_TFLOPS,
+                    hbm_gbs=chain_bytes(N) * K / (chain_ms * 1e-3) / 1e9, hbm_peak_gbs=pk["hbm"])
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=K, warmup=args.warmup,
+                    ms_per_step=total_ms / K, higher_is_better=True, scaling="weak", vs_baseline=None,
+                    dtype="bf16", data="synthetic",
+                    config=dict(workload="vit_b16_mlp_pair_r192", rows=N, layers=[list(s) for s in LAYERS], r=R,
+                                K=K_GROUPS, sync="mean+recombine+svd_split of both layers every step",
+                                l2="inputs larger than L2 (about 0.8 GB of activations read per step)"),
+                    chain_ms_per_step=chain_ms / K, group_sync_ms_per_step=sync_ms / K,
+                    pct_of_nominal_bf16_peak=100.0 * per_gpu / NOMINAL_BF16_TFLOPS,
+                    e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                             ms_per_step=e2e_ms / K),
+                    gpu_launches=int(launches), clocks=sampler.summary(), roofline=roof)
+        if world == 1 and not args.no_cpu_baseline:
+            cb = cpu_baseline(inputs, min(N, args.ref_rows))
+            line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--rows", type=int, default=256 * 197, help="token rows per layer (default: batch 256 x 197)")
+    ap.add_argument("--ref-rows", type=int, default=8192, help="rows of the CPU checker's bounded sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -56,6 +56,9 @@ const char* ab_status_string(int status);
 /* Library version, "major.minor". */
 const char* ab_version(void);
 
+/* Number of kernels this library has launched in this process since it was loaded. */
+long long ab_launch_count(void);
+
 /*
  * Scratch bytes a call needs (0 if none).  Arguments a given op does not use are ignored
  * (pass 0).  For AB_OP_SVD_SPLIT, r is r_max.  Returns 0 for unknown ops or bad sizes.

@@ -20,7 +20,7 @@ AB_OK = 0
 AB_ERR_INVALID_ARG, AB_ERR_UNSUPPORTED, AB_ERR_WORKSPACE = -1, -2, -3
 AB_ERR_NOT_CONVERGED, AB_ERR_TIMEOUT, AB_ERR_CUDA = -4, -5, -6
 
-EXPORTS = ["ab_status_string", "ab_version", "ab_workspace_bytes", "ab_layer_forward", "ab_layer_backward",
+EXPORTS = ["ab_status_string", "ab_version", "ab_launch_count", "ab_workspace_bytes", "ab_layer_forward", "ab_layer_backward",
            "ab_group_average", "ab_recombine", "ab_svd_split", "ab_group_sync", "ab_sync_workspace_bytes"]
 
 
@@ -51,6 +51,7 @@ def lib() -> ctypes.CDLL:
     L.ab_status_string.restype = c_char_p
     L.ab_status_string.argtypes = [c_int]
     L.ab_version.restype = c_char_p
+    L.ab_launch_count.restype = ctypes.c_longlong
     L.ab_workspace_bytes.restype = c_size_t
     L.ab_workspace_bytes.argtypes = [c_int, c_int64, c_int, c_int, c_int, c_int, c_int]
     L.ab_layer_forward.restype = c_int
@@ -71,6 +72,10 @@ def lib() -> ctypes.CDLL:
     L.ab_sync_workspace_bytes.argtypes = [ctypes.POINTER(ab_sync_desc), c_int, c_int, c_int]
     _lib = L
     return L
+
+
+def ab_launch_count() -> int:
+    return int(lib().ab_launch_count())
 
 
 def status_string(status: int) -> str:

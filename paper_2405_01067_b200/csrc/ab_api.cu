@@ -4,7 +4,12 @@
 
 #include "ab_common.cuh"
 
+#include <atomic>
+
 namespace ab {
+static std::atomic<long long> g_launches{0};
+void count_launches(long long n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
 namespace {
 
 template <typename TI, typename TO>
@@ -97,6 +102,8 @@ const char* ab_status_string(int s) {
 }
 
 const char* ab_version(void) { return "0.1"; }
+
+long long ab_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 size_t ab_workspace_bytes(int op, int64_t N, int m, int n, int r, int K, int dt) {
   (void)K;

@@ -18,8 +18,12 @@ typedef __nv_bfloat16 bf16;
     if (_e != cudaSuccess) return AB_ERR_CUDA;             \
   } while (0)
 
+// Every kernel launch site is followed by AB_LAUNCH_OK(), which also counts the launch.
+void count_launches(long long n);
+
 #define AB_LAUNCH_OK()                                     \
   do {                                                     \
+    ::ab::count_launches(1);                               \
     if (cudaPeekAtLastError() != cudaSuccess) {            \
       cudaGetLastError();                                  \
       return AB_ERR_CUDA;                                  \

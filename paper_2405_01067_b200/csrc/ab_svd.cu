@@ -483,6 +483,7 @@ int run_jacobi(float* X, float* Vt, JState* st, int s, int nb, int count, cudaSt
     }
     sweep_end_kernel<<<(count + 127) / 128, 128, 0, stream>>>(st, count, tol);
   }
+  count_launches((long long)kMaxSweeps * (rounds + 1) - 1);
   AB_LAUNCH_OK();
   return AB_OK;
 }
