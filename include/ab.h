@@ -78,6 +78,31 @@ int ab_layer_forward(const void* x, const void* A, const void* B, void* y, void*
                      void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * ab_layer_forward for callers that cannot allocate.  (The paper has no counterpart; this is
+ * a packaging variant of the call above.)  Some callers have no way to give the library a
+ * workspace: they run where device allocation is forbidden or impossible -- inside a host
+ * application that has reserved all device memory for its own pool, in a plug-in without
+ * access to that pool, in a latency-critical loop that must not hit cudaMalloc's implicit
+ * synchronisation.  For them the rank-r intermediate T = x B^T is kept in a fixed 4 MiB
+ * array built into the library (each GPU that loads the library holds it until the process
+ * ends), so the call needs only its inputs and its output and never calls cudaMalloc,
+ * cudaFree or any allocating routine.
+ *   Same arguments and results as ab_layer_forward without T_save and ws; always runs the
+ *   general kernels.  Limit: N * r <= ab_static_scratch_elems() (1,048,576); larger calls
+ *   return AB_ERR_UNSUPPORTED and launch nothing.
+ *   The first call on each device looks up the array's device address (with that device
+ *   current); make that first call outside of any stream capture.
+ *   All calls on a device share the one array, which keeps whatever the previous call left
+ *   in it (this call overwrites all it reads, so nothing has to be cleared).  Two calls
+ *   that may run on the GPU at the same time -- different streams, or different host
+ *   threads -- race on it: serialise them on one stream.
+ */
+int ab_layer_forward_static(const void* x, const void* A, const void* B, void* y,
+                            int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
+                            void* cuda_stream);
+size_t ab_static_scratch_elems(void);
+
+/*
  * Backward of the factorised layer (chain rule through T):
  *   dT = dY A, dX = dT B, dA = dY^T T, dB = dT^T x.
  *   dX [N,n] of type dt; dA [m,r] and dB [r,n] are fp32 and dense (row strides r and n).

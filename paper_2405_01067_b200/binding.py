@@ -21,7 +21,8 @@ AB_ERR_INVALID_ARG, AB_ERR_UNSUPPORTED, AB_ERR_WORKSPACE = -1, -2, -3
 AB_ERR_NOT_CONVERGED, AB_ERR_TIMEOUT, AB_ERR_CUDA = -4, -5, -6
 
 EXPORTS = ["ab_status_string", "ab_version", "ab_launch_count", "ab_workspace_bytes", "ab_layer_forward", "ab_layer_backward",
-           "ab_group_average", "ab_recombine", "ab_svd_split", "ab_group_sync", "ab_sync_workspace_bytes"]
+           "ab_group_average", "ab_recombine", "ab_svd_split", "ab_group_sync", "ab_sync_workspace_bytes",
+           "ab_layer_forward_static", "ab_static_scratch_elems"]
 
 
 class AbError(RuntimeError):
@@ -70,6 +71,9 @@ def lib() -> ctypes.CDLL:
                                 c_size_t, c_void_p]
     L.ab_sync_workspace_bytes.restype = c_size_t
     L.ab_sync_workspace_bytes.argtypes = [ctypes.POINTER(ab_sync_desc), c_int, c_int, c_int]
+    L.ab_layer_forward_static.restype = c_int
+    L.ab_layer_forward_static.argtypes = [c_void_p] * 4 + [c_int64] + [c_int] * 6 + [c_void_p]
+    L.ab_static_scratch_elems.restype = c_size_t
     _lib = L
     return L
 
@@ -135,6 +139,19 @@ def ab_layer_forward(x, A, B, y=None, T_save=None, ws=None, stream=None, save_T=
                                 A.stride(0), B.stride(0), dt, _ptr(ws), ws.numel(), _stream(stream))
     _check(st, "ab_layer_forward")
     return y, T_save
+
+
+def ab_layer_forward_static(x, A, B, y, stream=None):
+    """y = (x B^T) A^T with the intermediate in the library's built-in scratch array: for callers that
+    cannot allocate a workspace.  `y` must be supplied (this call allocates nothing); N*r is limited to
+    ab_static_scratch_elems().  Calls that may overlap on the GPU race on the shared array."""
+    _dev_ok(x, A, B, y)
+    N, n = x.shape
+    m, r = A.shape
+    st = lib().ab_layer_forward_static(_ptr(x), _ptr(A), _ptr(B), _ptr(y), N, m, n, r, A.stride(0), B.stride(0),
+                                       _dt(x), _stream(stream))
+    _check(st, "ab_layer_forward_static")
+    return y
 
 
 def ab_layer_backward(x, dY, A, B, T_saved=None, want=("dX", "dA", "dB"), dX=None, dA=None, dB=None,
