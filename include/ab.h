@@ -72,6 +72,9 @@ size_t ab_workspace_bytes(int op, int64_t N, int m, int n, int r, int K, int dt)
  *   backward call.  The rank-r intermediate stays on chip when dt = AB_BF16, r is a
  *   multiple of 16 with 16 <= r <= 256 and m, n are multiples of 8; other shapes take a
  *   slower general kernel (same results to rounding).  N = 0 is a no-op.
+ *   Device status: the first int of ws receives AB_OK, or AB_ERR_TIMEOUT if a bounded
+ *   on-chip wait of the fused kernel expired (outputs are then undefined).  The same holds
+ *   for ab_layer_backward.
  */
 int ab_layer_forward(const void* x, const void* A, const void* B, void* y, void* T_save,
                      int64_t N, int m, int n, int r, int ldA, int ldB, int dt,

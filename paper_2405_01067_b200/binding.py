@@ -119,6 +119,11 @@ def workspace(nbytes: int, device) -> torch.Tensor:
     return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
 
 
+def workspace_status(ws: torch.Tensor) -> int:
+    """Device status word a layer call left at the head of its workspace (synchronises)."""
+    return int(ws[:4].view(torch.int32).item())
+
+
 def ab_workspace_bytes(op: int, N: int, m: int, n: int, r: int, K: int = 1, dt: int = AB_F32) -> int:
     return int(lib().ab_workspace_bytes(op, N, m, n, r, K, dt))
 

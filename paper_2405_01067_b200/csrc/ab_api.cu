@@ -43,15 +43,18 @@ int check_layer_args(const void* x, const void* A, const void* B, int64_t N, int
 }
 
 // general path: every product is one strided GEMM on the fp32 pipes, T and dT live in the workspace
-size_t general_forward_ws(int64_t N, int r) { return align_up((size_t)N * r * sizeof(float), 256); }
-size_t general_backward_ws(int64_t N, int r) { return 2 * align_up((size_t)N * r * sizeof(float), 256); }
+// (the first 256 bytes of every layer workspace hold the device status word)
+size_t general_forward_ws(int64_t N, int r) { return 256 + align_up((size_t)N * r * sizeof(float), 256); }
+size_t general_backward_ws(int64_t N, int r) { return 256 + 2 * align_up((size_t)N * r * sizeof(float), 256); }
 
 int general_forward(const void* x, const void* A, const void* B, void* y, void* T_save,
                     int64_t N, int m, int n, int r, int ldA, int ldB, int dt, void* ws, size_t ws_bytes,
                     cudaStream_t st) {
   Arena ar(ws, ws_bytes);
+  int* status = ar.take_n<int>(64);
   float* T = ar.take_n<float>((size_t)N * r);
   if (!ws || !ar.fits()) return AB_ERR_WORKSPACE;
+  AB_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
   AB_TRY(gemm_simt(x, dt, n, 1, B, dt, 1, ldB, T, AB_F32, r, N, r, n, st));        // T = x B^T
   if (T_save) AB_TRY(cast_f32_to(T, T_save, dt, N * r, st));
   AB_TRY(gemm_simt(T, AB_F32, r, 1, A, dt, 1, ldA, y, dt, m, N, m, r, st));         // y = T A^T
@@ -62,9 +65,11 @@ int general_backward(const void* x, const void* dY, const void* A, const void* B
                      void* dX, float* dA, float* dB, int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
                      void* ws, size_t ws_bytes, cudaStream_t st) {
   Arena ar(ws, ws_bytes);
+  int* status = ar.take_n<int>(64);
   float* T = ar.take_n<float>((size_t)N * r);
   float* dT = ar.take_n<float>((size_t)N * r);
   if (!ws || !ar.fits()) return AB_ERR_WORKSPACE;
+  AB_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
   AB_TRY(gemm_simt(dY, dt, m, 1, A, dt, ldA, 1, dT, AB_F32, r, N, r, m, st));      // dT = dY A
   if (dX) AB_TRY(gemm_simt(dT, AB_F32, r, 1, B, dt, ldB, 1, dX, dt, n, N, n, r, st));   // dX = dT B
   if (dA) {

@@ -1,11 +1,636 @@
-// Fused tensor-core chain (placeholder until the tcgen05 kernels land): reports "not supported"
-// so every shape takes the general kernels.
+// Fused tensor-core chain for bf16 storage (fp32 accumulation) on sm_100a.
+//
+// row_chain_kernel: one CTA per block of 128 rows computes  S = In F1^T  (128 x r, K-loop over
+// the input width, accumulator in TMEM), rounds S to bf16 into shared memory, and multiplies
+// on:  Out = S F2^T  in 128-column chunks (two TMEM accumulators so the epilogue of one chunk
+// overlaps the MMAs of the next).  The rank-r intermediate never goes to HBM unless the
+// caller asks for a copy.
+//   forward : In = x,  F1 = B  (r x n), F2 = A   (m x r), Out = y,  S = T
+//   backward: In = dY, F1 = A^T (r x m), F2 = B^T (n x r), Out = dX, S = dT
+// grad_kernel: dA = dY^T T and dB^T = x^T dT are reductions over the rows; a CTA owns 128
+// output rows (a slice of m or of n) and one slice of the N rows, streams 64-row slabs of
+// both operands (both "MN-major": the reduction index is the slow one in memory) and leaves
+// an fp32 partial; reduce_kernel adds the partials in ascending slice order.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner),
+// warps 2-5 = epilogue (TMEM -> registers -> shared/global).  All operand tiles are TMA
+// boxes of 64 bf16 (128 bytes) x rows with 128-byte swizzle.  Every mbarrier wait gives up
+// after about a second, raises AB_ERR_TIMEOUT in the status word and unwinds to the common
+// exit, where TMEM is released.
+#include <mutex>
+
 #include "ab_common.cuh"
+#include "ab_tc_ptx.cuh"
 
 namespace ab {
-bool chain_tc_supported(int64_t, int, int, int, int, int, int, const void*, const void*, const void*, const void*) { return false; }
-size_t chain_tc_forward_ws(int64_t, int, int, int) { return 0; }
-size_t chain_tc_backward_ws(int64_t, int, int, int) { return 0; }
-int chain_tc_forward(const void*, const void*, const void*, void*, void*, int64_t, int, int, int, int, int, void*, size_t, cudaStream_t) { return AB_ERR_UNSUPPORTED; }
-int chain_tc_backward(const void*, const void*, const void*, const void*, const void*, void*, float*, float*, int64_t, int, int, int, int, int, void*, size_t, cudaStream_t) { return AB_ERR_UNSUPPORTED; }
+namespace {
+
+using namespace tc;
+
+constexpr int kAtomBytes = 16384;      // 128 rows x 128 bytes
+constexpr int kMaxStages = 6;
+constexpr int kSmemLimit = 227 * 1024;
+constexpr int kTmemCols = 512;
+constexpr int kEpiThreads = 128;
+
+struct RowChainParams {
+  int K1;        // width of In (reduction length of the first product)
+  int P;         // width of Out (0: first product only)
+  int r;
+  int nk1;       // ceil(K1 / 64)
+  int nchunks;   // ceil(P / 128)
+  int natoms;    // ceil(r / 64)
+  int ns;        // ring stages
+  int slot_bytes;
+  int save_s;    // 1: copy S to global through tmS
+  int* status;
+};
+
+struct Bars {
+  uint64_t full[kMaxStages], empty[kMaxStages];
+  uint64_t t_full, s_ready;
+  uint64_t acc_full[2], acc_empty[2];
+  uint32_t tmem_base;
+  int abort_any;   // set by any role that gave up
+  int epi_abort;   // written and read by the epilogue warps only, around their own barrier
+};
+
+__device__ __forceinline__ void raise_timeout(Bars* b, int* status) {
+  *reinterpret_cast<volatile int*>(&b->abort_any) = 1;
+  atomicExch(status, (int)AB_ERR_TIMEOUT);
+}
+
+// epilogue-wide wait: every epilogue thread calls it; the verdict is uniform
+__device__ __forceinline__ bool epi_wait(Bars* b, uint64_t* bar, uint32_t parity, int* status) {
+  if (!mbar_wait(bar, parity)) {
+    *reinterpret_cast<volatile int*>(&b->epi_abort) = 1;
+    raise_timeout(b, status);
+  }
+  named_bar_sync(1, kEpiThreads);
+  return *reinterpret_cast<volatile int*>(&b->epi_abort) == 0;
+}
+
+__device__ __forceinline__ void store_bf16x16_swizzled(uint8_t* row_base, int row, int c0, const float (&v)[16]) {
+  // 16 consecutive columns c0..c0+15 (c0 % 16 == 0) of a 128-byte row inside a swizzled atom
+  uint32_t w[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    w[i] = *reinterpret_cast<uint32_t*>(&h);
+  }
+  const int ch = (c0 & 63) >> 3;
+  uint4* p0 = reinterpret_cast<uint4*>(row_base + (((ch) ^ (row & 7)) << 4));
+  uint4* p1 = reinterpret_cast<uint4*>(row_base + (((ch + 1) ^ (row & 7)) << 4));
+  *p0 = make_uint4(w[0], w[1], w[2], w[3]);
+  *p1 = make_uint4(w[4], w[5], w[6], w[7]);
+}
+
+__global__ void __launch_bounds__(192, 1)
+row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ CUtensorMap tmF1,
+                 const __grid_constant__ CUtensorMap tmF2, const __grid_constant__ CUtensorMap tmOut,
+                 const __grid_constant__ CUtensorMap tmS, const RowChainParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* S = smem;
+  uint8_t* stg = S + p.natoms * kAtomBytes;
+  uint8_t* ring = stg + 2 * kAtomBytes;
+  Bars* bars = reinterpret_cast<Bars*>(ring + (size_t)p.ns * p.slot_bytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row0 = blockIdx.x * 128;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.ns; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
+    mbar_init(&bars->t_full, 1);
+    mbar_init(&bars->s_ready, kEpiThreads);
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 4); }
+    bars->abort_any = 0;
+    bars->epi_abort = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&tmIn); tma_prefetch_desc(&tmF1); tma_prefetch_desc(&tmF2);
+    tma_prefetch_desc(&tmOut); tma_prefetch_desc(&tmS);
+  }
+  if (warp == 1) tmem_alloc(&bars->tmem_base, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
+  const uint32_t tT = tmem_base;
+  const uint32_t tAcc0 = tmem_base + 256;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int i = 0;
+      bool ok = true;
+      for (int ks = 0; ks < p.nk1 && ok; ++ks, ++i) {
+        const int slot = i % p.ns, ph = (i / p.ns) & 1;
+        if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
+        uint8_t* dst = ring + (size_t)slot * p.slot_bytes;
+        mbar_arrive_expect_tx(&bars->full[slot], kAtomBytes + p.r * 128);
+        tma_load_2d(dst, &tmIn, &bars->full[slot], ks * 64, row0);
+        tma_load_2d(dst + kAtomBytes, &tmF1, &bars->full[slot], ks * 64, 0);
+      }
+      for (int c = 0; c < p.nchunks && ok; ++c) {
+        for (int j = 0; j < p.natoms; ++j, ++i) {
+          const int slot = i % p.ns, ph = (i / p.ns) & 1;
+          if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
+          uint8_t* dst = ring + (size_t)slot * p.slot_bytes;
+          mbar_arrive_expect_tx(&bars->full[slot], kAtomBytes);
+          tma_load_2d(dst, &tmF2, &bars->full[slot], j * 64, c * 128);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc1 = instr_desc_bf16(128, p.r, 0, 0);
+      const uint32_t idesc2 = instr_desc_bf16(128, 128, 0, 0);
+      int i = 0;
+      bool ok = true;
+      for (int ks = 0; ks < p.nk1; ++ks, ++i) {
+        const int slot = i % p.ns, ph = (i / p.ns) & 1;
+        if (!mbar_wait(&bars->full[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = smem_u32(ring + (size_t)slot * p.slot_bytes);
+        const uint64_t da = smem_desc_sw128(sa, 16), db = smem_desc_sw128(sa + kAtomBytes, 16);
+        int ksteps = (p.K1 - ks * 64 + 15) >> 4;
+        if (ksteps > 4) ksteps = 4;
+        for (int kk = 0; kk < ksteps; ++kk) tc_mma_bf16(tT, da + 2 * kk, db + 2 * kk, idesc1, (ks | kk) != 0);
+        tc_commit(&bars->empty[slot]);
+      }
+      if (ok) {
+        tc_commit(&bars->t_full);
+        if (p.nchunks > 0) {
+          if (!mbar_wait(&bars->s_ready, 0)) { raise_timeout(bars, p.status); ok = false; }
+          tc_fence_after();
+        }
+      }
+      for (int c = 0; c < p.nchunks && ok; ++c) {
+        const int b = c & 1;
+        if (!mbar_wait(&bars->acc_empty[b], ((c >> 1) & 1) ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
+        tc_fence_after();
+        const uint32_t tacc = tAcc0 + 128 * b;
+        for (int j = 0; j < p.natoms; ++j, ++i) {
+          const int slot = i % p.ns, ph = (i / p.ns) & 1;
+          if (!mbar_wait(&bars->full[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
+          tc_fence_after();
+          const uint64_t da = smem_desc_sw128(smem_u32(S + j * kAtomBytes), 16);
+          const uint64_t db = smem_desc_sw128(smem_u32(ring + (size_t)slot * p.slot_bytes), 16);
+          int ksteps = (p.r - j * 64) >> 4;
+          if (ksteps > 4) ksteps = 4;
+          for (int kk = 0; kk < ksteps; ++kk) tc_mma_bf16(tacc, da + 2 * kk, db + 2 * kk, idesc2, (j | kk) != 0);
+          tc_commit(&bars->empty[slot]);
+        }
+        if (ok) tc_commit(&bars->acc_full[b]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;                 // TMEM lane quarter this warp may read
+    const int row = q * 32 + lane;          // row of the 128-row block
+    const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+    const bool issuer = (threadIdx.x == 64);
+    bool ok = epi_wait(bars, &bars->t_full, 0, p.status);
+    if (ok) {
+      tc_fence_after();
+      for (int c0 = 0; c0 < p.r; c0 += 16) {
+        float v[16];
+        tmem_ld16(tT + lane_base + c0, v);
+        store_bf16x16_swizzled(S + (c0 >> 6) * kAtomBytes + row * 128, row, c0, v);
+      }
+      tc_fence_before();
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->s_ready);
+      if (p.save_s) {
+        named_bar_sync(1, kEpiThreads);
+        if (issuer) {
+          for (int j = 0; j < p.natoms; ++j) tma_store_2d(&tmS, S + j * kAtomBytes, j * 64, row0);
+          tma_store_commit();
+        }
+      }
+    }
+    for (int c = 0; c < p.nchunks && ok; ++c) {
+      const int b = c & 1;
+      ok = epi_wait(bars, &bars->acc_full[b], (c >> 1) & 1, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t tacc = tAcc0 + 128 * b + lane_base;
+      for (int h = 0; h < 2; ++h) {
+        uint8_t* buf = stg + h * kAtomBytes;
+        if (issuer) tma_store_wait_read<1>();       // the store that last read this buffer is done
+        named_bar_sync(1, kEpiThreads);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          float v[16];
+          tmem_ld16(tacc + h * 64 + g * 16, v);
+          store_bf16x16_swizzled(buf + row * 128, row, g * 16, v);
+        }
+        fence_proxy_async_smem();
+        named_bar_sync(1, kEpiThreads);
+        if (issuer && c * 128 + h * 64 < p.P) {
+          tma_store_2d(&tmOut, buf, c * 128 + h * 64, row0);
+          tma_store_commit();
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->acc_empty[b]);
+    }
+    if (issuer) tma_store_wait_all();
+  }
+
+  // ------------------------------------------------------------ common exit
+  tc_fence_before();
+  __syncthreads();
+  if (*reinterpret_cast<volatile int*>(&bars->abort_any)) {
+    // give loads that are still in flight time to land before the shared memory is released
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// grad kernel: partial[slice][p][j] = sum_{k in slice} act[k][p] * small[k][j]
+struct GradJob {
+  int P;          // columns of act = rows of the output
+  int chunks;     // ceil(P / 128)
+  float* partial; // [slices][P][r]
+};
+struct GradParams {
+  GradJob job[2];
+  int njobs;
+  int r, natoms, ns, slot_bytes;
+  int slices, rows_per_slice;   // rows_per_slice is a multiple of 64
+  int N;
+  int* status;
+};
+
+__global__ void __launch_bounds__(192, 1)
+grad_kernel(const __grid_constant__ CUtensorMap tmAct0, const __grid_constant__ CUtensorMap tmSmall0,
+            const __grid_constant__ CUtensorMap tmAct1, const __grid_constant__ CUtensorMap tmSmall1,
+            const GradParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* ring = smem;
+  Bars* bars = reinterpret_cast<Bars*>(ring + (size_t)p.ns * p.slot_bytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // which job, which 128-row chunk of its output, which slice of the N rows
+  int tile = blockIdx.x;
+  const int slice = tile % p.slices;
+  tile /= p.slices;
+  int jb = 0;
+  if (tile >= p.job[0].chunks) { jb = 1; tile -= p.job[0].chunks; }
+  const int chunk = tile;
+  const CUtensorMap* tmAct = jb ? &tmAct1 : &tmAct0;
+  const CUtensorMap* tmSmall = jb ? &tmSmall1 : &tmSmall0;
+  const int k_begin = slice * p.rows_per_slice;
+  int k_end = k_begin + p.rows_per_slice;
+  if (k_end > p.N) k_end = p.N;
+  const int nk = k_end > k_begin ? (k_end - k_begin + 63) / 64 : 0;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.ns; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
+    mbar_init(&bars->t_full, 1);
+    bars->abort_any = 0;
+    bars->epi_abort = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(tmAct); tma_prefetch_desc(tmSmall);
+  }
+  if (warp == 1) tmem_alloc(&bars->tmem_base, 256);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int i = 0; i < nk; ++i) {
+        const int slot = i % p.ns, ph = (i / p.ns) & 1;
+        if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { raise_timeout(bars, p.status); break; }
+        uint8_t* dst = ring + (size_t)slot * p.slot_bytes;
+        const int k0 = k_begin + i * 64;
+        // rows at or beyond k_end inside the last slab belong to the next slice: the box is
+        // clipped by loading them and masking through a zero "small" operand is not possible,
+        // so slices are cut on 64-row boundaries (rows_per_slice % 64 == 0) and only the
+        // global end (k >= N) is ragged, where TMA fills zeros.
+        mbar_arrive_expect_tx(&bars->full[slot], (2 + p.natoms) * 8192);
+        tma_load_2d(dst, tmAct, &bars->full[slot], chunk * 128, k0);
+        tma_load_2d(dst + 8192, tmAct, &bars->full[slot], chunk * 128 + 64, k0);
+        for (int a = 0; a < p.natoms; ++a)
+          tma_load_2d(dst + 16384 + a * 8192, tmSmall, &bars->full[slot], a * 64, k0);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_bf16(128, p.r, 1, 1);
+      bool ok = true;
+      for (int i = 0; i < nk; ++i) {
+        const int slot = i % p.ns, ph = (i / p.ns) & 1;
+        if (!mbar_wait(&bars->full[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = smem_u32(ring + (size_t)slot * p.slot_bytes);
+        for (int kk = 0; kk < 4; ++kk) {
+          const uint64_t da = smem_desc_sw128(sa + kk * 2048, 8192);
+          const uint64_t db = smem_desc_sw128(sa + 16384 + kk * 2048, 8192);
+          tc_mma_bf16(tmem_base, da, db, idesc, (i | kk) != 0);
+        }
+        tc_commit(&bars->empty[slot]);
+      }
+      if (ok) tc_commit(&bars->t_full);
+    }
+  } else {
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+    const GradJob& job = p.job[jb];
+    const int prow = chunk * 128 + row;
+    float* out = job.partial + ((size_t)slice * job.P + prow) * p.r;
+    bool ok = true;
+    if (nk > 0) ok = epi_wait(bars, &bars->t_full, 0, p.status);
+    if (ok) {
+      tc_fence_after();
+      for (int c0 = 0; c0 < p.r; c0 += 16) {
+        float v[16];
+        if (nk > 0) tmem_ld16(tmem_base + lane_base + c0, v);
+        else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = 0.f;
+        }
+        if (prow < job.P) {
+          float4* o = reinterpret_cast<float4*>(out + c0);
+          o[0] = make_float4(v[0], v[1], v[2], v[3]);
+          o[1] = make_float4(v[4], v[5], v[6], v[7]);
+          o[2] = make_float4(v[8], v[9], v[10], v[11]);
+          o[3] = make_float4(v[12], v[13], v[14], v[15]);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*reinterpret_cast<volatile int*>(&bars->abort_any)) {
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 256);
+  }
+}
+
+// out[p][j] = sum_s partial[s][p][j]  (transpose_out: out[j][p])
+__global__ void reduce_partials_kernel(const float* __restrict__ partial, int slices, int P, int r,
+                                       float* __restrict__ out, int transpose_out) {
+  const int64_t total = (int64_t)P * r;
+  const int64_t step = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += step) {
+    int64_t pp, j;
+    if (transpose_out) { j = idx / P; pp = idx - j * P; } else { pp = idx / r; j = idx - pp * r; }
+    float acc = 0.f;
+    for (int s = 0; s < slices; ++s) acc += partial[((int64_t)s * P + pp) * r + j];
+    out[idx] = acc;
+  }
+}
+
+// dst[j][i] = src[i][j], bf16, src rows x cols with row stride ld
+__global__ void transpose_bf16_kernel(const bf16* __restrict__ src, int rows, int cols, int ld, bf16* __restrict__ dst) {
+  __shared__ bf16 tile[32][33];
+  const int bx = blockIdx.x * 32, by = blockIdx.y * 32;
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    int rr = by + i, cc = bx + threadIdx.x;
+    tile[i][threadIdx.x] = (rr < rows && cc < cols) ? src[(size_t)rr * ld + cc] : __float2bfloat16(0.f);
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    int cc = bx + i, rr = by + threadIdx.x;
+    if (cc < cols && rr < rows) dst[(size_t)cc * rows + rr] = tile[threadIdx.x][i];
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+bool device_is_sm100() {
+  static std::mutex mu;
+  static int cache[64];
+  static bool init = false;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!init) { for (int i = 0; i < 64; ++i) cache[i] = -1; init = true; }
+  if (cache[dev] < 0) {
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
+    cache[dev] = (major == 10) ? 1 : 0;
+  }
+  return cache[dev] == 1;
+}
+
+// bf16 matrix [rows x cols], row stride ld elements, box of box_cols x box_rows, 128-byte swizzle
+int make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_cols,
+             uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return AB_ERR_CUDA;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult rc = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? AB_OK : AB_ERR_CUDA;
+}
+
+struct RowPlan { int natoms, ns, slot_bytes; size_t smem; };
+RowPlan row_plan(int r) {
+  RowPlan pl;
+  pl.natoms = (r + 63) / 64;
+  pl.slot_bytes = kAtomBytes + r * 128;
+  const int fixed = pl.natoms * kAtomBytes + 2 * kAtomBytes + (int)sizeof(Bars) + 1024;
+  pl.ns = (kSmemLimit - fixed) / pl.slot_bytes;
+  if (pl.ns > kMaxStages) pl.ns = kMaxStages;
+  pl.smem = (size_t)fixed + (size_t)pl.ns * pl.slot_bytes;
+  return pl;
+}
+
+struct GradPlan { int natoms, ns, slot_bytes, slices, rows_per_slice; size_t smem; };
+GradPlan grad_plan(int64_t N, int m, int n, int r) {
+  GradPlan pl;
+  pl.natoms = (r + 63) / 64;
+  pl.slot_bytes = 16384 + pl.natoms * 8192;
+  const int fixed = (int)sizeof(Bars) + 1024;
+  pl.ns = (kSmemLimit - fixed) / pl.slot_bytes;
+  if (pl.ns > kMaxStages) pl.ns = kMaxStages;
+  pl.smem = (size_t)fixed + (size_t)pl.ns * pl.slot_bytes;
+  const int tiles = (m + 127) / 128 + (n + 127) / 128;
+  int slices = 148 / tiles;
+  if (slices < 1) slices = 1;
+  const int64_t slabs = (N + 63) / 64;
+  if (slices > slabs) slices = (int)slabs;
+  int64_t per = (slabs + slices - 1) / slices;
+  pl.rows_per_slice = (int)(per * 64);
+  pl.slices = (int)((slabs + per - 1) / per);
+  return pl;
+}
+
+struct BwdWs { int* status; bf16 *At, *Bt, *T, *dT; float *pA, *pB; size_t bytes; };
+BwdWs bwd_ws(void* ws, int64_t N, int m, int n, int r) {
+  GradPlan gp = grad_plan(N, m, n, r);
+  Arena ar(ws, 0);
+  BwdWs w;
+  w.status = ar.take_n<int>(64);
+  w.At = ar.take_n<bf16>((size_t)r * m);
+  w.Bt = ar.take_n<bf16>((size_t)n * r);
+  w.T = ar.take_n<bf16>((size_t)N * r);
+  w.dT = ar.take_n<bf16>((size_t)N * r);
+  w.pA = ar.take_n<float>((size_t)gp.slices * m * r);
+  w.pB = ar.take_n<float>((size_t)gp.slices * n * r);
+  w.bytes = align_up(ar.used, 256);
+  return w;
+}
+
+// S = In F1^T (saved to Sg if not null), Out = S F2^T (skipped if Out is null)
+int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1, const void* F2, int ldF2, int P,
+                     void* Out, void* Sg, int r, int* status, cudaStream_t st) {
+  RowPlan pl = row_plan(r);
+  if (pl.ns < 2) return AB_ERR_UNSUPPORTED;
+  CUtensorMap tmIn, tmF1, tmF2, tmOut, tmS;
+  AB_TRY(make_map(&tmIn, In, (uint64_t)N, K1, K1, 64, 128));
+  AB_TRY(make_map(&tmF1, F1, r, K1, ldF1, 64, r));
+  const bool second = Out != nullptr && P > 0;
+  // unused maps still have to be valid objects: alias them to the first operand
+  if (second) {
+    AB_TRY(make_map(&tmF2, F2, P, r, ldF2, 64, 128));
+    AB_TRY(make_map(&tmOut, Out, (uint64_t)N, P, P, 64, 128));
+  } else {
+    tmF2 = tmIn;
+    tmOut = tmIn;
+  }
+  if (Sg) AB_TRY(make_map(&tmS, Sg, (uint64_t)N, r, r, 64, 128));
+  else tmS = tmIn;
+  RowChainParams p;
+  p.K1 = K1; p.P = second ? P : 0; p.r = r; p.nk1 = (K1 + 63) / 64; p.nchunks = second ? (P + 127) / 128 : 0;
+  p.natoms = pl.natoms; p.ns = pl.ns; p.slot_bytes = pl.slot_bytes; p.save_s = Sg ? 1 : 0; p.status = status;
+  AB_CUDA_OK(cudaFuncSetAttribute(row_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
+  const unsigned grid = (unsigned)((N + 127) / 128);
+  row_chain_kernel<<<grid, 192, pl.smem, st>>>(tmIn, tmF1, tmF2, tmOut, tmS, p);
+  AB_LAUNCH_OK();
+  return AB_OK;
+}
+
+}  // namespace
+
+bool chain_tc_supported(int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
+                        const void* x, const void* A, const void* B, const void* y) {
+  if (dt != AB_BF16) return false;
+  if (r % 16 != 0 || r < 16 || r > 256) return false;
+  if (m % 8 != 0 || n % 8 != 0 || ldA % 8 != 0 || ldB % 8 != 0) return false;
+  if (N > (int64_t)1 << 30) return false;
+  if (!aligned(x, 16) || !aligned(A, 16) || !aligned(B, 16) || !aligned(y, 16)) return false;
+  if (!device_is_sm100() || !encode_fn()) return false;
+  return row_plan(r).ns >= 2;
+}
+
+size_t chain_tc_forward_ws(int64_t, int, int, int) { return 256; }
+size_t chain_tc_backward_ws(int64_t N, int m, int n, int r) {
+  if (r % 16 != 0 || r < 16 || r > 256) return 0;
+  return bwd_ws(nullptr, N, m, n, r).bytes;
+}
+
+int chain_tc_forward(const void* x, const void* A, const void* B, void* y, void* T_save,
+                     int64_t N, int m, int n, int r, int ldA, int ldB,
+                     void* ws, size_t ws_bytes, cudaStream_t st) {
+  if (!ws || ws_bytes < 256) return AB_ERR_WORKSPACE;
+  if (T_save && !aligned(T_save, 16)) return AB_ERR_INVALID_ARG;
+  int* status = static_cast<int*>(ws);
+  AB_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
+  return launch_row_chain(x, N, n, B, ldB, A, ldA, m, y, T_save, r, status, st);
+}
+
+int chain_tc_backward(const void* x, const void* dY, const void* A, const void* B,
+                      const void* T_saved, void* dX, float* dA, float* dB,
+                      int64_t N, int m, int n, int r, int ldA, int ldB,
+                      void* ws, size_t ws_bytes, cudaStream_t st) {
+  if (!ws) return AB_ERR_WORKSPACE;
+  BwdWs w = bwd_ws(ws, N, m, n, r);
+  if (w.bytes > ws_bytes) return AB_ERR_WORKSPACE;
+  if ((dX && !aligned(dX, 16)) || (T_saved && !aligned(T_saved, 16)) || (dA && !aligned(dA, 16)) ||
+      (dB && !aligned(dB, 16)))
+    return AB_ERR_INVALID_ARG;
+  AB_CUDA_OK(cudaMemsetAsync(w.status, 0, sizeof(int), st));
+  const bf16* T = static_cast<const bf16*>(T_saved);
+  if (dA && !T) {   // recompute T = x B^T (first product only)
+    AB_TRY(launch_row_chain(x, N, n, B, ldB, nullptr, 0, 0, nullptr, w.T, r, w.status, st));
+    T = w.T;
+  }
+  if (dX || dB) {
+    dim3 tb(32, 8);
+    transpose_bf16_kernel<<<dim3((r + 31) / 32, (m + 31) / 32), tb, 0, st>>>(static_cast<const bf16*>(A), m, r, ldA, w.At);
+    AB_LAUNCH_OK();
+    if (dX) {
+      transpose_bf16_kernel<<<dim3((n + 31) / 32, (r + 31) / 32), tb, 0, st>>>(static_cast<const bf16*>(B), r, n, ldB, w.Bt);
+      AB_LAUNCH_OK();
+    }
+    // dT = dY A (kept for dB), dX = dT B
+    AB_TRY(launch_row_chain(dY, N, m, w.At, m, w.Bt, r, n, dX, dB ? w.dT : nullptr, r, w.status, st));
+  }
+  if (dA || dB) {
+    GradPlan gp = grad_plan(N, m, n, r);
+    GradParams p;
+    CUtensorMap tmAct[2], tmSmall[2];
+    int nj = 0;
+    if (dA) {
+      AB_TRY(make_map(&tmAct[nj], dY, (uint64_t)N, m, m, 64, 64));
+      AB_TRY(make_map(&tmSmall[nj], T, (uint64_t)N, r, r, 64, 64));
+      p.job[nj].P = m; p.job[nj].chunks = (m + 127) / 128; p.job[nj].partial = w.pA;
+      ++nj;
+    }
+    if (dB) {
+      AB_TRY(make_map(&tmAct[nj], x, (uint64_t)N, n, n, 64, 64));
+      AB_TRY(make_map(&tmSmall[nj], w.dT, (uint64_t)N, r, r, 64, 64));
+      p.job[nj].P = n; p.job[nj].chunks = (n + 127) / 128; p.job[nj].partial = w.pB;
+      ++nj;
+    }
+    if (nj == 1) { tmAct[1] = tmAct[0]; tmSmall[1] = tmSmall[0]; p.job[1] = p.job[0]; p.job[1].chunks = 0; }
+    p.njobs = nj; p.r = r; p.natoms = gp.natoms; p.ns = gp.ns; p.slot_bytes = gp.slot_bytes;
+    p.slices = gp.slices; p.rows_per_slice = gp.rows_per_slice; p.N = (int)N; p.status = w.status;
+    AB_CUDA_OK(cudaFuncSetAttribute(grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gp.smem));
+    const unsigned grid = (unsigned)((p.job[0].chunks + p.job[1].chunks) * gp.slices);
+    grad_kernel<<<grid, 192, gp.smem, st>>>(tmAct[0], tmSmall[0], tmAct[1], tmSmall[1], p);
+    AB_LAUNCH_OK();
+    if (dA) {
+      reduce_partials_kernel<<<148 * 4, 256, 0, st>>>(w.pA, gp.slices, m, r, dA, 0);
+      AB_LAUNCH_OK();
+    }
+    if (dB) {
+      reduce_partials_kernel<<<148 * 4, 256, 0, st>>>(w.pB, gp.slices, n, r, dB, 1);
+      AB_LAUNCH_OK();
+    }
+  }
+  return AB_OK;
+}
+
 }  // namespace ab

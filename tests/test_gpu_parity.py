@@ -35,9 +35,15 @@ def host(t):
 
 def run_chain(ab, d, bf16, save_T):
     x, dY, A, B = (dev(d[k], bf16) for k in ("x", "dY", "A", "B"))
-    y, T = ab.ab_layer_forward(x, A, B, save_T=save_T)
-    dX, dA, dB = ab.ab_layer_backward(x, dY, A, B, T_saved=T)
+    N, n = x.shape
+    m, r = A.shape
+    dt = ab.AB_BF16 if bf16 else ab.AB_F32
+    ws_f = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_FORWARD, N, m, n, r, 1, dt), "cuda")
+    ws_b = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_BACKWARD, N, m, n, r, 1, dt), "cuda")
+    y, T = ab.ab_layer_forward(x, A, B, save_T=save_T, ws=ws_f)
+    dX, dA, dB = ab.ab_layer_backward(x, dY, A, B, T_saved=T, ws=ws_b)
     torch.cuda.synchronize()
+    assert ab.workspace_status(ws_f) == 0 and ab.workspace_status(ws_b) == 0
     return host(y), (host(T) if T is not None else None), host(dX), host(dA), host(dB)
 
 
