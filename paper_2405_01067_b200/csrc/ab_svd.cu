@@ -5,9 +5,9 @@
 // X = G with the rotations accumulated in V^T, all in fp32:
 //   * vectors are stored as ROWS (X is s x s, V^T is s x s), split into blocks of b rows;
 //   * a sweep is nb-1 rounds of disjoint block pairs (round-robin); one CTA per pair keeps the
-//     2b x s panel in shared memory, forms its 2b x 2b Gram matrix M, diagonalises M with a
-//     parallel two-sided cyclic Jacobi (M, Q in shared memory), applies Q^T to the panel and
-//     to the matching panel of V^T;
+//     2b x s panel in shared memory (b = 16), forms its 32 x 32 Gram matrix M, runs a few
+//     sweeps of a two-sided cyclic Jacobi on M inside one warp's registers (accumulating Q),
+//     applies Q^T to the panel and to the matching panel of V^T;
 //   * sweeps repeat until no pair of rows has |x_i.x_j| > tol |x_i||x_j| (a device flag; the
 //     host enqueues a fixed number of sweeps and converged matrices return at once).
 // At convergence the rows of V^T are eigenvectors of G (singular vectors of the short side)
@@ -30,15 +30,20 @@ struct JState {
   unsigned maxn2_bits;      // largest squared row norm of the previous sweep (float bits)
   unsigned next_maxn2_bits; // the same, being collected in the running sweep
   int status;
+  float off_hist[26];       // off-orthogonality after each sweep (diagnostics)
 };
 
-constexpr int kMaxSweeps = 14;
-constexpr int kInnerSweeps = 10;
+constexpr int kMaxSweeps = 30;
+constexpr int kInnerSweeps = 2;
+constexpr float kCountRel2 = 1e-8f;  // rows below 1e-4 of the largest norm do not hold up convergence
 constexpr float kDeadRel2 = 1e-12f;   // rows below 1e-6 of the largest norm count as zero
 
+// Rows count as orthogonal when |x_i.x_j| <= tol |x_i||x_j|.  An fp32 dot product of length s
+// carries rounding noise of about 6e-8 sqrt(s) relative to |x_i||x_j|; the maximum over all
+// pairs sits a few times above that, so tol is placed at eight times the noise.
 __host__ __device__ inline float jacobi_tol(int s) {
-  float t = 2e-7f * sqrtf((float)s);
-  return t < 2e-6f ? 2e-6f : t;
+  float t = 5e-7f * sqrtf((float)s);
+  return t < 4e-6f ? 4e-6f : t;
 }
 
 __global__ void init_state_kernel(float* __restrict__ Vt, JState* __restrict__ st, int s, int count) {
@@ -50,6 +55,7 @@ __global__ void init_state_kernel(float* __restrict__ Vt, JState* __restrict__ s
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     JState z;
     z.done = 0; z.off_bits = 0; z.sweeps = 0; z.maxn2_bits = 0; z.next_maxn2_bits = 0; z.status = AB_OK;
+    for (int i = 0; i < 26; ++i) z.off_hist[i] = 0.f;
     st[mat] = z;
   }
 }
@@ -59,6 +65,7 @@ __global__ void sweep_end_kernel(JState* __restrict__ st, int count, float tol) 
   if (i >= count) return;
   JState z = st[i];
   if (z.done) return;
+  if (z.sweeps < 26) z.off_hist[z.sweeps] = __uint_as_float(z.off_bits);
   z.sweeps += 1;
   if (__uint_as_float(z.off_bits) <= tol) z.done = 1;
   else if (z.sweeps >= kMaxSweeps) { z.done = 1; z.status = AB_ERR_NOT_CONVERGED; }
@@ -76,13 +83,94 @@ __device__ __forceinline__ void rr_pair(int ne, int t, int k, int& p, int& q) {
   if (p > q) { int tmp = p; p = q; q = tmp; }
 }
 
+// ---- 32 x 32 symmetric eigenproblem in one warp ------------------------------------------------
+// Two-sided cyclic Jacobi with the tournament ordering: pairs always sit at positions (2k, 2k+1),
+// and after every step all positions but 0 move one place round the cycle
+// 2 -> 4 -> ... -> 30 -> 31 -> 29 -> ... -> 3 -> 1 -> 2, so that in 31 steps every pair has met
+// once and everything is back in place.  Lane l holds column l of the working matrix and of Q
+// (rows in registers): column rotations and the column moves are warp shuffles, row rotations
+// and the row moves act on registers with compile-time indices.  No shared memory, no barrier.
+__host__ __device__ constexpr int tour_cycle(int i) { return i < 15 ? 2 * (i + 1) : 31 - 2 * (i - 15); }
+__host__ __device__ constexpr int tour_index(int pos) { return (pos & 1) ? 15 + (31 - pos) / 2 : pos / 2 - 1; }
+__host__ __device__ constexpr int tour_next(int pos) { return pos == 0 ? 0 : tour_cycle((tour_index(pos) + 1) % 31); }
+__host__ __device__ constexpr int tour_prev(int pos) { return pos == 0 ? 0 : tour_cycle((tour_index(pos) + 30) % 31); }
+
+template <int J> struct TourMove {
+  __device__ static __forceinline__ void run(const float (&y)[32], float (&ny)[32]) {
+    ny[tour_next(J)] = y[J];
+    TourMove<J + 1>::run(y, ny);
+  }
+};
+template <> struct TourMove<32> {
+  __device__ static __forceinline__ void run(const float (&)[32], float (&)[32]) {}
+};
+
+// y: column `lane` of the symmetric matrix, q: column `lane` of Q (identity on entry).
+// Rotates pairs whose |m_pq| > thr sqrt(m_pp m_qq); rows whose diagonal is <= dead2 are left alone.
+__device__ __forceinline__ void warp_eig32(float (&y)[32], float (&q)[32], float thr, float dead2, int max_sweeps) {
+  constexpr unsigned FULL = 0xffffffffu;
+  const int lane = threadIdx.x & 31;
+  const bool even = (lane & 1) == 0;
+  const int src = tour_prev(lane);     // the lane whose column moves here after a step
+  for (int sweep = 0; sweep < max_sweeps; ++sweep) {
+    bool rotated = false;
+    for (int step = 0; step < 31; ++step) {
+      float d = 0.f, e = 0.f;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        if (j == lane) d = y[j];
+        if (j == (lane ^ 1)) e = y[j];
+      }
+      const float dpart = __shfl_xor_sync(FULL, d, 1);
+      const float g = __shfl_sync(FULL, e, lane & ~1);
+      const float app = even ? d : dpart, aqq = even ? dpart : d;
+      float c = 1.f, sn = 0.f;
+      if (app > dead2 && aqq > dead2 && app > 0.f && aqq > 0.f && fabsf(g) > thr * sqrtf(app) * sqrtf(aqq)) {
+        const float zeta = (aqq - app) / (2.f * g);
+        const float t = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
+        c = 1.f / sqrtf(1.f + t * t);   // IEEE sqrt and divide: c^2 + s^2 = 1 to an ulp, no drift
+        sn = c * t;
+      }
+      const bool any = __any_sync(FULL, sn != 0.f);
+      if (any) {
+        rotated = true;
+        const float ss = even ? -sn : sn;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {   // columns p, q of M and of Q
+          const float o = __shfl_xor_sync(FULL, y[j], 1);
+          y[j] = c * y[j] + ss * o;
+          const float oq = __shfl_xor_sync(FULL, q[j], 1);
+          q[j] = c * q[j] + ss * oq;
+        }
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {   // rows 2k, 2k+1 of M with that pair's rotation
+          const float ck = __shfl_sync(FULL, c, 2 * k), sk = __shfl_sync(FULL, sn, 2 * k);
+          const float a = y[2 * k], b = y[2 * k + 1];
+          y[2 * k] = ck * a - sk * b;
+          y[2 * k + 1] = sk * a + ck * b;
+        }
+      }
+      float ny[32];
+      TourMove<0>::run(y, ny);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        y[j] = __shfl_sync(FULL, ny[j], src);
+        q[j] = __shfl_sync(FULL, q[j], src);
+      }
+    }
+    if (!rotated) break;
+  }
+}
+
+// One CTA per block pair: PB = 32 rows (16 + 16) or PB = 16 (8 + 8, for long vectors).
 template <int PB>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, int nb, int round,
                    float tol, JState* __restrict__ states) {
   constexpr int HB = PB / 2;          // rows per block
   constexpr int RT = PB / 16;         // register tile of the panel Gram
-  constexpr int LDM = PB + 1;
+  constexpr int LDM = 33;
+  constexpr int LDQ = PB + 4;
   extern __shared__ __align__(16) float smem[];
   const int mat = blockIdx.y;
   JState* st = states + mat;
@@ -93,17 +181,16 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
   if (bj >= nb && nb > 1) return;     // this block sits the round out
   const int ldp = ((s + 3) & ~3) + 4;
   float* P = smem;                    // PB x ldp
-  float* Ms = P + (size_t)PB * ldp;   // PB x LDM
-  float* Qt = Ms + PB * LDM;          // PB x PB, Qt[c][i] = Q[i][c]
-  float* cs = Qt + PB * PB;           // HB
-  float* sn = cs + HB;                // HB
-  int* pq = reinterpret_cast<int*>(sn + HB);   // 2*HB
+  float* Ms = P + (size_t)PB * ldp;   // 32 x LDM (zero beyond PB)
+  float* Qt = Ms + 32 * LDM + 3;      // PB x LDQ, Qt[c][i] = Q[i][c]; (32*33+3) % 4 == 3 -> realigned below
+  Qt = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(Qt) + 15) & ~(uintptr_t)15);
   __shared__ int any_rot;
   const int tid = threadIdx.x;
   float* X = Xall + (size_t)mat * s * s;
   float* V = Vall + (size_t)mat * s * s;
   const float maxn2 = __uint_as_float(st->maxn2_bits);
   const float dead2 = kDeadRel2 * maxn2;
+  const float count2 = kCountRel2 * maxn2;
 
   auto grow = [&](int lr) -> int {    // local panel row -> global row (or -1)
     int g = (lr < HB) ? bi * HB + lr : bj * HB + (lr - HB);
@@ -112,17 +199,17 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
   };
   auto load_panel = [&](const float* src) {
     const int s4 = ldp - 4;           // padded row length handled, multiple of 4
-    for (int idx = tid; idx < PB * s4; idx += 256) {
-      int lr = idx / s4, k = idx - lr * s4;
-      int g = grow(lr);
-      P[(size_t)lr * ldp + k] = (g >= 0 && k < s) ? src[(size_t)g * s + k] : 0.f;
+    for (int lr = tid >> 5; lr < PB; lr += 8) {      // a warp per row: coalesced
+      const int g = grow(lr);
+      for (int k = tid & 31; k < s4; k += 32)
+        P[(size_t)lr * ldp + k] = (g >= 0 && k < s) ? src[(size_t)g * s + k] : 0.f;
     }
   };
   auto store_panel = [&](float* dst) {
-    for (int idx = tid; idx < PB * s; idx += 256) {
-      int lr = idx / s, k = idx - lr * s;
-      int g = grow(lr);
-      if (g >= 0) dst[(size_t)g * s + k] = P[(size_t)lr * ldp + k];
+    for (int lr = tid >> 5; lr < PB; lr += 8) {
+      const int g = grow(lr);
+      if (g < 0) continue;
+      for (int k = tid & 31; k < s; k += 32) dst[(size_t)g * s + k] = P[(size_t)lr * ldp + k];
     }
   };
   auto apply_q = [&]() {              // P <- Q^T P, one panel column per thread at a time
@@ -130,8 +217,9 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
       float col[PB];
 #pragma unroll
       for (int j = 0; j < PB; ++j) col[j] = P[(size_t)j * ldp + k];
+#pragma unroll 4
       for (int i = 0; i < PB; ++i) {
-        const float4* qrow = reinterpret_cast<const float4*>(Qt + i * PB);
+        const float4* qrow = reinterpret_cast<const float4*>(Qt + i * LDQ);
         float acc = 0.f;
 #pragma unroll
         for (int j4 = 0; j4 < PB / 4; ++j4) {
@@ -147,7 +235,7 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
   };
 
   load_panel(X);
-  for (int idx = tid; idx < PB * PB; idx += 256) Qt[idx] = (idx / PB == idx % PB) ? 1.f : 0.f;
+  for (int idx = tid; idx < 32 * LDM; idx += 256) Ms[idx] = 0.f;
   if (tid == 0) any_rot = 0;
   __syncthreads();
 
@@ -186,13 +274,17 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
   // ---- how far from orthogonal is this panel?  (also collects the largest squared norm)
   {
     float worst = 0.f, big = 0.f;
+    int rot = 0;
     for (int idx = tid; idx < PB * PB; idx += 256) {
       int i = idx / PB, j = idx - i * PB;
       float mii = Ms[i * LDM + i], mjj = Ms[j * LDM + j];
       if (i == j) { big = fmaxf(big, mii); continue; }
       if (i < j && mii > dead2 && mjj > dead2 && mii > 0.f && mjj > 0.f) {
         float rel = fabsf(Ms[i * LDM + j]) / (sqrtf(mii) * sqrtf(mjj));
-        worst = fmaxf(worst, rel);
+        if (rel > tol) rot = 1;
+        // rows far below the largest norm are rounding noise of the large ones: they are still
+        // rotated, but the sweep counts as converged without them
+        if (mii > count2 && mjj > count2) worst = fmaxf(worst, rel);
       }
     }
 #pragma unroll
@@ -203,64 +295,27 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
     if ((tid & 31) == 0) {
       atomicMax(&st->off_bits, __float_as_uint(worst));
       atomicMax(&st->next_maxn2_bits, __float_as_uint(big));
-      if (worst > tol) atomicExch(&any_rot, 1);
     }
+    if (rot) atomicExch(&any_rot, 1);
   }
   __syncthreads();
   if (!any_rot) return;               // panel already orthogonal: nothing to write
-  __syncthreads();
 
-  // ---- diagonalise M: parallel cyclic two-sided Jacobi, HB disjoint rotations per step
-  for (int sweep = 0; sweep < kInnerSweeps; ++sweep) {
-    if (tid == 0) any_rot = 0;
-    __syncthreads();
-    for (int t = 0; t < PB - 1; ++t) {
-      if (tid < HB) {
-        int p, q;
-        rr_pair(PB, t, tid, p, q);
-        float app = Ms[p * LDM + p], aqq = Ms[q * LDM + q], apq = Ms[p * LDM + q];
-        float c = 1.f, sv = 0.f;
-        if (app > dead2 && aqq > dead2 && app > 0.f && aqq > 0.f &&
-            fabsf(apq) > 0.25f * tol * sqrtf(app) * sqrtf(aqq)) {
-          float zeta = (aqq - app) / (2.f * apq);
-          float tt = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
-          c = 1.f / sqrtf(1.f + tt * tt);   // IEEE sqrt and divide: c^2 + s^2 = 1 to an ulp, no drift
-          sv = c * tt;
-          any_rot = 1;
-        }
-        cs[tid] = c; sn[tid] = sv; pq[2 * tid] = p; pq[2 * tid + 1] = q;
-      }
-      __syncthreads();
-      // 2x2 blocks of M (rows of pair a, columns of pair b), then rows of Qt
-      for (int task = tid; task < HB * HB + PB * HB; task += 256) {
-        if (task < HB * HB) {
-          int a = task / HB, b = task - a * HB;
-          int pa = pq[2 * a], qa = pq[2 * a + 1], pb = pq[2 * b], qb = pq[2 * b + 1];
-          float ca = cs[a], sa = sn[a], cb = cs[b], sb = sn[b];
-          float m00 = Ms[pa * LDM + pb], m01 = Ms[pa * LDM + qb];
-          float m10 = Ms[qa * LDM + pb], m11 = Ms[qa * LDM + qb];
-          float n00 = cb * m00 - sb * m01, n01 = sb * m00 + cb * m01;
-          float n10 = cb * m10 - sb * m11, n11 = sb * m10 + cb * m11;
-          float r00 = ca * n00 - sa * n10, r10 = sa * n00 + ca * n10;
-          float r01 = ca * n01 - sa * n11, r11 = sa * n01 + ca * n11;
-          if (a == b && sa != 0.f) { r01 = 0.f; r10 = 0.f; }
-          Ms[pa * LDM + pb] = r00; Ms[pa * LDM + qb] = r01;
-          Ms[qa * LDM + pb] = r10; Ms[qa * LDM + qb] = r11;
-        } else {
-          int u = task - HB * HB;
-          int b = u / PB, i = u - b * PB;
-          int pb = pq[2 * b], qb = pq[2 * b + 1];
-          float cb = cs[b], sb = sn[b];
-          float q0 = Qt[pb * PB + i], q1 = Qt[qb * PB + i];
-          Qt[pb * PB + i] = cb * q0 - sb * q1;
-          Qt[qb * PB + i] = sb * q0 + cb * q1;
-        }
-      }
-      __syncthreads();
+  // ---- diagonalise M in warp 0 (the other warps wait at the barrier)
+  if (tid < 32) {
+    float y[32], q[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      y[j] = Ms[j * LDM + tid];
+      q[j] = (j == tid) ? 1.f : 0.f;
     }
-    if (!any_rot) break;              // uniform: read after the step's barrier
-    __syncthreads();
+    warp_eig32(y, q, 0.25f * tol, dead2, kInnerSweeps);
+    if (tid < PB) {
+#pragma unroll
+      for (int i = 0; i < PB; ++i) Qt[tid * LDQ + i] = q[i];
+    }
   }
+  __syncthreads();
 
   // ---- rotate the panel of X, then the same rows of V^T
   apply_q();
@@ -277,7 +332,7 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
 template <int PB>
 size_t jacobi_smem_bytes(int s) {
   const int ldp = ((s + 3) & ~3) + 4;
-  return sizeof(float) * ((size_t)PB * ldp + (size_t)PB * (PB + 1) + (size_t)PB * PB + PB) + sizeof(int) * PB;
+  return sizeof(float) * ((size_t)PB * ldp + 32 * 33 + 8 + (size_t)PB * (PB + 4));
 }
 
 // lam[i] = |row i of X|, perm = indices by descending lam (ties by index).  One CTA per matrix.
@@ -416,7 +471,7 @@ Plan make_plan(const SvdItem& it) {
   p.s = p.tall ? it.n : it.m;
   p.L = p.tall ? it.m : it.n;
   p.r_cap = std::min(it.r_max, p.s);
-  p.pb = p.s <= 768 ? 64 : (p.s <= 1536 ? 32 : 16);
+  p.pb = p.s <= 1536 ? 32 : 16;
   int hb = p.pb / 2;
   p.nb = (p.s + hb - 1) / hb;
   return p;
@@ -517,8 +572,7 @@ int svd_batch(const SvdItem* items, int L, float sigma_cutoff, void* ws, size_t 
     init_state_kernel<<<ig, 256, 0, stream>>>(lo.Vt[s], lo.st[s], s, count);
     AB_LAUNCH_OK();
     int rc;
-    if (p.pb == 64) rc = run_jacobi<64>(lo.X[s], lo.Vt[s], lo.st[s], s, p.nb, count, stream);
-    else if (p.pb == 32) rc = run_jacobi<32>(lo.X[s], lo.Vt[s], lo.st[s], s, p.nb, count, stream);
+    if (p.pb == 32) rc = run_jacobi<32>(lo.X[s], lo.Vt[s], lo.st[s], s, p.nb, count, stream);
     else rc = run_jacobi<16>(lo.X[s], lo.Vt[s], lo.st[s], s, p.nb, count, stream);
     AB_TRY(rc);
     norms_sort_kernel<<<count, 256, (size_t)s * sizeof(float), stream>>>(
