@@ -29,6 +29,9 @@ using namespace tc;
 
 constexpr int kAtomBytes = 16384;      // 128 rows x 128 bytes
 constexpr int kMaxStages = 6;
+constexpr int kMaxStages2 = 6;         // 32 KB slots of the second product, carved from the same ring memory
+constexpr int kChunk = 256;            // output columns per accumulator of the second product
+constexpr int kAtom2Bytes = kChunk * 128;   // one 256 x 64 tile of F2
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kTmemCols = 512;
 constexpr int kEpiThreads = 128;
@@ -38,16 +41,18 @@ struct RowChainParams {
   int P;         // width of Out (0: first product only)
   int r;
   int nk1;       // ceil(K1 / 64)
-  int nchunks;   // ceil(P / 128)
+  int nchunks;   // ceil(P / 256)
   int natoms;    // ceil(r / 64)
   int ns;        // ring stages
   int slot_bytes;
+  int ns2;       // stages of the second product's ring (one 128 x 64 atom of F2 each)
   int save_s;    // 1: copy S to global through tmS
   int* status;
 };
 
 struct Bars {
   uint64_t full[kMaxStages], empty[kMaxStages];
+  uint64_t full2[kMaxStages2], empty2[kMaxStages2];
   uint64_t t_full, s_ready;
   uint64_t acc_full[2], acc_empty[2];
   uint32_t tmem_base;
@@ -70,12 +75,12 @@ __device__ __forceinline__ bool epi_wait(Bars* b, uint64_t* bar, uint32_t parity
   return *reinterpret_cast<volatile int*>(&b->epi_abort) == 0;
 }
 
-__device__ __forceinline__ void store_bf16x16_swizzled(uint8_t* row_base, int row, int c0, const float (&v)[16]) {
+__device__ __forceinline__ void store_bf16x16_swizzled(uint8_t* row_base, int row, int c0, const uint32_t (&v)[16]) {
   // 16 consecutive columns c0..c0+15 (c0 % 16 == 0) of a 128-byte row inside a swizzled atom
   uint32_t w[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
     w[i] = *reinterpret_cast<uint32_t*>(&h);
   }
   const int ch = (c0 & 63) >> 3;
@@ -98,9 +103,15 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row0 = blockIdx.x * 128;
+  // All CTAs walk the same factor tiles.  Started together they would all ask L2 for the same
+  // few lines at the same moment (measured: 29 GB/s per SM); each CTA therefore starts its walk
+  // at a different slab / chunk and wraps round.  The order is a function of blockIdx only.
+  const int rot1 = blockIdx.x % p.nk1;
+  const int rot2 = p.nchunks > 0 ? (blockIdx.x * 5) % p.nchunks : 0;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.ns; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
+    for (int i = 0; i < p.ns2; ++i) { mbar_init(&bars->full2[i], 1); mbar_init(&bars->empty2[i], 1); }
     mbar_init(&bars->t_full, 1);
     mbar_init(&bars->s_ready, kEpiThreads);
     for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 4); }
@@ -115,8 +126,10 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
+  // T (r <= 256 columns) is read out into S before the second product starts, so the two
+  // 256-column accumulators of the second product reuse its columns.
   const uint32_t tT = tmem_base;
-  const uint32_t tAcc0 = tmem_base + 256;
+  const uint32_t tAcc0 = tmem_base;
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -128,16 +141,21 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
         if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
         uint8_t* dst = ring + (size_t)slot * p.slot_bytes;
         mbar_arrive_expect_tx(&bars->full[slot], kAtomBytes + p.r * 128);
-        tma_load_2d(dst, &tmIn, &bars->full[slot], ks * 64, row0);
-        tma_load_2d(dst + kAtomBytes, &tmF1, &bars->full[slot], ks * 64, 0);
+        const int kr = (ks + rot1) % p.nk1;   // every CTA starts on a different slab: see rot1
+        tma_load_2d(dst, &tmIn, &bars->full[slot], kr * 64, row0);
+        tma_load_2d(dst + kAtomBytes, &tmF1, &bars->full[slot], kr * 64, 0);
       }
+      // The second product re-cuts the ring memory into 16 KB slots, so that many atoms of F2
+      // are in flight at once (L2 latency x the rate the MMAs need is > 100 KB); it may only be
+      // refilled once every MMA of the first product has read its slabs.
+      if (ok && p.nchunks > 0 && !mbar_wait(&bars->t_full, 0)) { raise_timeout(bars, p.status); ok = false; }
+      i = 0;
       for (int c = 0; c < p.nchunks && ok; ++c) {
         for (int j = 0; j < p.natoms; ++j, ++i) {
-          const int slot = i % p.ns, ph = (i / p.ns) & 1;
-          if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
-          uint8_t* dst = ring + (size_t)slot * p.slot_bytes;
-          mbar_arrive_expect_tx(&bars->full[slot], kAtomBytes);
-          tma_load_2d(dst, &tmF2, &bars->full[slot], j * 64, c * 128);
+          const int slot = i % p.ns2, ph = (i / p.ns2) & 1;
+          if (!mbar_wait(&bars->empty2[slot], ph ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
+          mbar_arrive_expect_tx(&bars->full2[slot], kAtom2Bytes);
+          tma_load_2d(ring + (size_t)slot * kAtom2Bytes, &tmF2, &bars->full2[slot], j * 64, ((c + rot2) % p.nchunks) * kChunk);
         }
       }
     }
@@ -145,7 +163,7 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc1 = instr_desc_bf16(128, p.r, 0, 0);
-      const uint32_t idesc2 = instr_desc_bf16(128, 128, 0, 0);
+      const uint32_t idesc2 = instr_desc_bf16(128, kChunk, 0, 0);
       int i = 0;
       bool ok = true;
       for (int ks = 0; ks < p.nk1; ++ks, ++i) {
@@ -154,7 +172,7 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
         tc_fence_after();
         const uint32_t sa = smem_u32(ring + (size_t)slot * p.slot_bytes);
         const uint64_t da = smem_desc_sw128(sa, 16), db = smem_desc_sw128(sa + kAtomBytes, 16);
-        int ksteps = (p.K1 - ks * 64 + 15) >> 4;
+        int ksteps = (p.K1 - ((ks + rot1) % p.nk1) * 64 + 15) >> 4;
         if (ksteps > 4) ksteps = 4;
         for (int kk = 0; kk < ksteps; ++kk) tc_mma_bf16(tT, da + 2 * kk, db + 2 * kk, idesc1, (ks | kk) != 0);
         tc_commit(&bars->empty[slot]);
@@ -166,21 +184,22 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
           tc_fence_after();
         }
       }
+      i = 0;
       for (int c = 0; c < p.nchunks && ok; ++c) {
         const int b = c & 1;
         if (!mbar_wait(&bars->acc_empty[b], ((c >> 1) & 1) ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
         tc_fence_after();
-        const uint32_t tacc = tAcc0 + 128 * b;
+        const uint32_t tacc = tAcc0 + kChunk * b;
         for (int j = 0; j < p.natoms; ++j, ++i) {
-          const int slot = i % p.ns, ph = (i / p.ns) & 1;
-          if (!mbar_wait(&bars->full[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
+          const int slot = i % p.ns2, ph = (i / p.ns2) & 1;
+          if (!mbar_wait(&bars->full2[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
           tc_fence_after();
           const uint64_t da = smem_desc_sw128(smem_u32(S + j * kAtomBytes), 16);
-          const uint64_t db = smem_desc_sw128(smem_u32(ring + (size_t)slot * p.slot_bytes), 16);
+          const uint64_t db = smem_desc_sw128(smem_u32(ring + (size_t)slot * kAtom2Bytes), 16);
           int ksteps = (p.r - j * 64) >> 4;
           if (ksteps > 4) ksteps = 4;
           for (int kk = 0; kk < ksteps; ++kk) tc_mma_bf16(tacc, da + 2 * kk, db + 2 * kk, idesc2, (j | kk) != 0);
-          tc_commit(&bars->empty[slot]);
+          tc_commit(&bars->empty2[slot]);
         }
         if (ok) tc_commit(&bars->acc_full[b]);
       }
@@ -194,10 +213,15 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
     bool ok = epi_wait(bars, &bars->t_full, 0, p.status);
     if (ok) {
       tc_fence_after();
-      for (int c0 = 0; c0 < p.r; c0 += 16) {
-        float v[16];
-        tmem_ld16(tT + lane_base + c0, v);
-        store_bf16x16_swizzled(S + (c0 >> 6) * kAtomBytes + row * 128, row, c0, v);
+      for (int c0 = 0; c0 < p.r; c0 += 64) {       // up to four 16-column loads in flight per wait
+        uint32_t v[4][16];
+#pragma unroll
+        for (int g = 0; g < 4; ++g)
+          if (c0 + g * 16 < p.r) tmem_ld16_nowait(tT + lane_base + c0 + g * 16, v[g]);
+        tmem_wait_ld();
+#pragma unroll
+        for (int g = 0; g < 4; ++g)
+          if (c0 + g * 16 < p.r) store_bf16x16_swizzled(S + (c0 >> 6) * kAtomBytes + row * 128, row, c0 + g * 16, v[g]);
       }
       tc_fence_before();
       fence_proxy_async_smem();
@@ -215,27 +239,30 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
       ok = epi_wait(bars, &bars->acc_full[b], (c >> 1) & 1, p.status);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t tacc = tAcc0 + 128 * b + lane_base;
-      for (int h = 0; h < 2; ++h) {
-        uint8_t* buf = stg + h * kAtomBytes;
+      const uint32_t tacc = tAcc0 + kChunk * b + lane_base;
+      for (int h = 0; h < kChunk / 64; ++h) {
+        uint8_t* buf = stg + (h & 1) * kAtomBytes;
+        uint32_t v[4][16];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) tmem_ld16_nowait(tacc + h * 64 + g * 16, v[g]);
+        tmem_wait_ld();
+        if (h == kChunk / 64 - 1) {                  // the last columns are in registers: release the accumulator
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->acc_empty[b]);
+        }
         if (issuer) tma_store_wait_read<1>();       // the store that last read this buffer is done
         named_bar_sync(1, kEpiThreads);
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          float v[16];
-          tmem_ld16(tacc + h * 64 + g * 16, v);
-          store_bf16x16_swizzled(buf + row * 128, row, g * 16, v);
-        }
+        for (int g = 0; g < 4; ++g) store_bf16x16_swizzled(buf + row * 128, row, g * 16, v[g]);
         fence_proxy_async_smem();
         named_bar_sync(1, kEpiThreads);
-        if (issuer && c * 128 + h * 64 < p.P) {
-          tma_store_2d(&tmOut, buf, c * 128 + h * 64, row0);
+        const int col = ((c + rot2) % p.nchunks) * kChunk + h * 64;
+        if (issuer && col < p.P) {
+          tma_store_2d(&tmOut, buf, col, row0);
           tma_store_commit();
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->acc_empty[b]);
     }
     if (issuer) tma_store_wait_all();
   }
@@ -464,7 +491,7 @@ int make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint
   return rc == CUDA_SUCCESS ? AB_OK : AB_ERR_CUDA;
 }
 
-struct RowPlan { int natoms, ns, slot_bytes; size_t smem; };
+struct RowPlan { int natoms, ns, slot_bytes, ns2; size_t smem; };
 RowPlan row_plan(int r) {
   RowPlan pl;
   pl.natoms = (r + 63) / 64;
@@ -473,6 +500,8 @@ RowPlan row_plan(int r) {
   pl.ns = (kSmemLimit - fixed) / pl.slot_bytes;
   if (pl.ns > kMaxStages) pl.ns = kMaxStages;
   pl.smem = (size_t)fixed + (size_t)pl.ns * pl.slot_bytes;
+  pl.ns2 = pl.ns * pl.slot_bytes / kAtom2Bytes;
+  if (pl.ns2 > kMaxStages2) pl.ns2 = kMaxStages2;
   return pl;
 }
 
@@ -516,14 +545,14 @@ BwdWs bwd_ws(void* ws, int64_t N, int m, int n, int r) {
 int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1, const void* F2, int ldF2, int P,
                      void* Out, void* Sg, int r, int* status, cudaStream_t st) {
   RowPlan pl = row_plan(r);
-  if (pl.ns < 2) return AB_ERR_UNSUPPORTED;
+  if (pl.ns < 2 || pl.ns2 < 2) return AB_ERR_UNSUPPORTED;
   CUtensorMap tmIn, tmF1, tmF2, tmOut, tmS;
   AB_TRY(make_map(&tmIn, In, (uint64_t)N, K1, K1, 64, 128));
   AB_TRY(make_map(&tmF1, F1, r, K1, ldF1, 64, r));
   const bool second = Out != nullptr && P > 0;
   // unused maps still have to be valid objects: alias them to the first operand
   if (second) {
-    AB_TRY(make_map(&tmF2, F2, P, r, ldF2, 64, 128));
+    AB_TRY(make_map(&tmF2, F2, P, r, ldF2, 64, kChunk));
     AB_TRY(make_map(&tmOut, Out, (uint64_t)N, P, P, 64, 128));
   } else {
     tmF2 = tmIn;
@@ -532,8 +561,9 @@ int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1
   if (Sg) AB_TRY(make_map(&tmS, Sg, (uint64_t)N, r, r, 64, 128));
   else tmS = tmIn;
   RowChainParams p;
-  p.K1 = K1; p.P = second ? P : 0; p.r = r; p.nk1 = (K1 + 63) / 64; p.nchunks = second ? (P + 127) / 128 : 0;
-  p.natoms = pl.natoms; p.ns = pl.ns; p.slot_bytes = pl.slot_bytes; p.save_s = Sg ? 1 : 0; p.status = status;
+  p.K1 = K1; p.P = second ? P : 0; p.r = r; p.nk1 = (K1 + 63) / 64; p.nchunks = second ? (P + kChunk - 1) / kChunk : 0;
+  p.natoms = pl.natoms; p.ns = pl.ns; p.slot_bytes = pl.slot_bytes; p.ns2 = pl.ns2; p.save_s = Sg ? 1 : 0;
+  p.status = status;
   AB_CUDA_OK(cudaFuncSetAttribute(row_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
   const unsigned grid = (unsigned)((N + 127) / 128);
   row_chain_kernel<<<grid, 192, pl.smem, st>>>(tmIn, tmF1, tmF2, tmOut, tmS, p);
@@ -551,7 +581,7 @@ bool chain_tc_supported(int64_t N, int m, int n, int r, int ldA, int ldB, int dt
   if (N > (int64_t)1 << 30) return false;
   if (!aligned(x, 16) || !aligned(A, 16) || !aligned(B, 16) || !aligned(y, 16)) return false;
   if (!device_is_sm100() || !encode_fn()) return false;
-  return row_plan(r).ns >= 2;
+  return row_plan(r).ns >= 2 && row_plan(r).ns2 >= 2;
 }
 
 size_t chain_tc_forward_ws(int64_t, int, int, int) { return 256; }
