@@ -234,6 +234,7 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
         }
       }
     }
+    int nstores = 0;
     for (int c = 0; c < p.nchunks && ok; ++c) {
       const int b = c & 1;
       ok = epi_wait(bars, &bars->acc_full[b], (c >> 1) & 1, p.status);
@@ -241,24 +242,31 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
       tc_fence_after();
       const uint32_t tacc = tAcc0 + kChunk * b + lane_base;
       for (int h = 0; h < kChunk / 64; ++h) {
-        uint8_t* buf = stg + (h & 1) * kAtomBytes;
+        const int col = ((c + rot2) % p.nchunks) * kChunk + h * 64;
+        const bool live = col < p.P;                 // columns beyond the output are not staged at all
         uint32_t v[4][16];
+        if (live) {
 #pragma unroll
-        for (int g = 0; g < 4; ++g) tmem_ld16_nowait(tacc + h * 64 + g * 16, v[g]);
-        tmem_wait_ld();
+          for (int g = 0; g < 4; ++g) tmem_ld16_nowait(tacc + h * 64 + g * 16, v[g]);
+          tmem_wait_ld();
+        }
         if (h == kChunk / 64 - 1) {                  // the last columns are in registers: release the accumulator
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars->acc_empty[b]);
         }
-        if (issuer) tma_store_wait_read<1>();       // the store that last read this buffer is done
+        if (!live) continue;
+        // staging tiles alternate with every store issued, so "at most one store still reading"
+        // always means the other tile
+        uint8_t* buf = stg + (nstores & 1) * kAtomBytes;
+        ++nstores;
+        if (issuer) tma_store_wait_read<1>();
         named_bar_sync(1, kEpiThreads);
 #pragma unroll
         for (int g = 0; g < 4; ++g) store_bf16x16_swizzled(buf + row * 128, row, g * 16, v[g]);
         fence_proxy_async_smem();
         named_bar_sync(1, kEpiThreads);
-        const int col = ((c + rot2) % p.nchunks) * kChunk + h * 64;
-        if (issuer && col < p.P) {
+        if (issuer) {
           tma_store_2d(&tmOut, buf, col, row0);
           tma_store_commit();
         }
