@@ -70,6 +70,24 @@ int gemm_simt(const void* A, int a_dt, int64_t sAm, int64_t sAk,
               void* C, int c_dt, int64_t ldc,
               int64_t M, int64_t N, int64_t K, cudaStream_t st);
 
+// Batched form for the small products of the factored group sync: problem z of the batch is
+// described by one GemmDesc in device memory.  fp32 operands; optional diagonal scalings
+//   C[i,j] = rs(i) * cs(j) * sum_k A(i,k) * ks(k) * B(k,j)
+// where each of rs/cs/ks is derived from a vector v sorted in descending order:
+//   mode 0: 1,  mode 1: sqrt(v),  mode 2: 1/sqrt(v);  entries with v <= thr * v[0] count as 0.
+// Rows >= *live_rows and columns >= *live_cols (device ints, optional) are written as zero.
+struct GemmDesc {
+  const float* A; const float* B; void* C;
+  int64_t sAm, sAk, sBk, sBn, ldc;
+  int M, N, K;
+  int c_bf16;
+  const float* row_vec; const float* col_vec; const float* k_vec;
+  int row_mode, col_mode, k_mode;
+  float thr;
+  const int* live_rows; const int* live_cols;
+};
+int gemm_simt_batched(const GemmDesc* d_descs, int count, int max_M, int max_N, cudaStream_t st);
+
 // ---- fused tensor-core chain (ab_chain_tc.cu) --------------------------------------------------
 bool chain_tc_supported(int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
                         const void* x, const void* A, const void* B, const void* y);

@@ -93,7 +93,95 @@ int launch(const void* A, int64_t sAm, int64_t sAk, const void* B, int64_t sBk, 
   return AB_OK;
 }
 
+__device__ __forceinline__ float diag_scale(const float* v, int idx, int mode, float thr) {
+  if (mode == 0 || v == nullptr) return 1.f;
+  const float x = v[idx];
+  if (!(x > thr * v[0]) || !(x > 0.f)) return 0.f;
+  return mode == 1 ? sqrtf(x) : 1.f / sqrtf(x);
+}
+
+__global__ void __launch_bounds__(256)
+gemm_simt_batched_kernel(const GemmDesc* __restrict__ descs) {
+  const GemmDesc d = descs[blockIdx.z];
+  const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
+  if (m0 >= d.M || n0 >= d.N) return;
+  __shared__ float As[BK][BM + PAD];
+  __shared__ float Bs[BK][BN + PAD];
+  const int tid = threadIdx.x;
+  const int tx = tid & 15, ty = tid >> 4;
+  const bool a_kfast = (d.sAk == 1), b_nfast = (d.sBn == 1);
+  double acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+  for (int64_t k0 = 0; k0 < d.K; k0 += BK) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      int idx = tid + e * 256;
+      int kk, mm;
+      if (a_kfast) { kk = idx % BK; mm = idx / BK; } else { mm = idx % BM; kk = idx / BM; }
+      int64_t gm = m0 + mm, gk = k0 + kk;
+      float av = 0.f;
+      if (gm < d.M && gk < d.K) av = d.A[gm * d.sAm + gk * d.sAk] * diag_scale(d.k_vec, (int)gk, d.k_mode, d.thr);
+      As[kk][mm] = av;
+      int nn;
+      if (b_nfast) { nn = idx % BN; kk = idx / BN; } else { kk = idx % BK; nn = idx / BK; }
+      int64_t gn = n0 + nn;
+      gk = k0 + kk;
+      Bs[kk][nn] = (gn < d.N && gk < d.K) ? d.B[gk * d.sBk + gn * d.sBn] : 0.f;
+    }
+    __syncthreads();
+    float part[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) part[i][j] = 0.f;
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) part[i][j] = fmaf(av[i], bv[j], part[i][j]);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] += (double)part[i][j];
+    __syncthreads();
+  }
+  const int live_r = d.live_rows ? *d.live_rows : d.M;
+  const int live_c = d.live_cols ? *d.live_cols : d.N;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    int64_t gm = m0 + ty * 4 + i;
+    if (gm >= d.M) continue;
+    const float rs = gm < live_r ? diag_scale(d.row_vec, (int)gm, d.row_mode, d.thr) : 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      int64_t gn = n0 + tx * 4 + j;
+      if (gn >= d.N) continue;
+      const float cs = gn < live_c ? diag_scale(d.col_vec, (int)gn, d.col_mode, d.thr) : 0.f;
+      const float v = (float)acc[i][j] * rs * cs;
+      if (d.c_bf16) static_cast<bf16*>(d.C)[gm * d.ldc + gn] = __float2bfloat16_rn(v);
+      else static_cast<float*>(d.C)[gm * d.ldc + gn] = v;
+    }
+  }
+}
+
 }  // namespace
+
+int gemm_simt_batched(const GemmDesc* d_descs, int count, int max_M, int max_N, cudaStream_t st) {
+  if (count <= 0 || max_M <= 0 || max_N <= 0) return AB_OK;
+  dim3 grid((unsigned)((max_N + BN - 1) / BN), (unsigned)((max_M + BM - 1) / BM), (unsigned)count);
+  if (grid.y > 65535u || grid.z > 65535u) return AB_ERR_UNSUPPORTED;
+  gemm_simt_batched_kernel<<<grid, 256, 0, st>>>(d_descs);
+  AB_LAUNCH_OK();
+  return AB_OK;
+}
 
 int gemm_simt(const void* A, int a_dt, int64_t sAm, int64_t sAk,
               const void* B, int b_dt, int64_t sBk, int64_t sBn,
