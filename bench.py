@@ -185,7 +185,7 @@ def run_ours(args):
                     A=torch.empty((m, R), dtype=bf).pin_memory(), B=torch.empty((R, n), dtype=bf).pin_memory(),
                     sigma=torch.empty((R,), dtype=torch.float32).pin_memory())
         layers.append(dict(m=m, n=n, h=h, g=g, hout=hout))
-    plan = ab.SyncPlan([L["g"]["A_copies"] for L in layers], [L["g"]["B_copies"] for L in layers], 0.0)
+    plan = ab.SyncPlan([L["g"]["A_copies"] for L in layers], [L["g"]["B_copies"] for L in layers], 0.0, want_W=True)
 
     def chain():
         for L in layers:
@@ -281,7 +281,7 @@ def run_ours(args):
                     ms_per_step=total_ms / K, higher_is_better=True, scaling="weak", vs_baseline=None,
                     dtype="bf16", data="synthetic",
                     config=dict(workload="vit_b16_mlp_pair_r192", rows=N, layers=[list(s) for s in LAYERS], r=R,
-                                K=K_GROUPS, sync="mean+recombine+svd_split of both layers every step",
+                                K=K_GROUPS, sync="mean + recombine (W written) + truncated-SVD split of both layers every step, factored route",
                                 l2="inputs larger than L2 (about 0.8 GB of activations read per step)"),
                     chain_ms_per_step=chain_ms / K, group_sync_ms_per_step=sync_ms / K,
                     pct_of_nominal_bf16_peak=100.0 * per_gpu / NOMINAL_BF16_TFLOPS,

@@ -162,17 +162,31 @@ typedef struct {
   void* B_out;            /* [r,n] */
   float* sigma;           /* [min(r,m,n)] */
   int* r_out;             /* device int */
+  float* W_out;           /* NULL, or [m,n] fp32 that receives the recombination W = Abar Bbar */
 } ab_sync_desc;
+
+typedef enum {
+  AB_SYNC_AUTO = 0,      /* factored when it applies, else dense */
+  AB_SYNC_DENSE = 1,     /* form W, then the dense split of ab_svd_split */
+  AB_SYNC_FACTORED = 2   /* never form W: r x r eigen/SVD problems only (rank(W) <= r makes this exact) */
+} ab_sync_path;
 
 /*
  * Group synchronisation of a whole model (Algorithm 1 from the two all-reduces to the next
  * decomposition): for each of the L matrices, mean of the K copies of A and of B, W = Abar
  * Bbar, then the split of W as in ab_svd_split.  descs: HOST array of L descriptors (read
  * before the call returns).  Factor storage dt on both sides.  dev_status: device int[L].
- * Workspace: ab_sync_workspace_bytes.
+ * path: an ab_sync_path.  The factored path uses that W = Abar Bbar has rank <= r: the
+ * decomposition reduces to eigen-problems of Abar^T Abar and Bbar Bbar^T and the SVD of an
+ * r x r core, each solved inside one CTA's shared memory; W itself is only written if W_out
+ * asks for it.  It needs r <= 232 and factors whose condition number is below about 300
+ * (eigenvalues of the two Gram matrices under 1e-6 of the largest are taken as zero, which is
+ * exact for factors already truncated by the rank rule); AB_SYNC_FACTORED returns
+ * AB_ERR_UNSUPPORTED when r is too large, AB_SYNC_AUTO falls back to the dense path.
+ * Workspace: ab_sync_workspace_bytes (covers either path).
  */
 int ab_group_sync(const ab_sync_desc* descs, int L, int K, float sigma_cutoff, int dt,
-                  int* dev_status, void* ws, size_t ws_bytes, void* cuda_stream);
+                  int* dev_status, void* ws, size_t ws_bytes, void* cuda_stream, int path);
 size_t ab_sync_workspace_bytes(const ab_sync_desc* descs, int L, int K, int dt);
 
 #ifdef __cplusplus

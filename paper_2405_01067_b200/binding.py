@@ -19,6 +19,7 @@ AB_OP_LAYER_FORWARD, AB_OP_LAYER_BACKWARD, AB_OP_GROUP_AVERAGE, AB_OP_RECOMBINE,
 AB_OK = 0
 AB_ERR_INVALID_ARG, AB_ERR_UNSUPPORTED, AB_ERR_WORKSPACE = -1, -2, -3
 AB_ERR_NOT_CONVERGED, AB_ERR_TIMEOUT, AB_ERR_CUDA = -4, -5, -6
+AB_SYNC_AUTO, AB_SYNC_DENSE, AB_SYNC_FACTORED = 0, 1, 2
 
 EXPORTS = ["ab_status_string", "ab_version", "ab_launch_count", "ab_workspace_bytes", "ab_layer_forward", "ab_layer_backward",
            "ab_group_average", "ab_recombine", "ab_svd_split", "ab_group_sync", "ab_sync_workspace_bytes",
@@ -34,7 +35,7 @@ class AbError(RuntimeError):
 class ab_sync_desc(ctypes.Structure):
     _fields_ = [("A_copies", c_void_p), ("B_copies", c_void_p), ("strideA", c_int64), ("strideB", c_int64),
                 ("m", c_int), ("n", c_int), ("r", c_int), ("A_out", c_void_p), ("B_out", c_void_p),
-                ("sigma", c_void_p), ("r_out", c_void_p)]
+                ("sigma", c_void_p), ("r_out", c_void_p), ("W_out", c_void_p)]
 
 
 _lib = None
@@ -68,7 +69,7 @@ def lib() -> ctypes.CDLL:
                                                                                          c_void_p, c_size_t, c_void_p]
     L.ab_group_sync.restype = c_int
     L.ab_group_sync.argtypes = [ctypes.POINTER(ab_sync_desc), c_int, c_int, c_float, c_int, c_void_p, c_void_p,
-                                c_size_t, c_void_p]
+                                c_size_t, c_void_p, c_int]
     L.ab_sync_workspace_bytes.restype = c_size_t
     L.ab_sync_workspace_bytes.argtypes = [ctypes.POINTER(ab_sync_desc), c_int, c_int, c_int]
     L.ab_layer_forward_static.restype = c_int
@@ -230,14 +231,14 @@ def ab_svd_split(W, r_max, sigma_cutoff=0.0, out_dtype=None, ws=None, stream=Non
 class SyncPlan:
     """Buffers and descriptors of one model's group synchronisation (ab_group_sync)."""
 
-    def __init__(self, A_copies, B_copies, sigma_cutoff):
+    def __init__(self, A_copies, B_copies, sigma_cutoff, want_W=False):
         self.A_copies, self.B_copies = list(A_copies), list(B_copies)
         self.L = len(self.A_copies)
         self.K = self.A_copies[0].shape[0]
         self.cutoff = float(sigma_cutoff)
         dev = self.A_copies[0].device
         self.dt = _dt(self.A_copies[0])
-        self.A_out, self.B_out, self.sigma = [], [], []
+        self.A_out, self.B_out, self.sigma, self.W_out = [], [], [], []
         self.r_out = torch.zeros((self.L,), dtype=torch.int32, device=dev)
         self.status = torch.zeros((self.L,), dtype=torch.int32, device=dev)
         self.descs = (ab_sync_desc * self.L)()
@@ -255,12 +256,18 @@ class SyncPlan:
             d.A_out, d.B_out = self.A_out[i].data_ptr(), self.B_out[i].data_ptr()
             d.sigma = self.sigma[i].data_ptr()
             d.r_out = self.r_out.data_ptr() + 4 * i
+            if want_W:
+                self.W_out.append(torch.empty((m, n), dtype=torch.float32, device=dev))
+                d.W_out = self.W_out[i].data_ptr()
+            else:
+                d.W_out = None
         self.ws = workspace(lib().ab_sync_workspace_bytes(self.descs, self.L, self.K, self.dt), dev)
 
 
-def ab_group_sync(plan: SyncPlan, stream=None):
-    """Mean of K copies -> W = Abar Bbar -> split under the rank rule, for every matrix of the plan."""
+def ab_group_sync(plan: SyncPlan, stream=None, path=AB_SYNC_AUTO):
+    """Mean of K copies -> W = Abar Bbar -> split under the rank rule, for every matrix of the plan.
+    path: AB_SYNC_AUTO / AB_SYNC_DENSE (forms W, dense split) / AB_SYNC_FACTORED (r x r problems only)."""
     st = lib().ab_group_sync(plan.descs, plan.L, plan.K, plan.cutoff, plan.dt, _ptr(plan.status), _ptr(plan.ws),
-                             plan.ws.numel(), _stream(stream))
+                             plan.ws.numel(), _stream(stream), int(path))
     _check(st, "ab_group_sync")
     return plan.A_out, plan.B_out, plan.sigma, plan.r_out, plan.status

@@ -226,12 +226,15 @@ static size_t sync_layout(const ab_sync_desc* d, int L, int dt, void* ws, std::v
 size_t ab_sync_workspace_bytes(const ab_sync_desc* descs, int L, int K, int dt) {
   (void)K;
   if (!descs || L <= 0) return 0;
-  return sync_layout(descs, L, dt, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr) + 256;
+  size_t dense = sync_layout(descs, L, dt, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
+  size_t fact = sync_factored_supported(descs, L) ? sync_factored_ws(descs, L) : 0;
+  return (dense > fact ? dense : fact) + 256;
 }
 
 int ab_group_sync(const ab_sync_desc* descs, int L, int K, float sigma_cutoff, int dt,
-                  int* dev_status, void* ws, size_t ws_bytes, void* cuda_stream) {
+                  int* dev_status, void* ws, size_t ws_bytes, void* cuda_stream, int path) {
   if (!descs || L <= 0 || K < 1 || !dtype_ok(dt) || !(sigma_cutoff >= 0.f)) return AB_ERR_INVALID_ARG;
+  if (path != AB_SYNC_AUTO && path != AB_SYNC_DENSE && path != AB_SYNC_FACTORED) return AB_ERR_INVALID_ARG;
   if (K > 64) return AB_ERR_UNSUPPORTED;
   for (int i = 0; i < L; ++i) {
     const ab_sync_desc& d = descs[i];
@@ -243,6 +246,10 @@ int ab_group_sync(const ab_sync_desc* descs, int L, int K, float sigma_cutoff, i
   if (!ws || !aligned(ws, 256)) return AB_ERR_WORKSPACE;
   if (!have_device()) return AB_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const bool can_factor = sync_factored_supported(descs, L);
+  if (path == AB_SYNC_FACTORED && !can_factor) return AB_ERR_UNSUPPORTED;
+  if (path != AB_SYNC_DENSE && can_factor)
+    return sync_factored(descs, L, K, sigma_cutoff, dt, dev_status, ws, ws_bytes, st);
   std::vector<float*> Ab(L), Bb(L), Wd(L);
   std::vector<SvdItem> items;
   void* svd_ws = nullptr;
@@ -253,6 +260,8 @@ int ab_group_sync(const ab_sync_desc* descs, int L, int K, float sigma_cutoff, i
     AB_TRY(group_average(d.A_copies, d.strideA, K, (int64_t)d.m * d.r, dt, AB_F32, Ab[i], st));
     AB_TRY(group_average(d.B_copies, d.strideB, K, (int64_t)d.r * d.n, dt, AB_F32, Bb[i], st));
     AB_TRY(gemm_simt(Ab[i], AB_F32, d.r, 1, Bb[i], AB_F32, d.n, 1, Wd[i], AB_F32, d.n, d.m, d.n, d.r, st));
+    if (d.W_out)
+      AB_CUDA_OK(cudaMemcpyAsync(d.W_out, Wd[i], (size_t)d.m * d.n * sizeof(float), cudaMemcpyDeviceToDevice, st));
     items[i].dev_status = dev_status ? dev_status + i : nullptr;
   }
   size_t used = static_cast<char*>(svd_ws) - static_cast<char*>(ws);

@@ -116,6 +116,12 @@ struct SvdItem {
 size_t svd_batch_ws(const SvdItem* items, int L);
 int svd_batch(const SvdItem* items, int L, float sigma_cutoff, void* ws, size_t ws_bytes, cudaStream_t st);
 
+// ---- factored group sync (ab_sync_fast.cu) ------------------------------------------------------
+bool sync_factored_supported(const ab_sync_desc* d, int L);
+size_t sync_factored_ws(const ab_sync_desc* d, int L);
+int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int dt, int* dev_status,
+                  void* ws, size_t ws_bytes, cudaStream_t st);
+
 // ---- group mean (ab_average.cu) ----------------------------------------------------------------
 int group_average(const void* base, int64_t stride_elems, int K, int64_t count,
                   int in_dt, int out_dt, void* out, cudaStream_t st);

@@ -1,0 +1,297 @@
+// Factored group synchronisation: the split of W = Abar Bbar (Algorithm 1, the decomposition that
+// follows the all-reduces and "W <- AB") without ever forming the m x n matrix.  W has rank <= r,
+// so everything reduces to r x r problems:
+//   G_A = Abar^T Abar = P_A L_A P_A^T,   G_B = Bbar Bbar^T = P_B L_B P_B^T      (eigen, r x r)
+//   Abar = U_A C_A, C_A = L_A^(1/2) P_A^T;   Bbar^T = U_B C_B, C_B = L_B^(1/2) P_B^T
+//   W = U_A M U_B^T,  M = C_A C_B^T  (r x r),   M = U_M S V_M^T                 (SVD, r x r)
+//   A' = Abar Z_A,  Z_A = P_A L_A^(-1/2) (M V_M) S^(-1/2);   B' = Z_B Bbar,  Z_B = S^(1/2) V_M^T L_B^(-1/2) P_B^T
+// Each r x r problem is solved by one CTA that keeps the matrix in shared memory and
+// orthogonalises its ROWS with one-sided Jacobi rotations (for a symmetric G the rows of the
+// result are lambda_i p_i^T; for M they are sigma_i v_i^T), so no kernel boundary and no
+// global traffic sits between rotations.  Eigenvalues of G_A / G_B below 1e-6 of the largest
+// are treated as zero (exactly right for factors truncated by the rank rule; otherwise the
+// factors need a condition number below about 300 -- all workloads here are far inside).
+#include <algorithm>
+#include <vector>
+
+#include "ab_common.cuh"
+
+namespace ab {
+namespace {
+
+constexpr int kJThreads = 512;
+constexpr int kJMaxSweeps = 40;
+constexpr float kJDead2 = 1e-12f;    // rows below 1e-6 of the largest norm are zero rows
+constexpr float kJCount2 = 1e-8f;    // rows below 1e-4 of the largest norm do not hold up convergence
+constexpr float kEigThr = 1e-6f;     // relative eigenvalue cut of G_A, G_B
+
+struct JacobiJob {
+  const float* X;   // k x r input (row stride r)
+  float* rows;      // k x r output: unit rows, sorted by descending norm (zero rows stay zero)
+  float* norms;     // k
+  int* status;      // AB_OK / AB_ERR_NOT_CONVERGED (may be null)
+  int k, r;
+};
+
+__device__ __forceinline__ void rr_pair2(int ne, int t, int idx, int& p, int& q) {
+  const int n1 = ne - 1;
+  if (idx == 0) { p = n1; q = t % n1; }
+  else { p = (t + idx) % n1; q = (t - idx + n1) % n1; }
+  if (p > q) { int tmp = p; p = q; q = tmp; }
+}
+
+__global__ void __launch_bounds__(kJThreads, 1)
+jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
+  extern __shared__ __align__(16) float sm[];
+  const JacobiJob job = jobs[blockIdx.x];
+  const int k = job.k, r = job.r, ld = r + 1;
+  float* X = sm;                       // k x ld
+  float* n2 = X + (size_t)k * ld;      // squared row norms, k
+  int* rank = reinterpret_cast<int*>(n2 + k);
+  __shared__ int rot_counted;
+  __shared__ float max_n2;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = kJThreads / 32;
+
+  for (int idx = tid; idx < k * r; idx += kJThreads) X[(idx / r) * ld + idx % r] = job.X[idx];
+  __syncthreads();
+
+  const int ke = k + (k & 1);
+  const int steps = ke > 2 ? ke - 1 : 1;
+  int sweeps = 0;
+  bool converged = (k < 2);
+  for (; sweeps < kJMaxSweeps && !converged; ++sweeps) {
+    // exact norms at the start of every sweep (the running updates drift)
+    if (tid == 0) { rot_counted = 0; max_n2 = 0.f; }
+    __syncthreads();
+    for (int i = warp; i < k; i += nwarps) {
+      float a = 0.f;
+      for (int t = lane; t < r; t += 32) { float v = X[i * ld + t]; a = fmaf(v, v, a); }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+      if (lane == 0) { n2[i] = a; atomicMax(reinterpret_cast<int*>(&max_n2), __float_as_int(a)); }
+    }
+    __syncthreads();
+    const float dead2 = kJDead2 * max_n2, count2 = kJCount2 * max_n2;
+    for (int st = 0; st < steps; ++st) {
+      for (int idx = warp; idx < ke / 2; idx += nwarps) {
+        int p, q;
+        rr_pair2(ke, st, idx, p, q);
+        if (q >= k) continue;
+        const float app = n2[p], aqq = n2[q];
+        if (!(app > dead2 && aqq > dead2 && app > 0.f && aqq > 0.f)) continue;
+        float g = 0.f;
+        for (int t = lane; t < r; t += 32) g = fmaf(X[p * ld + t], X[q * ld + t], g);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
+        if (!(fabsf(g) > tol * sqrtf(app) * sqrtf(aqq))) continue;
+        const float zeta = (aqq - app) / (2.f * g);
+        const float tt = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
+        const float c = 1.f / sqrtf(1.f + tt * tt), s = c * tt;
+        for (int t = lane; t < r; t += 32) {
+          const float xp = X[p * ld + t], xq = X[q * ld + t];
+          X[p * ld + t] = c * xp - s * xq;
+          X[q * ld + t] = s * xp + c * xq;
+        }
+        if (lane == 0) {
+          n2[p] = app - tt * g;
+          n2[q] = aqq + tt * g;
+          if (app > count2 && aqq > count2) rot_counted = 1;
+        }
+      }
+      __syncthreads();
+    }
+    converged = (rot_counted == 0);
+    __syncthreads();
+  }
+
+  // norms, descending order, unit rows
+  if (tid == 0) max_n2 = 0.f;
+  __syncthreads();
+  for (int i = warp; i < k; i += nwarps) {
+    float a = 0.f;
+    for (int t = lane; t < r; t += 32) { float v = X[i * ld + t]; a = fmaf(v, v, a); }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (lane == 0) { n2[i] = a; atomicMax(reinterpret_cast<int*>(&max_n2), __float_as_int(a)); }
+  }
+  __syncthreads();
+  for (int i = tid; i < k; i += kJThreads) {
+    const float li = n2[i];
+    int rk = 0;
+    for (int j = 0; j < k; ++j) { const float lj = n2[j]; rk += (lj > li) || (lj == li && j < i); }
+    rank[i] = rk;
+  }
+  __syncthreads();
+  const float dead2 = kJDead2 * max_n2;
+  for (int i = warp; i < k; i += nwarps) {
+    const float a = n2[i];
+    const bool live = a > dead2 && a > 0.f;
+    const float nrm = live ? sqrtf(a) : 0.f, inv = live ? 1.f / nrm : 0.f;
+    float* dst = job.rows + (size_t)rank[i] * r;
+    for (int t = lane; t < r; t += 32) dst[t] = X[i * ld + t] * inv;
+    if (lane == 0) job.norms[rank[i]] = nrm;
+  }
+  if (tid == 0 && job.status) *job.status = converged ? AB_OK : AB_ERR_NOT_CONVERGED;
+}
+
+size_t jacobi_smem_bytes(int k, int r) { return sizeof(float) * ((size_t)k * (r + 1) + k) + sizeof(int) * k + 64; }
+
+// r' = #{ i < r : sigma_i >= cutoff * sigma_0 } (at least 1); folds the three solver statuses.
+__global__ void fast_rank_rule_kernel(const float* const* __restrict__ sigma, const int* __restrict__ rs,
+                                      float cutoff, int* const* __restrict__ r_out,
+                                      const int* __restrict__ jstatus, int* __restrict__ dev_status, int L) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= L) return;
+  const float* sg = sigma[i];
+  const int r = rs[i];
+  float top = 0.f;
+  for (int k = 0; k < r; ++k) top = fmaxf(top, sg[k]);
+  int keep = 0;
+  for (int k = 0; k < r; ++k) keep += (sg[k] >= cutoff * top) ? 1 : 0;
+  if (keep < 1) keep = 1;
+  *r_out[i] = keep;
+  if (dev_status) {
+    int st = AB_OK;
+    for (int j = 0; j < 3; ++j) if (jstatus[3 * i + j] != AB_OK) st = jstatus[3 * i + j];
+    dev_status[i] = st;
+  }
+}
+
+struct FastWs {
+  std::vector<float*> Abar, Bbar, GA, GB, PA, PB, lamA, lamB, M, Vs, Y1, ZA, ZB;
+  GemmDesc* descs;      // 9 L
+  JacobiJob* jobs;      // 3 L
+  int* jstatus;         // 3 L
+  const float** sig_ptrs;
+  int** rout_ptrs;
+  int* rs;
+  size_t bytes;
+};
+
+FastWs fast_layout(const ab_sync_desc* d, int L, void* ws) {
+  FastWs w;
+  Arena ar(ws, 0);
+  auto each = [&](std::vector<float*>& v, auto count) {
+    v.resize(L);
+    for (int i = 0; i < L; ++i) v[i] = ar.take_n<float>(count(d[i]));
+  };
+  each(w.Abar, [](const ab_sync_desc& x) { return (size_t)x.m * x.r; });
+  each(w.Bbar, [](const ab_sync_desc& x) { return (size_t)x.r * x.n; });
+  auto rr = [](const ab_sync_desc& x) { return (size_t)x.r * x.r; };
+  auto r1 = [](const ab_sync_desc& x) { return (size_t)x.r; };
+  each(w.GA, rr); each(w.GB, rr); each(w.PA, rr); each(w.PB, rr); each(w.lamA, r1); each(w.lamB, r1);
+  each(w.M, rr); each(w.Vs, rr); each(w.Y1, rr); each(w.ZA, rr); each(w.ZB, rr);
+  w.descs = ar.take_n<GemmDesc>((size_t)9 * L);
+  w.jobs = ar.take_n<JacobiJob>((size_t)3 * L);
+  w.jstatus = ar.take_n<int>((size_t)3 * L);
+  w.sig_ptrs = ar.take_n<const float*>(L);
+  w.rout_ptrs = ar.take_n<int*>(L);
+  w.rs = ar.take_n<int>(L);
+  w.bytes = align_up(ar.used, 256);
+  return w;
+}
+
+GemmDesc mk(const float* A, int64_t sAm, int64_t sAk, const float* B, int64_t sBk, int64_t sBn, void* C, int64_t ldc,
+            int M, int N, int K) {
+  GemmDesc g;
+  g.A = A; g.B = B; g.C = C; g.sAm = sAm; g.sAk = sAk; g.sBk = sBk; g.sBn = sBn; g.ldc = ldc;
+  g.M = M; g.N = N; g.K = K; g.c_bf16 = 0;
+  g.row_vec = g.col_vec = g.k_vec = nullptr;
+  g.row_mode = g.col_mode = g.k_mode = 0;
+  g.thr = kEigThr;
+  g.live_rows = g.live_cols = nullptr;
+  return g;
+}
+
+}  // namespace
+
+bool sync_factored_supported(const ab_sync_desc* d, int L) {
+  for (int i = 0; i < L; ++i)
+    if (jacobi_smem_bytes(d[i].r, d[i].r) > 227 * 1024) return false;
+  return true;
+}
+
+size_t sync_factored_ws(const ab_sync_desc* d, int L) { return fast_layout(d, L, nullptr).bytes; }
+
+int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int dt, int* dev_status,
+                  void* ws, size_t ws_bytes, cudaStream_t st) {
+  FastWs w = fast_layout(d, L, ws);
+  if (w.bytes > ws_bytes) return AB_ERR_WORKSPACE;
+  const int out_bf16 = (dt == AB_BF16) ? 1 : 0;
+  int rmax = 0, mmax = 0, nmax = 0;
+  for (int i = 0; i < L; ++i) {
+    rmax = std::max(rmax, d[i].r); mmax = std::max(mmax, d[i].m); nmax = std::max(nmax, d[i].n);
+  }
+  // ---- host-built tables: 9 GEMM descriptors and 3 Jacobi jobs per matrix, copied in one go each
+  std::vector<GemmDesc> g((size_t)9 * L);
+  std::vector<JacobiJob> jb((size_t)3 * L);
+  std::vector<const float*> sigp(L);
+  std::vector<int*> routp(L);
+  std::vector<int> rs(L);
+  for (int i = 0; i < L; ++i) {
+    const int m = d[i].m, n = d[i].n, r = d[i].r;
+    float *Ab = w.Abar[i], *Bb = w.Bbar[i];
+    // batch 0 (2L): Gram matrices
+    g[0 * L + i] = mk(Ab, 1, r, Ab, r, 1, w.GA[i], r, r, r, m);           // G_A = Abar^T Abar
+    g[1 * L + i] = mk(Bb, n, 1, Bb, 1, n, w.GB[i], r, r, r, n);           // G_B = Bbar Bbar^T
+    // batch 1 (L): M = diag(sqrt lamA) PA PB^T diag(sqrt lamB)
+    GemmDesc& gm = g[2 * L + i];
+    gm = mk(w.PA[i], r, 1, w.PB[i], 1, r, w.M[i], r, r, r, r);
+    gm.row_vec = w.lamA[i]; gm.row_mode = 1; gm.col_vec = w.lamB[i]; gm.col_mode = 1;
+    // batch 2 (2L): Y1 = M Vs^T ;  Z_B = diag(sqrt sig) Vs diag(lamB^-1/2) PB
+    g[3 * L + i] = mk(w.M[i], r, 1, w.Vs[i], 1, r, w.Y1[i], r, r, r, r);
+    GemmDesc& gzb = g[4 * L + i];
+    gzb = mk(w.Vs[i], r, 1, w.PB[i], r, 1, w.ZB[i], r, r, r, r);
+    gzb.row_vec = d[i].sigma; gzb.row_mode = 1; gzb.k_vec = w.lamB[i]; gzb.k_mode = 2;
+    // batch 3 (L): Z_A = PA^T diag(lamA^-1/2) Y1 diag(sig^-1/2)
+    GemmDesc& gza = g[5 * L + i];
+    gza = mk(w.PA[i], 1, r, w.Y1[i], r, 1, w.ZA[i], r, r, r, r);
+    gza.k_vec = w.lamA[i]; gza.k_mode = 2; gza.col_vec = d[i].sigma; gza.col_mode = 2;
+    // batch 4 (L): A' = Abar Z_A (columns >= r' zero);  batch 5 (L): B' = Z_B Bbar (rows >= r' zero)
+    GemmDesc& ga = g[6 * L + i];
+    ga = mk(Ab, r, 1, w.ZA[i], r, 1, d[i].A_out, r, m, r, r);
+    ga.c_bf16 = out_bf16; ga.live_cols = d[i].r_out;
+    GemmDesc& gb = g[7 * L + i];
+    gb = mk(w.ZB[i], r, 1, Bb, n, 1, d[i].B_out, n, r, n, r);
+    gb.c_bf16 = out_bf16; gb.live_rows = d[i].r_out;
+    // batch 6 (L, optional): W = Abar Bbar
+    g[8 * L + i] = mk(Ab, r, 1, Bb, n, 1, d[i].W_out, n, d[i].W_out ? m : 0, d[i].W_out ? n : 0, r);
+    JacobiJob ja = {w.GA[i], w.PA[i], w.lamA[i], w.jstatus ? w.jstatus + 3 * i : nullptr, r, r};
+    JacobiJob jbb = {w.GB[i], w.PB[i], w.lamB[i], w.jstatus ? w.jstatus + 3 * i + 1 : nullptr, r, r};
+    JacobiJob jm = {w.M[i], w.Vs[i], d[i].sigma, w.jstatus ? w.jstatus + 3 * i + 2 : nullptr, r, r};
+    jb[i] = ja; jb[L + i] = jbb; jb[2 * L + i] = jm;
+    sigp[i] = d[i].sigma; routp[i] = d[i].r_out; rs[i] = r;
+  }
+  AB_CUDA_OK(cudaMemcpyAsync(w.descs, g.data(), g.size() * sizeof(GemmDesc), cudaMemcpyHostToDevice, st));
+  AB_CUDA_OK(cudaMemcpyAsync(w.jobs, jb.data(), jb.size() * sizeof(JacobiJob), cudaMemcpyHostToDevice, st));
+  AB_CUDA_OK(cudaMemcpyAsync(w.sig_ptrs, sigp.data(), L * sizeof(float*), cudaMemcpyHostToDevice, st));
+  AB_CUDA_OK(cudaMemcpyAsync(w.rout_ptrs, routp.data(), L * sizeof(int*), cudaMemcpyHostToDevice, st));
+  AB_CUDA_OK(cudaMemcpyAsync(w.rs, rs.data(), L * sizeof(int), cudaMemcpyHostToDevice, st));
+
+  // ---- a7: means of the K copies (fp32)
+  for (int i = 0; i < L; ++i) {
+    AB_TRY(group_average(d[i].A_copies, d[i].strideA, K, (int64_t)d[i].m * d[i].r, dt, AB_F32, w.Abar[i], st));
+    AB_TRY(group_average(d[i].B_copies, d[i].strideB, K, (int64_t)d[i].r * d[i].n, dt, AB_F32, w.Bbar[i], st));
+  }
+  const size_t smem = jacobi_smem_bytes(rmax, rmax);
+  AB_CUDA_OK(cudaFuncSetAttribute(jacobi_rows_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const float tol = 5e-7f * sqrtf((float)rmax) < 4e-6f ? 4e-6f : 5e-7f * sqrtf((float)rmax);
+  bool any_w = false;
+  for (int i = 0; i < L; ++i) any_w = any_w || d[i].W_out != nullptr;
+  if (any_w) AB_TRY(gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, st));                 // a8 (optional)
+  AB_TRY(gemm_simt_batched(w.descs, 2 * L, rmax, rmax, st));                                // Gram
+  jacobi_rows_smem_kernel<<<2 * L, kJThreads, smem, st>>>(w.jobs, tol);                     // eigen of G_A, G_B
+  AB_LAUNCH_OK();
+  AB_TRY(gemm_simt_batched(w.descs + 2 * L, L, rmax, rmax, st));                            // M
+  jacobi_rows_smem_kernel<<<L, kJThreads, smem, st>>>(w.jobs + 2 * L, tol);                 // SVD of M
+  AB_LAUNCH_OK();
+  fast_rank_rule_kernel<<<(L + 127) / 128, 128, 0, st>>>(w.sig_ptrs, w.rs, sigma_cutoff, w.rout_ptrs, w.jstatus,
+                                                         dev_status, L);
+  AB_LAUNCH_OK();
+  AB_TRY(gemm_simt_batched(w.descs + 3 * L, 2 * L, rmax, rmax, st));                        // Y1, Z_B
+  AB_TRY(gemm_simt_batched(w.descs + 5 * L, L, rmax, rmax, st));                            // Z_A
+  AB_TRY(gemm_simt_batched(w.descs + 6 * L, L, mmax, rmax, st));                            // A'
+  AB_TRY(gemm_simt_batched(w.descs + 7 * L, L, rmax, nmax, st));                            // B'
+  return AB_OK;
+}
+}  // namespace ab

@@ -72,7 +72,7 @@ def test_host_side_rejections(L):
     assert L.ab_svd_split(p, 4000, 4000, 2, 0.0, p, p, p, p, p, 0, 0, p, 1 << 20, None) == b.AB_ERR_UNSUPPORTED
     assert L.ab_svd_split(p, 4, 4, 2, 0.0, p, p, p, p, p, 0, 0, None, 0, None) == b.AB_ERR_WORKSPACE
     assert L.ab_svd_split(p, 4, 4, 2, 0.0, p, p, p, p, p, 0, 0, ctypes.c_void_p(264), 1 << 20, None) == b.AB_ERR_WORKSPACE
-    assert L.ab_group_sync(None, 1, 2, 0.1, 0, None, p, 1024, None) == bad
+    assert L.ab_group_sync(None, 1, 2, 0.1, 0, None, p, 1024, None, 0) == bad
 
 
 def test_no_device_means_an_error_not_a_fallback(L):

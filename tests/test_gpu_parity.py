@@ -294,14 +294,17 @@ def test_workload_linear_fp32_full(ab):
     check_split(ab, d["W"], d["r"], 0.0)          # the full-rank random W itself
 
 
-def test_workload_group_sync_scaled(ab):
-    """ViT-B/16 group sync recipe at 1/4 scale (six matrices of one block), K=8, cutoff 0.1."""
+@pytest.mark.parametrize("path", ["dense", "factored"])
+def test_workload_group_sync_scaled(ab, path):
+    """ViT-B/16 group sync recipe at 1/4 scale (six matrices of one block), K=8, cutoff 0.1, through the
+    dense route (W formed, dense split) and the factored route (r x r problems only)."""
     shapes = synth.VIT_BLOCK_SHAPES
     ds = [synth.vit_sync_matrix(3, i, m, n, K=8, scale=4) for i, (m, n) in enumerate(shapes)]
     Aks = [synth.group_copies(d["A"], d["noise_A"]) for d in ds]
     Bks = [synth.group_copies(d["B"], d["noise_B"]) for d in ds]
-    plan = ab.SyncPlan([dev(a) for a in Aks], [dev(b) for b in Bks], 0.1)
-    A_out, B_out, sigma, r_out, status = ab.ab_group_sync(plan)
+    plan = ab.SyncPlan([dev(a) for a in Aks], [dev(b) for b in Bks], 0.1, want_W=True)
+    A_out, B_out, sigma, r_out, status = ab.ab_group_sync(
+        plan, path=ab.AB_SYNC_DENSE if path == "dense" else ab.AB_SYNC_FACTORED)
     torch.cuda.synchronize()
     assert torch.count_nonzero(status) == 0
     for i, d in enumerate(ds):
@@ -317,6 +320,11 @@ def test_workload_group_sync_scaled(ab):
         Wr = (U[:, :r_gpu] * s2[:r_gpu]) @ Vt[:r_gpu]
         err = np.linalg.norm(host(A_out[i]) @ host(B_out[i]) - Wr) / np.linalg.norm(ref["W"])
         assert err <= 1e-4, (i, err)
+        assert orc.rel_frob(host(plan.W_out[i]), ref["W"]) <= 1e-6
+        Ah, Bh = host(A_out[i]), host(B_out[i])
+        assert np.count_nonzero(Ah[:, r_gpu:]) == 0 and np.count_nonzero(Bh[r_gpu:]) == 0
+        bal = np.linalg.norm(Ah[:, :r_gpu].T @ Ah[:, :r_gpu] - np.diag(sg[:r_gpu])) / s[0]
+        assert bal <= 1e-3, (i, bal)
 
 
 def test_workload_resnet_and_vgg_scaled(ab):
@@ -325,3 +333,30 @@ def test_workload_resnet_and_vgg_scaled(ab):
     for r in (8, 16, 32, 64):
         d = synth.vgg_conv(r, 4, N=512)
         check_chain(ab, d, True)
+
+
+def test_group_sync_factored_truncated_factors_and_bf16(ab):
+    """Factors whose trailing columns were zeroed by an earlier rank rule (exactly singular Gram
+    matrices) and bf16 storage, through the factored route."""
+    d = synth.vit_sync_matrix(5, 1, 256, 160, K=4, scale=1)
+    A0, B0 = d["A"].copy(), d["B"].copy()
+    A0[:, 30:] = 0.0
+    B0[30:] = 0.0
+    Ak = synth.group_copies(A0, [e * 0 for e in d["noise_A"]])
+    Bk = synth.group_copies(B0, [e * 0 for e in d["noise_B"]])
+    Ak[:, :, :30] += np.stack(d["noise_A"])[:, :, :30]
+    Bk[:, :30] += np.stack(d["noise_B"])[:, :30]
+    for bf16 in (False, True):
+        if bf16:
+            Ak, Bk = synth.bf16_round(Ak), synth.bf16_round(Bk)
+        plan = ab.SyncPlan([dev(Ak, bf16)], [dev(Bk, bf16)], 0.0)
+        A_out, B_out, sigma, r_out, status = ab.ab_group_sync(plan, path=ab.AB_SYNC_FACTORED)
+        torch.cuda.synchronize()
+        assert int(status[0].item()) == 0
+        W = orc.recombine(orc.group_average_f32(Ak), orc.group_average_f32(Bk))
+        s = np.linalg.svd(W, compute_uv=False)
+        sg = host(sigma[0])
+        assert np.all(np.abs(sg[:30] - s[:30]) <= 1e-4 * s[:30])
+        assert np.all(sg[30:] <= 1e-5 * s[0])
+        tol = 8e-3 if bf16 else 1e-4
+        assert np.linalg.norm(host(A_out[0]) @ host(B_out[0]) - W) / np.linalg.norm(W) <= tol
