@@ -12,6 +12,7 @@
 // are treated as zero (exactly right for factors truncated by the rank rule; otherwise the
 // factors need a condition number below about 300 -- all workloads here are far inside).
 #include <algorithm>
+#include <cstdio>
 #include <vector>
 
 #include "ab_common.cuh"
@@ -19,7 +20,8 @@
 namespace ab {
 namespace {
 
-constexpr int kJThreads = 512;
+constexpr int kJThreads = 1024;
+constexpr int kPW = 3;               // pairs a warp works on side by side
 constexpr int kJMaxSweeps = 40;
 constexpr float kJDead2 = 1e-12f;    // rows below 1e-6 of the largest norm are zero rows
 constexpr float kJCount2 = 1e-8f;    // rows below 1e-4 of the largest norm do not hold up convergence
@@ -34,9 +36,13 @@ struct JacobiJob {
 };
 
 __device__ __forceinline__ void rr_pair2(int ne, int t, int idx, int& p, int& q) {
+  // t < ne - 1 and idx < ne / 2: one conditional subtraction replaces each modulo
   const int n1 = ne - 1;
-  if (idx == 0) { p = n1; q = t % n1; }
-  else { p = (t + idx) % n1; q = (t - idx + n1) % n1; }
+  if (idx == 0) { p = n1; q = t; }
+  else {
+    p = t + idx; if (p >= n1) p -= n1;
+    q = t - idx + n1; if (q >= n1) q -= n1;
+  }
   if (p > q) { int tmp = p; p = q; q = tmp; }
 }
 
@@ -73,29 +79,65 @@ jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
     __syncthreads();
     const float dead2 = kJDead2 * max_n2, count2 = kJCount2 * max_n2;
     for (int st = 0; st < steps; ++st) {
-      for (int idx = warp; idx < ke / 2; idx += nwarps) {
-        int p, q;
-        rr_pair2(ke, st, idx, p, q);
-        if (q >= k) continue;
-        const float app = n2[p], aqq = n2[q];
-        if (!(app > dead2 && aqq > dead2 && app > 0.f && aqq > 0.f)) continue;
-        float g = 0.f;
-        for (int t = lane; t < r; t += 32) g = fmaf(X[p * ld + t], X[q * ld + t], g);
+      // a warp takes kPW pairs at a time and works on them side by side, so that the shuffle and
+      // square-root latencies of one pair hide behind the other pairs' work
+      for (int base = warp * kPW; base < ke / 2; base += nwarps * kPW) {
+        int p[kPW], q[kPW];
+        bool act[kPW];
+        float app[kPW], aqq[kPW], g[kPW];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
-        if (!(fabsf(g) > tol * sqrtf(app) * sqrtf(aqq))) continue;
-        const float zeta = (aqq - app) / (2.f * g);
-        const float tt = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
-        const float c = 1.f / sqrtf(1.f + tt * tt), s = c * tt;
+        for (int u = 0; u < kPW; ++u) {
+          p[u] = 0; q[u] = 0;
+          act[u] = base + u < ke / 2;
+          if (act[u]) { rr_pair2(ke, st, base + u, p[u], q[u]); act[u] = q[u] < k; }
+          app[u] = act[u] ? n2[p[u]] : 0.f;
+          aqq[u] = act[u] ? n2[q[u]] : 0.f;
+          act[u] = act[u] && app[u] > dead2 && aqq[u] > dead2 && app[u] > 0.f && aqq[u] > 0.f;
+          g[u] = 0.f;
+        }
         for (int t = lane; t < r; t += 32) {
-          const float xp = X[p * ld + t], xq = X[q * ld + t];
-          X[p * ld + t] = c * xp - s * xq;
-          X[q * ld + t] = s * xp + c * xq;
+#pragma unroll
+          for (int u = 0; u < kPW; ++u)
+            if (act[u]) g[u] = fmaf(X[p[u] * ld + t], X[q[u] * ld + t], g[u]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+          for (int u = 0; u < kPW; ++u) g[u] += __shfl_xor_sync(0xffffffffu, g[u], o);
+        }
+        // Rotation parameters with the approximate reciprocal / rsqrt units: every lane computes
+        // them, so IEEE divide and square-root sequences here would dominate the step.  A rotation
+        // that is orthogonal only to ~1e-7 merely rescales the two rows, and the rows are
+        // normalised at the end (no product of rotations is accumulated in this kernel).
+        float c[kPW], s[kPW], tt[kPW];
+#pragma unroll
+        for (int u = 0; u < kPW; ++u) {
+          act[u] = act[u] && g[u] * g[u] > tol * tol * app[u] * aqq[u];
+          const float gg = act[u] ? g[u] : 1.f;
+          float zeta = __fdividef(aqq[u] - app[u], 2.f * gg);
+          zeta = fminf(fmaxf(zeta, -1e15f), 1e15f);
+          const float h = fmaf(zeta, zeta, 1.f);
+          tt[u] = __fdividef(copysignf(1.f, zeta), fabsf(zeta) + h * rsqrtf(h));
+          c[u] = rsqrtf(fmaf(tt[u], tt[u], 1.f));
+          s[u] = c[u] * tt[u];
+        }
+        for (int t = lane; t < r; t += 32) {
+#pragma unroll
+          for (int u = 0; u < kPW; ++u)
+            if (act[u]) {
+              const float xp = X[p[u] * ld + t], xq = X[q[u] * ld + t];
+              X[p[u] * ld + t] = c[u] * xp - s[u] * xq;
+              X[q[u] * ld + t] = s[u] * xp + c[u] * xq;
+            }
         }
         if (lane == 0) {
-          n2[p] = app - tt * g;
-          n2[q] = aqq + tt * g;
-          if (app > count2 && aqq > count2) rot_counted = 1;
+#pragma unroll
+          for (int u = 0; u < kPW; ++u)
+            if (act[u]) {
+              n2[p[u]] = app[u] - tt[u] * g[u];
+              n2[q[u]] = aqq[u] + tt[u] * g[u];
+              if (app[u] > count2 && aqq[u] > count2) rot_counted = 1;
+            }
         }
       }
       __syncthreads();
@@ -132,6 +174,9 @@ jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
     if (lane == 0) job.norms[rank[i]] = nrm;
   }
   if (tid == 0 && job.status) *job.status = converged ? AB_OK : AB_ERR_NOT_CONVERGED;
+#ifdef AB_TRACE_SWEEPS
+  if (tid == 0) printf("jacobi job %d: k=%d r=%d sweeps=%d converged=%d\n", (int)blockIdx.x, k, r, sweeps, (int)converged);
+#endif
 }
 
 size_t jacobi_smem_bytes(int k, int r) { return sizeof(float) * ((size_t)k * (r + 1) + k) + sizeof(int) * k + 64; }
