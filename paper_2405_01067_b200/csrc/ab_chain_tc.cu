@@ -294,7 +294,7 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
 // grad kernel: partial[slice][p][j] = sum_{k in slice} act[k][p] * small[k][j]
 struct GradJob {
   int P;          // columns of act = rows of the output
-  int chunks;     // ceil(P / 128)
+  int chunks;     // ceil(P / 256)
   float* partial; // [slices][P][r]
 };
 struct GradParams {
@@ -338,7 +338,7 @@ grad_kernel(const __grid_constant__ CUtensorMap tmAct0, const __grid_constant__ 
     fence_barrier_init();
     tma_prefetch_desc(tmAct); tma_prefetch_desc(tmSmall);
   }
-  if (warp == 1) tmem_alloc(&bars->tmem_base, 256);
+  if (warp == 1) tmem_alloc(&bars->tmem_base, kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -351,15 +351,11 @@ grad_kernel(const __grid_constant__ CUtensorMap tmAct0, const __grid_constant__ 
         if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { raise_timeout(bars, p.status); break; }
         uint8_t* dst = ring + (size_t)slot * p.slot_bytes;
         const int k0 = k_begin + i * 64;
-        // rows at or beyond k_end inside the last slab belong to the next slice: the box is
-        // clipped by loading them and masking through a zero "small" operand is not possible,
-        // so slices are cut on 64-row boundaries (rows_per_slice % 64 == 0) and only the
-        // global end (k >= N) is ragged, where TMA fills zeros.
-        mbar_arrive_expect_tx(&bars->full[slot], (2 + p.natoms) * 8192);
-        tma_load_2d(dst, tmAct, &bars->full[slot], chunk * 128, k0);
-        tma_load_2d(dst + 8192, tmAct, &bars->full[slot], chunk * 128 + 64, k0);
+        // two 128-row accumulators share every slab of `small`: four 64-wide boxes of act, then small
+        mbar_arrive_expect_tx(&bars->full[slot], (4 + p.natoms) * 8192);
+        for (int a = 0; a < 4; ++a) tma_load_2d(dst + a * 8192, tmAct, &bars->full[slot], chunk * 256 + a * 64, k0);
         for (int a = 0; a < p.natoms; ++a)
-          tma_load_2d(dst + 16384 + a * 8192, tmSmall, &bars->full[slot], a * 64, k0);
+          tma_load_2d(dst + 32768 + a * 8192, tmSmall, &bars->full[slot], a * 64, k0);
       }
     }
   } else if (warp == 1) {
@@ -372,9 +368,9 @@ grad_kernel(const __grid_constant__ CUtensorMap tmAct0, const __grid_constant__ 
         tc_fence_after();
         const uint32_t sa = smem_u32(ring + (size_t)slot * p.slot_bytes);
         for (int kk = 0; kk < 4; ++kk) {
-          const uint64_t da = smem_desc_sw128(sa + kk * 2048, 8192);
-          const uint64_t db = smem_desc_sw128(sa + 16384 + kk * 2048, 8192);
-          tc_mma_bf16(tmem_base, da, db, idesc, (i | kk) != 0);
+          const uint64_t db = smem_desc_sw128(sa + 32768 + kk * 2048, 8192);
+          tc_mma_bf16(tmem_base, smem_desc_sw128(sa + kk * 2048, 8192), db, idesc, (i | kk) != 0);
+          tc_mma_bf16(tmem_base + 256, smem_desc_sw128(sa + 16384 + kk * 2048, 8192), db, idesc, (i | kk) != 0);
         }
         tc_commit(&bars->empty[slot]);
       }
@@ -385,25 +381,27 @@ grad_kernel(const __grid_constant__ CUtensorMap tmAct0, const __grid_constant__ 
     const int row = q * 32 + lane;
     const uint32_t lane_base = (uint32_t)(q * 32) << 16;
     const GradJob& job = p.job[jb];
-    const int prow = chunk * 128 + row;
-    float* out = job.partial + ((size_t)slice * job.P + prow) * p.r;
     bool ok = true;
     if (nk > 0) ok = epi_wait(bars, &bars->t_full, 0, p.status);
     if (ok) {
       tc_fence_after();
-      for (int c0 = 0; c0 < p.r; c0 += 16) {
-        float v[16];
-        if (nk > 0) tmem_ld16(tmem_base + lane_base + c0, v);
-        else {
+      for (int mt = 0; mt < 2; ++mt) {
+        const int prow = chunk * 256 + mt * 128 + row;
+        float* out = job.partial + ((size_t)slice * job.P + prow) * p.r;
+        for (int c0 = 0; c0 < p.r; c0 += 16) {
+          float v[16];
+          if (nk > 0) tmem_ld16(tmem_base + mt * 256 + lane_base + c0, v);
+          else {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) v[i] = 0.f;
-        }
-        if (prow < job.P) {
-          float4* o = reinterpret_cast<float4*>(out + c0);
-          o[0] = make_float4(v[0], v[1], v[2], v[3]);
-          o[1] = make_float4(v[4], v[5], v[6], v[7]);
-          o[2] = make_float4(v[8], v[9], v[10], v[11]);
-          o[3] = make_float4(v[12], v[13], v[14], v[15]);
+            for (int i = 0; i < 16; ++i) v[i] = 0.f;
+          }
+          if (prow < job.P) {
+            float4* o = reinterpret_cast<float4*>(out + c0);
+            o[0] = make_float4(v[0], v[1], v[2], v[3]);
+            o[1] = make_float4(v[4], v[5], v[6], v[7]);
+            o[2] = make_float4(v[8], v[9], v[10], v[11]);
+            o[3] = make_float4(v[12], v[13], v[14], v[15]);
+          }
         }
       }
     }
@@ -417,7 +415,7 @@ grad_kernel(const __grid_constant__ CUtensorMap tmAct0, const __grid_constant__ 
   }
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 256);
+    tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -517,12 +515,12 @@ struct GradPlan { int natoms, ns, slot_bytes, slices, rows_per_slice; size_t sme
 GradPlan grad_plan(int64_t N, int m, int n, int r) {
   GradPlan pl;
   pl.natoms = (r + 63) / 64;
-  pl.slot_bytes = 16384 + pl.natoms * 8192;
+  pl.slot_bytes = 32768 + pl.natoms * 8192;
   const int fixed = (int)sizeof(Bars) + 1024;
   pl.ns = (kSmemLimit - fixed) / pl.slot_bytes;
   if (pl.ns > kMaxStages) pl.ns = kMaxStages;
   pl.smem = (size_t)fixed + (size_t)pl.ns * pl.slot_bytes;
-  const int tiles = (m + 127) / 128 + (n + 127) / 128;
+  const int tiles = (m + 255) / 256 + (n + 255) / 256;
   int slices = 148 / tiles;
   if (slices < 1) slices = 1;
   const int64_t slabs = (N + 63) / 64;
@@ -643,13 +641,13 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
     if (dA) {
       AB_TRY(make_map(&tmAct[nj], dY, (uint64_t)N, m, m, 64, 64));
       AB_TRY(make_map(&tmSmall[nj], T, (uint64_t)N, r, r, 64, 64));
-      p.job[nj].P = m; p.job[nj].chunks = (m + 127) / 128; p.job[nj].partial = w.pA;
+      p.job[nj].P = m; p.job[nj].chunks = (m + 255) / 256; p.job[nj].partial = w.pA;
       ++nj;
     }
     if (dB) {
       AB_TRY(make_map(&tmAct[nj], x, (uint64_t)N, n, n, 64, 64));
       AB_TRY(make_map(&tmSmall[nj], w.dT, (uint64_t)N, r, r, 64, 64));
-      p.job[nj].P = n; p.job[nj].chunks = (n + 127) / 128; p.job[nj].partial = w.pB;
+      p.job[nj].P = n; p.job[nj].chunks = (n + 255) / 256; p.job[nj].partial = w.pB;
       ++nj;
     }
     if (nj == 1) { tmAct[1] = tmAct[0]; tmSmall[1] = tmSmall[0]; p.job[1] = p.job[0]; p.job[1].chunks = 0; }
