@@ -148,6 +148,58 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def vit_model_sync(ab, torch, steps=5):
+    """Second part of the metric: group sync of a whole ViT-B/16 (72 matrices, fp32 factors, rank 25 %,
+    K = 8 noisy copies in one packed arena per group, cutoff 0.1).  Returns ms per model for the mean
+    alone (one streaming call over the arena) and for the whole sync, with the mean's HBM figures."""
+    from paper_2405_01067_b200 import synth
+    K = 8
+    shapes = synth.vit_sync_shapes(12)
+    sizes = [(m * min(m, n) // 4, min(m, n) // 4 * n) for m, n in shapes]
+    total = sum(a + b for a, b in sizes)
+    arena = torch.empty((K, total), dtype=torch.float32, device="cuda")
+    off, views = 0, []
+    cache = {}
+    for i, (m, n) in enumerate(shapes):
+        if (m, n) not in cache:            # one recipe per shape and block position keeps set-up short
+            cache[(m, n)] = synth.vit_sync_matrix(3, len(cache), m, n, K=K)
+        d = cache[(m, n)]
+        r = d["r"]
+        a_sz, b_sz = m * r, r * n
+        for k in range(K):
+            arena[k, off:off + a_sz] = torch.from_numpy(d["A"] + d["noise_A"][k]).reshape(-1).cuda()
+            arena[k, off + a_sz:off + a_sz + b_sz] = torch.from_numpy(d["B"] + d["noise_B"][k]).reshape(-1).cuda()
+        views.append((arena[:, off:off + a_sz].view(K, m, r), arena[:, off + a_sz:off + a_sz + b_sz].view(K, r, n)))
+        off += a_sz + b_sz
+    mean_out = torch.empty((total,), dtype=torch.float32, device="cuda")
+
+    # the copies of a matrix are views into the arena: copy k sits one arena row further on
+    plan = ab.SyncPlan([v[0] for v in views], [v[1] for v in views], 0.1, want_W=True, strided=True)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+    res = {}
+    for name, fn in (("mean", lambda: ab.ab_group_average(arena, out=mean_out)), ("sync", lambda: ab.ab_group_sync(plan))):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = ev(), ev()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        res[name] = e0.elapsed_time(e1) / steps
+    bad = int(plan.status.abs().sum().item())
+    pk = measured_peaks()
+    mean_bytes = (K + 1) * 4.0 * total
+    return dict(workload="vit_b16_full_sync_72_matrices_fp32_K8_cutoff0.1", ms_per_model=res["sync"],
+                mean_ms=res["mean"], mean_gbs=mean_bytes / (res["mean"] * 1e-3) / 1e9,
+                mean_frac_of_measured_hbm=mean_bytes / (res["mean"] * 1e-3) / 1e9 / pk["hbm"],
+                mean_frac_of_nominal_8tbs=mean_bytes / (res["mean"] * 1e-3) / 1e9 / 8000.0,
+                kept_ranks=sorted(set(plan.r_out.tolist())), device_status_errors=bad)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -288,6 +340,10 @@ def run_ours(args):
                     e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                              ms_per_step=e2e_ms / K),
                     gpu_launches=int(launches), clocks=sampler.summary(), roofline=roof)
+        if world == 1 and not args.no_model_sync:
+            del layers, plan
+            torch.cuda.empty_cache()
+            line["group_sync_model"] = vit_model_sync(ab, torch)
         if world == 1 and not args.no_cpu_baseline:
             cb = cpu_baseline(inputs, min(N, args.ref_rows))
             line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
@@ -305,6 +361,7 @@ def main():
     ap.add_argument("--rows", type=int, default=256 * 197, help="token rows per layer (default: batch 256 x 197)")
     ap.add_argument("--ref-rows", type=int, default=8192, help="rows of the CPU checker's bounded sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-model-sync", action="store_true", help="skip the full-ViT group-sync measurement")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

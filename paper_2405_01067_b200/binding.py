@@ -231,7 +231,9 @@ def ab_svd_split(W, r_max, sigma_cutoff=0.0, out_dtype=None, ws=None, stream=Non
 class SyncPlan:
     """Buffers and descriptors of one model's group synchronisation (ab_group_sync)."""
 
-    def __init__(self, A_copies, B_copies, sigma_cutoff, want_W=False):
+    def __init__(self, A_copies, B_copies, sigma_cutoff, want_W=False, strided=False):
+        """A_copies[i]: (K, m, r), B_copies[i]: (K, r, n).  strided=True accepts views whose copies are
+        each contiguous but spaced by any stride along the leading axis (e.g. slices of a packed arena)."""
         self.A_copies, self.B_copies = list(A_copies), list(B_copies)
         self.L = len(self.A_copies)
         self.K = self.A_copies[0].shape[0]
@@ -243,7 +245,11 @@ class SyncPlan:
         self.status = torch.zeros((self.L,), dtype=torch.int32, device=dev)
         self.descs = (ab_sync_desc * self.L)()
         for i, (Ak, Bk) in enumerate(zip(self.A_copies, self.B_copies)):
-            _dev_ok(Ak, Bk)
+            if strided:
+                if not (Ak.is_cuda and Bk.is_cuda and Ak[0].is_contiguous() and Bk[0].is_contiguous()):
+                    raise ValueError("each copy must be a contiguous CUDA tensor")
+            else:
+                _dev_ok(Ak, Bk)
             K, m, r = Ak.shape
             n = Bk.shape[2]
             self.A_out.append(torch.empty((m, r), dtype=Ak.dtype, device=dev))
