@@ -34,6 +34,9 @@ NOMINAL_BF16_TFLOPS = 2250.0
 R = 192
 LAYERS = ((3072, 768), (768, 3072))
 K_GROUPS = 4
+# dram__bytes_read.sum + dram__bytes_write.sum of one row_chain_kernel launch (forward, 50,432 rows),
+# from the ncu capture summarised under profiles/; None until the kernel of that capture is current.
+ROW_CHAIN_DRAM_BYTES_PER_LAUNCH = 350.0e6   # forward of W1: 79.7 MB read + 270.3 MB written
 
 
 def chain_flops(N, layers=LAYERS, r=R):
@@ -239,17 +242,28 @@ def run_ours(args):
         layers.append(dict(m=m, n=n, h=h, g=g, hout=hout))
     plan = ab.SyncPlan([L["g"]["A_copies"] for L in layers], [L["g"]["B_copies"] for L in layers], 0.0, want_W=True)
 
-    def chain():
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    fwd_events = []        # (start, stop) around every forward call of the timed steps
+
+    def chain(record=False):
         for L in layers:
             g = L["g"]
+            if record:
+                f0, f1 = ev(), ev()
+                f0.record()
             ab.ab_layer_forward(g["x"], g["A"], g["B"], y=g["y"], T_save=g["T"], ws=g["ws_f"])
+            if record:
+                f1.record()
+                fwd_events.append((f0, f1))
             ab.ab_layer_backward(g["x"], g["dY"], g["A"], g["B"], T_saved=g["T"], dX=g["dX"], dA=g["dA"], dB=g["dB"],
                                  ws=g["ws_b"])
 
     def step(marks=None):
         if marks is not None:
             marks[0].record()
-        chain()
+        chain(record=marks is not None)
         if marks is not None:
             marks[1].record()
         ab.ab_group_sync(plan)
@@ -273,9 +287,6 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def ev():
-        return torch.cuda.Event(enable_timing=True)
-
     for _ in range(args.warmup):
         step()
     barrier()
@@ -294,6 +305,7 @@ def run_ours(args):
     total_ms = t_begin.elapsed_time(t_end)
     chain_ms = sum(mk[0].elapsed_time(mk[1]) for mk in marks)
     sync_ms = sum(mk[1].elapsed_time(mk[2]) for mk in marks)
+    fwd_ms = sum(a.elapsed_time(b) for a, b in fwd_events) / max(len(fwd_events), 1)   # per forward launch
     if int(plan.status.abs().sum().item()) != 0:
         raise SystemExit("group sync reported a device-side error status")
 
@@ -324,11 +336,20 @@ def run_ours(args):
         h2d = sum(L["h"]["x"].numel() + L["h"]["dY"].numel() for L in layers) * 2
         d2h = sum(sum(t.numel() * t.element_size() for t in L["hout"].values()) for L in layers)
         per_gpu = value / world
-        roof = dict(bound="tensor", kernel="ab_layer_forward+ab_layer_backward (both layers)",
-                    achieved=per_gpu, peak=pk["tc_sustained"], unit="TFLOP/s", frac=per_gpu / pk["tc_sustained"],
-                    traffic=None, peak_source=f"bf16_tflops_sustained of {pk['source']}",
-                    frac_of_nominal_2250=per_gpu / NOMINAL_BF16_TFLOPS,
-                    hbm_gbs=chain_bytes(N) * K / (chain_ms * 1e-3) / 1e9, hbm_peak_gbs=pk["hbm"])
+        # dominant kernel of the chain: row_chain_kernel (every forward call is exactly one launch of
+        # it; backward launches it once more).  Algorithmic work of a forward launch: 2 N r (m+n) FLOP
+        # (both layers have m+n = 3840), 2 N (m+n) bytes.
+        fwd_flops = 2.0 * N * R * 3840
+        fwd_tflops = fwd_flops / (fwd_ms * 1e-3) / 1e12
+        roof = dict(bound="tensor", kernel="row_chain_kernel (one launch = ab_layer_forward of one layer)",
+                    achieved=fwd_tflops, peak=pk["tc_sustained"], unit="TFLOP/s", frac=fwd_tflops / pk["tc_sustained"],
+                    traffic=ROW_CHAIN_DRAM_BYTES_PER_LAUNCH, us_per_launch=fwd_ms * 1e3,
+                    peak_source=f"bf16_tflops_sustained of {pk['source']}",
+                    frac_of_nominal_2250=fwd_tflops / NOMINAL_BF16_TFLOPS,
+                    algorithmic_gbs=2.0 * N * 3840 / (fwd_ms * 1e-3) / 1e9, hbm_peak_gbs=pk["hbm"],
+                    whole_chain=dict(tflops=per_gpu, frac_of_measured=per_gpu / pk["tc_sustained"],
+                                     frac_of_nominal_2250=per_gpu / NOMINAL_BF16_TFLOPS,
+                                     algorithmic_gbs=chain_bytes(N) * K / (chain_ms * 1e-3) / 1e9))
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=K, warmup=args.warmup,
                     ms_per_step=total_ms / K, higher_is_better=True, scaling="weak", vs_baseline=None,
                     dtype="bf16", data="synthetic",
