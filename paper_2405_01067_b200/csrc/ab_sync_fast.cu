@@ -20,8 +20,6 @@
 namespace ab {
 namespace {
 
-constexpr int kJThreads = 1024;
-constexpr int kPW = 3;               // pairs a warp works on side by side
 constexpr int kJMaxSweeps = 40;
 constexpr float kJDead2 = 1e-12f;    // rows below 1e-6 of the largest norm are zero rows
 constexpr float kJCount2 = 1e-8f;    // rows below 1e-4 of the largest norm do not hold up convergence
@@ -46,6 +44,7 @@ __device__ __forceinline__ void rr_pair2(int ne, int t, int idx, int& p, int& q)
   if (p > q) { int tmp = p; p = q; q = tmp; }
 }
 
+template <int kEL, int kJThreads>      // kEL elements per lane and row in registers: r <= 32 kEL
 __global__ void __launch_bounds__(kJThreads, 1)
 jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
   extern __shared__ __align__(16) float sm[];
@@ -61,8 +60,9 @@ jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
   for (int idx = tid; idx < k * r; idx += kJThreads) X[(idx / r) * ld + idx % r] = job.X[idx];
   __syncthreads();
 
-  const int ke = k + (k & 1);
-  const int steps = ke > 2 ? ke - 1 : 1;
+  const int nb = (k + 3) / 4;                  // blocks of 4 rows
+  const int nbe = nb + (nb & 1);
+  const int brounds = nbe > 2 ? nbe - 1 : 1;
   int sweeps = 0;
   bool converged = (k < 2);
   for (; sweeps < kJMaxSweeps && !converged; ++sweeps) {
@@ -78,67 +78,113 @@ jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
     }
     __syncthreads();
     const float dead2 = kJDead2 * max_n2, count2 = kJCount2 * max_n2;
-    for (int st = 0; st < steps; ++st) {
-      // a warp takes kPW pairs at a time and works on them side by side, so that the shuffle and
-      // square-root latencies of one pair hide behind the other pairs' work
-      for (int base = warp * kPW; base < ke / 2; base += nwarps * kPW) {
-        int p[kPW], q[kPW];
-        bool act[kPW];
-        float app[kPW], aqq[kPW], g[kPW];
+    // Rows are grouped in blocks of 4.  In each round a warp takes one pair of blocks, pulls its 8
+    // rows into registers (r/32 elements per lane and row), rotates the 16 cross pairs (4 steps of
+    // 4 disjoint pairs worked on side by side; in the first round of a sweep also the pairs inside
+    // each block) and writes the rows back: shared memory is touched once per 16 rotations
+    // instead of three times per rotation.
+    for (int round = 0; round < brounds; ++round) {
+      for (int task = warp; task < nbe / 2; task += nwarps) {
+        int bi, bj;
+        rr_pair2(nbe, round, task, bi, bj);
+        const bool has_j = bj < nb;
+        if (bi >= nb) continue;
+        if (!has_j && round != 0) continue;
+        float x[8][kEL];
+        float nn[8];
 #pragma unroll
-        for (int u = 0; u < kPW; ++u) {
-          p[u] = 0; q[u] = 0;
-          act[u] = base + u < ke / 2;
-          if (act[u]) { rr_pair2(ke, st, base + u, p[u], q[u]); act[u] = q[u] < k; }
-          app[u] = act[u] ? n2[p[u]] : 0.f;
-          aqq[u] = act[u] ? n2[q[u]] : 0.f;
-          act[u] = act[u] && app[u] > dead2 && aqq[u] > dead2 && app[u] > 0.f && aqq[u] > 0.f;
-          g[u] = 0.f;
+        for (int a = 0; a < 8; ++a) {
+          const int row = (a < 4 ? bi * 4 + a : bj * 4 + (a - 4));
+          const bool in = row < k && (a < 4 || has_j);
+          nn[a] = in ? n2[row] : 0.f;
+#pragma unroll
+          for (int e = 0; e < kEL; ++e) {
+            const int t = lane + 32 * e;
+            x[a][e] = (in && t < r) ? X[row * ld + t] : 0.f;
+          }
         }
-        for (int t = lane; t < r; t += 32) {
+        bool counted = false;
 #pragma unroll
-          for (int u = 0; u < kPW; ++u)
-            if (act[u]) g[u] = fmaf(X[p[u] * ld + t], X[q[u] * ld + t], g[u]);
+        for (int stp = 0; stp < 7; ++stp) {     // fully unrolled: every register index below is a constant
+          if (stp >= 4 && round != 0) break;
+          // pairs of this step: cross steps pair row a with row 4 + (a + stp) % 4; the three extra
+          // steps of round 0 are the rest of an 8-player tournament (pairs inside the blocks)
+          float g[4], c[4], sn[4], tt[4];
+          int pa[4], pb[4];
+          bool act[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            if (stp < 4) { pa[u] = u; pb[u] = 4 + ((u + stp) & 3); }
+            else if (stp == 4) { pa[u] = (u < 2) ? 0 + 2 * u : 4 + 2 * (u - 2); pb[u] = pa[u] + 1; }          // (0,1)(2,3)(4,5)(6,7)
+            else if (stp == 5) { pa[u] = (u < 2) ? u : 4 + (u - 2); pb[u] = pa[u] + 2; }                         // (0,2)(1,3)(4,6)(5,7)
+            else { pa[u] = (u < 2) ? u : 4 + (u - 2); pb[u] = (u < 2) ? 3 - u : 7 - (u - 2); }                  // (0,3)(1,2)(4,7)(5,6)
+            g[u] = 0.f;
+          }
+          // dot products (register indices are resolved by full unrolling over the 8 x 8 choices)
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+#pragma unroll
+            for (int a = 0; a < 8; ++a)
+#pragma unroll
+              for (int bb = 0; bb < 8; ++bb)
+                if (a == pa[u] && bb == pb[u]) {
+#pragma unroll
+                  for (int e = 0; e < kEL; ++e) g[u] = fmaf(x[a][e], x[bb][e], g[u]);
+                }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) g[u] += __shfl_xor_sync(0xffffffffu, g[u], o);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            float app = 0.f, aqq = 0.f;
+#pragma unroll
+            for (int a = 0; a < 8; ++a) { if (a == pa[u]) app = nn[a]; if (a == pb[u]) aqq = nn[a]; }
+            act[u] = app > dead2 && aqq > dead2 && app > 0.f && aqq > 0.f && g[u] * g[u] > tol * tol * app * aqq;
+            const float gg = act[u] ? g[u] : 1.f;
+            float zeta = __fdividef(aqq - app, 2.f * gg);
+            zeta = fminf(fmaxf(zeta, -1e15f), 1e15f);
+            const float h = fmaf(zeta, zeta, 1.f);
+            tt[u] = __fdividef(copysignf(1.f, zeta), fabsf(zeta) + h * rsqrtf(h));
+            c[u] = act[u] ? rsqrtf(fmaf(tt[u], tt[u], 1.f)) : 1.f;
+            sn[u] = act[u] ? c[u] * tt[u] : 0.f;
+            const float dn = act[u] ? tt[u] * g[u] : 0.f;
+            if (act[u] && app > count2 && aqq > count2) counted = true;
+#pragma unroll
+            for (int a = 0; a < 8; ++a) { if (a == pa[u]) nn[a] = app - dn; if (a == pb[u]) nn[a] = aqq + dn; }
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+#pragma unroll
+            for (int a = 0; a < 8; ++a)
+#pragma unroll
+              for (int bb = 0; bb < 8; ++bb)
+                if (a == pa[u] && bb == pb[u]) {
+#pragma unroll
+                  for (int e = 0; e < kEL; ++e) {
+                    const float xp = x[a][e], xq = x[bb][e];
+                    x[a][e] = c[u] * xp - sn[u] * xq;
+                    x[bb][e] = sn[u] * xp + c[u] * xq;
+                  }
+                }
+          }
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
+        for (int a = 0; a < 8; ++a) {
+          const int row = (a < 4 ? bi * 4 + a : bj * 4 + (a - 4));
+          const bool in = row < k && (a < 4 || has_j);
+          if (in) {
 #pragma unroll
-          for (int u = 0; u < kPW; ++u) g[u] += __shfl_xor_sync(0xffffffffu, g[u], o);
-        }
-        // Rotation parameters with the approximate reciprocal / rsqrt units: every lane computes
-        // them, so IEEE divide and square-root sequences here would dominate the step.  A rotation
-        // that is orthogonal only to ~1e-7 merely rescales the two rows, and the rows are
-        // normalised at the end (no product of rotations is accumulated in this kernel).
-        float c[kPW], s[kPW], tt[kPW];
-#pragma unroll
-        for (int u = 0; u < kPW; ++u) {
-          act[u] = act[u] && g[u] * g[u] > tol * tol * app[u] * aqq[u];
-          const float gg = act[u] ? g[u] : 1.f;
-          float zeta = __fdividef(aqq[u] - app[u], 2.f * gg);
-          zeta = fminf(fmaxf(zeta, -1e15f), 1e15f);
-          const float h = fmaf(zeta, zeta, 1.f);
-          tt[u] = __fdividef(copysignf(1.f, zeta), fabsf(zeta) + h * rsqrtf(h));
-          c[u] = rsqrtf(fmaf(tt[u], tt[u], 1.f));
-          s[u] = c[u] * tt[u];
-        }
-        for (int t = lane; t < r; t += 32) {
-#pragma unroll
-          for (int u = 0; u < kPW; ++u)
-            if (act[u]) {
-              const float xp = X[p[u] * ld + t], xq = X[q[u] * ld + t];
-              X[p[u] * ld + t] = c[u] * xp - s[u] * xq;
-              X[q[u] * ld + t] = s[u] * xp + c[u] * xq;
+            for (int e = 0; e < kEL; ++e) {
+              const int t = lane + 32 * e;
+              if (t < r) X[row * ld + t] = x[a][e];
             }
+            if (lane == 0) n2[row] = nn[a];
+          }
         }
-        if (lane == 0) {
-#pragma unroll
-          for (int u = 0; u < kPW; ++u)
-            if (act[u]) {
-              n2[p[u]] = app[u] - tt[u] * g[u];
-              n2[q[u]] = aqq[u] + tt[u] * g[u];
-              if (app[u] > count2 && aqq[u] > count2) rot_counted = 1;
-            }
-        }
+        if (lane == 0 && counted) rot_counted = 1;
       }
       __syncthreads();
     }
@@ -177,6 +223,20 @@ jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
 #ifdef AB_TRACE_SWEEPS
   if (tid == 0) printf("jacobi job %d: k=%d r=%d sweeps=%d converged=%d\n", (int)blockIdx.x, k, r, sweeps, (int)converged);
 #endif
+}
+
+template <int EL, int TH>
+int launch_jacobi_t(const JacobiJob* jobs, int count, size_t smem, float tol, cudaStream_t st) {
+  AB_CUDA_OK(cudaFuncSetAttribute(jacobi_rows_smem_kernel<EL, TH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  jacobi_rows_smem_kernel<EL, TH><<<count, TH, smem, st>>>(jobs, tol);
+  AB_LAUNCH_OK();
+  return AB_OK;
+}
+int launch_jacobi(const JacobiJob* jobs, int count, int rmax, size_t smem, float tol, cudaStream_t st) {
+  if (rmax <= 64) return launch_jacobi_t<2, 512>(jobs, count, smem, tol, st);
+  if (rmax <= 128) return launch_jacobi_t<4, 768>(jobs, count, smem, tol, st);
+  if (rmax <= 192) return launch_jacobi_t<6, 768>(jobs, count, smem, tol, st);
+  return launch_jacobi_t<8, 512>(jobs, count, smem, tol, st);
 }
 
 size_t jacobi_smem_bytes(int k, int r) { return sizeof(float) * ((size_t)k * (r + 1) + k) + sizeof(int) * k + 64; }
@@ -252,7 +312,7 @@ GemmDesc mk(const float* A, int64_t sAm, int64_t sAk, const float* B, int64_t sB
 
 bool sync_factored_supported(const ab_sync_desc* d, int L) {
   for (int i = 0; i < L; ++i)
-    if (jacobi_smem_bytes(d[i].r, d[i].r) > 227 * 1024) return false;
+    if (jacobi_smem_bytes(d[i].r, d[i].r) > 227 * 1024 || d[i].r > 256) return false;
   return true;
 }
 
@@ -319,17 +379,14 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
     AB_TRY(group_average(d[i].B_copies, d[i].strideB, K, (int64_t)d[i].r * d[i].n, dt, AB_F32, w.Bbar[i], st));
   }
   const size_t smem = jacobi_smem_bytes(rmax, rmax);
-  AB_CUDA_OK(cudaFuncSetAttribute(jacobi_rows_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const float tol = 5e-7f * sqrtf((float)rmax) < 4e-6f ? 4e-6f : 5e-7f * sqrtf((float)rmax);
   bool any_w = false;
   for (int i = 0; i < L; ++i) any_w = any_w || d[i].W_out != nullptr;
   if (any_w) AB_TRY(gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, st));                 // a8 (optional)
   AB_TRY(gemm_simt_batched(w.descs, 2 * L, rmax, rmax, st));                                // Gram
-  jacobi_rows_smem_kernel<<<2 * L, kJThreads, smem, st>>>(w.jobs, tol);                     // eigen of G_A, G_B
-  AB_LAUNCH_OK();
+  AB_TRY(launch_jacobi(w.jobs, 2 * L, rmax, smem, tol, st));                                // eigen of G_A, G_B
   AB_TRY(gemm_simt_batched(w.descs + 2 * L, L, rmax, rmax, st));                            // M
-  jacobi_rows_smem_kernel<<<L, kJThreads, smem, st>>>(w.jobs + 2 * L, tol);                 // SVD of M
-  AB_LAUNCH_OK();
+  AB_TRY(launch_jacobi(w.jobs + 2 * L, L, rmax, smem, tol, st));                            // SVD of M
   fast_rank_rule_kernel<<<(L + 127) / 128, 128, 0, st>>>(w.sig_ptrs, w.rs, sigma_cutoff, w.rout_ptrs, w.jstatus,
                                                          dev_status, L);
   AB_LAUNCH_OK();
