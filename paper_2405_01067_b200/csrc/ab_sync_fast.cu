@@ -109,9 +109,8 @@ jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
           if (stp >= 4 && round != 0) break;
           // pairs of this step: cross steps pair row a with row 4 + (a + stp) % 4; the three extra
           // steps of round 0 are the rest of an 8-player tournament (pairs inside the blocks)
-          float g[4], c[4], sn[4], tt[4];
+          float g[4], c[4], sn[4];
           int pa[4], pb[4];
-          bool act[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
             if (stp < 4) { pa[u] = u; pb[u] = 4 + ((u + stp) & 3); }
@@ -137,23 +136,40 @@ jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
 #pragma unroll
             for (int u = 0; u < 4; ++u) g[u] += __shfl_xor_sync(0xffffffffu, g[u], o);
           }
+          // rotation parameters: lane u (u < 4) works out pair u, then the results are broadcast --
+          // the parameter arithmetic would otherwise be repeated by all 32 lanes for all 4 pairs
+          float appv[4], aqqv[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
-            float app = 0.f, aqq = 0.f;
+            appv[u] = 0.f; aqqv[u] = 0.f;
 #pragma unroll
-            for (int a = 0; a < 8; ++a) { if (a == pa[u]) app = nn[a]; if (a == pb[u]) aqq = nn[a]; }
-            act[u] = app > dead2 && aqq > dead2 && app > 0.f && aqq > 0.f && g[u] * g[u] > tol * tol * app * aqq;
-            const float gg = act[u] ? g[u] : 1.f;
-            float zeta = __fdividef(aqq - app, 2.f * gg);
+            for (int a = 0; a < 8; ++a) { if (a == pa[u]) appv[u] = nn[a]; if (a == pb[u]) aqqv[u] = nn[a]; }
+          }
+          const int lu = lane & 3;
+          const float my_g = lu == 0 ? g[0] : lu == 1 ? g[1] : lu == 2 ? g[2] : g[3];
+          const float my_app = lu == 0 ? appv[0] : lu == 1 ? appv[1] : lu == 2 ? appv[2] : appv[3];
+          const float my_aqq = lu == 0 ? aqqv[0] : lu == 1 ? aqqv[1] : lu == 2 ? aqqv[2] : aqqv[3];
+          const bool my_act = my_app > dead2 && my_aqq > dead2 && my_app > 0.f && my_aqq > 0.f &&
+                              my_g * my_g > tol * tol * my_app * my_aqq;
+          float my_c = 1.f, my_s = 0.f, my_dn = 0.f;
+          if (my_act) {
+            float zeta = __fdividef(my_aqq - my_app, 2.f * my_g);
             zeta = fminf(fmaxf(zeta, -1e15f), 1e15f);
             const float h = fmaf(zeta, zeta, 1.f);
-            tt[u] = __fdividef(copysignf(1.f, zeta), fabsf(zeta) + h * rsqrtf(h));
-            c[u] = act[u] ? rsqrtf(fmaf(tt[u], tt[u], 1.f)) : 1.f;
-            sn[u] = act[u] ? c[u] * tt[u] : 0.f;
-            const float dn = act[u] ? tt[u] * g[u] : 0.f;
-            if (act[u] && app > count2 && aqq > count2) counted = true;
+            const float t1 = __fdividef(copysignf(1.f, zeta), fabsf(zeta) + h * rsqrtf(h));
+            my_c = rsqrtf(fmaf(t1, t1, 1.f));
+            my_s = my_c * t1;
+            my_dn = t1 * my_g;
+          }
+          const bool my_counted = my_act && my_app > count2 && my_aqq > count2;
+          if (__any_sync(0xffffffffu, my_counted)) counted = true;
 #pragma unroll
-            for (int a = 0; a < 8; ++a) { if (a == pa[u]) nn[a] = app - dn; if (a == pb[u]) nn[a] = aqq + dn; }
+          for (int u = 0; u < 4; ++u) {
+            c[u] = __shfl_sync(0xffffffffu, my_c, u);
+            sn[u] = __shfl_sync(0xffffffffu, my_s, u);
+            const float dn = __shfl_sync(0xffffffffu, my_dn, u);
+#pragma unroll
+            for (int a = 0; a < 8; ++a) { if (a == pa[u]) nn[a] = appv[u] - dn; if (a == pb[u]) nn[a] = aqqv[u] + dn; }
           }
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
@@ -234,7 +250,7 @@ int launch_jacobi_t(const JacobiJob* jobs, int count, size_t smem, float tol, cu
 }
 int launch_jacobi(const JacobiJob* jobs, int count, int rmax, size_t smem, float tol, cudaStream_t st) {
   if (rmax <= 64) return launch_jacobi_t<2, 512>(jobs, count, smem, tol, st);
-  if (rmax <= 128) return launch_jacobi_t<4, 768>(jobs, count, smem, tol, st);
+  if (rmax <= 128) return launch_jacobi_t<4, 512>(jobs, count, smem, tol, st);
   if (rmax <= 192) return launch_jacobi_t<6, 768>(jobs, count, smem, tol, st);
   return launch_jacobi_t<8, 512>(jobs, count, smem, tol, st);
 }
