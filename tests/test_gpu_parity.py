@@ -360,3 +360,117 @@ def test_group_sync_factored_truncated_factors_and_bf16(ab):
         assert np.all(sg[30:] <= 1e-5 * s[0])
         tol = 8e-3 if bf16 else 1e-4
         assert np.linalg.norm(host(A_out[0]) @ host(B_out[0]) - W) / np.linalg.norm(W) <= tol
+
+
+# ------------------------------------------------------------------ full-size workloads
+
+def _oracle_backward_chunked(x, dY, A, B, rows=8192):
+    """orc.forward/orc.backward over row chunks (their sums over rows add up), to bound host memory."""
+    m, r = A.shape
+    n = B.shape[1]
+    dA = np.zeros((m, r))
+    dB = np.zeros((r, n))
+    for s in range(0, x.shape[0], rows):
+        dXc, dAc, dBc, _ = orc.backward(x[s:s + rows], dY[s:s + rows], A, B)
+        dA += dAc
+        dB += dBc
+    return dA, dB
+
+
+def _full_size_chain(ab, d, sample=384):
+    """Chain at full size in the benchmark's launch configuration: dA, dB against the checker over all
+    rows; y, dX, T on a seeded sample of rows (each row of those outputs depends on its own row only)."""
+    x, dY, A, B = (dev(d[k], True) for k in ("x", "dY", "A", "B"))
+    N, n = x.shape
+    m, r = A.shape
+    ws_f = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_FORWARD, N, m, n, r, 1, ab.AB_BF16), "cuda")
+    ws_b = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_BACKWARD, N, m, n, r, 1, ab.AB_BF16), "cuda")
+    y, T = ab.ab_layer_forward(x, A, B, save_T=True, ws=ws_f)
+    dX, dA, dB = ab.ab_layer_backward(x, dY, A, B, T_saved=T, ws=ws_b)
+    torch.cuda.synchronize()
+    assert ab.workspace_status(ws_f) == 0 and ab.workspace_status(ws_b) == 0
+    rows = np.sort(np.random.default_rng(1).choice(N, size=min(sample, N), replace=False))
+    rows[-1] = N - 1                                   # always include the ragged tail
+    idx = torch.from_numpy(rows).cuda()
+    T_ref, y_ref = orc.forward(d["x"][rows], d["A"], d["B"])
+    dX_ref = orc.backward(d["x"][rows], d["dY"][rows], d["A"], d["B"])[0]
+    assert orc.rel_frob(host(y[idx]), y_ref) <= TOL_BF16
+    assert orc.rel_frob(host(T[idx]), T_ref) <= TOL_BF16
+    assert orc.rel_frob(host(dX[idx]), dX_ref) <= TOL_BF16
+    dA_ref, dB_ref = _oracle_backward_chunked(d["x"], d["dY"], d["A"], d["B"])
+    assert orc.rel_frob(host(dA), dA_ref) <= TOL_BF16
+    assert orc.rel_frob(host(dB), dB_ref) <= TOL_BF16
+    del x, dY, y, T, dX
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("layer", [1, 2])
+def test_full_size_vit_mlp(ab, layer):
+    """ViT-B/16 MLP layer at 50,432 rows, rank 192, bf16: the benchmark's workload."""
+    _full_size_chain(ab, synth.vit_mlp(layer, seed=1, N=256 * 197, K=1))
+
+
+def test_full_size_resnet_conv(ab):
+    """ResNet-50 layer3 3x3 convolution as GEMM, 25,088 im2col rows, rank 128, then the rank-truncation
+    split of the recombined W."""
+    d = synth.resnet_conv(2)
+    _full_size_chain(ab, d)
+    W = ab.ab_recombine(dev(d["A"]), dev(d["B"]))
+    torch.cuda.synchronize()
+    check_split(ab, W.cpu().numpy(), d["r"], 0.0)
+
+
+def test_full_size_vgg_conv_sweep(ab):
+    """VGG16 512 x 4608 layer, 16,384 rows, ranks 8..64 (the skinny, memory-bound regime), then the sync."""
+    for r in (8, 16, 32, 64):
+        d = synth.vgg_conv(r, 4)
+        _full_size_chain(ab, d, sample=128)
+        Ak = synth.group_copies(d["A"], d["noise_A"], bf16=True)
+        Bk = synth.group_copies(d["B"], d["noise_B"], bf16=True)
+        plan = ab.SyncPlan([dev(Ak, True)], [dev(Bk, True)], 0.0)
+        A_out, B_out, sigma, r_out, status = ab.ab_group_sync(plan)
+        torch.cuda.synchronize()
+        assert int(status[0].item()) == 0 and int(r_out[0].item()) == r
+        W = orc.recombine(orc.group_average_f32(Ak), orc.group_average_f32(Bk))
+        s = np.linalg.svd(W, compute_uv=False)      # LAPACK: the checker's own SVD is pinned to it on the CPU
+        assert np.all(np.abs(host(sigma[0]) - s[:r]) <= 1e-4 * s[:r])
+        assert np.linalg.norm(host(A_out[0]) @ host(B_out[0]) - W) / np.linalg.norm(W) <= 8e-3   # bf16 factors
+
+
+def test_full_size_vit_group_sync(ab):
+    """Whole ViT-B/16 group sync (72 matrices, K=8, cutoff 0.1) in the benchmark's configuration; three
+    matrices, one per shape, are checked: mean bit-exact, recombination, sigma and the truncated product
+    against LAPACK on the checker's W (too large for the checker's own Jacobi to finish in seconds)."""
+    K = 8
+    shapes = synth.vit_sync_shapes(12)
+    cache, Aks, Bks = {}, [], []
+    for (m, n) in shapes:
+        if (m, n) not in cache:
+            d = synth.vit_sync_matrix(3, len(cache), m, n, K=K)
+            cache[(m, n)] = (synth.group_copies(d["A"], d["noise_A"]), synth.group_copies(d["B"], d["noise_B"]), d["r"])
+        Aks.append(cache[(m, n)][0])
+        Bks.append(cache[(m, n)][1])
+    devA = {k: dev(v[0]) for k, v in cache.items()}
+    devB = {k: dev(v[1]) for k, v in cache.items()}
+    plan = ab.SyncPlan([devA[s] for s in shapes], [devB[s] for s in shapes], 0.1, want_W=True)
+    A_out, B_out, sigma, r_out, status = ab.ab_group_sync(plan)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(status) == 0
+    for i in (0, 4, 5):                       # 768x768, 3072x768, 768x3072
+        m, n = shapes[i]
+        r = cache[(m, n)][2]
+        Abar, Bbar = orc.group_average_f32(Aks[i]), orc.group_average_f32(Bks[i])
+        W = orc.recombine(Abar, Bbar)
+        assert orc.rel_frob(host(plan.W_out[i]), W) <= 1e-6
+        U, s, Vt = np.linalg.svd(W, full_matrices=False)
+        r_ref = orc.rank_rule(s, 0.1, r)
+        r_gpu = int(r_out[i].item())
+        near = np.any(np.abs(s[:r] - 0.1 * s[0]) <= 1e-3 * s[0])
+        assert abs(r_gpu - r_ref) <= (1 if near else 0), (i, r_gpu, r_ref)
+        kk = min(r_gpu, r_ref)
+        sg = host(sigma[i])
+        assert np.all(np.abs(sg[:kk] - s[:kk]) <= 1e-4 * s[:kk])
+        Wr = (U[:, :r_gpu] * s[:r_gpu]) @ Vt[:r_gpu]
+        assert np.linalg.norm(host(A_out[i]) @ host(B_out[i]) - Wr) / np.linalg.norm(W) <= 1e-4
+    # all blocks built from the same recipe must give the same bits (no cross-matrix interference)
+    assert torch.equal(A_out[0], A_out[6]) and torch.equal(B_out[4], B_out[10]) and torch.equal(sigma[5], sigma[11])
