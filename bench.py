@@ -92,7 +92,7 @@ def make_inputs(rank, N):
     from paper_2405_01067_b200 import synth
     out = []
     for li in (1, 2):
-        d = synth.vit_mlp(li, seed=1 + 100 * rank, N=N, K=K_GROUPS)
+        d = synth.vit_mlp(li, seed=rank_seed(rank), N=N, K=K_GROUPS)
         d["A_copies"] = synth.group_copies(d["A"], d["noise_A"], bf16=True)
         d["B_copies"] = synth.group_copies(d["B"], d["noise_B"], bf16=True)
         out.append(d)
@@ -149,6 +149,26 @@ def run_reference(args):
                 cpu_baseline=dict(value=v, unit=UNIT, cores=last["cores"], kind="oracle", sample=last["sample"]),
                 e2e=dict(value=v, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
     print(json.dumps(line))
+
+
+def rank_seed(rank):
+    """Every rank draws its own batch: the path shards by independent batches (weak scaling)."""
+    return 1 + 100 * rank
+
+
+def max_over_ranks(values, device, world):
+    """Slowest rank's times: element-wise MAX all-reduce (the only collective, outside the timed region)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_tflops(N, world, steps, chain_ms):
+    """Aggregate chain throughput of all ranks: every rank does chain_flops(N) per step."""
+    return chain_flops(N) * world * steps / (chain_ms * 1e-3) / 1e12
 
 
 def vit_model_sync(ab, torch, steps=5):
@@ -321,16 +341,13 @@ def run_ours(args):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    times = torch.tensor([total_ms, chain_ms, sync_ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, chain_ms, sync_ms, e2e_ms = [float(v) for v in times.tolist()]
+    total_ms, chain_ms, sync_ms, e2e_ms = max_over_ranks([total_ms, chain_ms, sync_ms, e2e_ms], "cuda", world)
     sampler.join(timeout=2.0)
     if rank == 0:
         pk = measured_peaks()
         K = args.steps
         flops_step = chain_flops(N) * world
-        value = flops_step * K / (chain_ms * 1e-3) / 1e12
+        value = whole_job_tflops(N, world, K, chain_ms)
         e2e_chain_share = e2e_ms - sync_ms   # same sync work; the rest is chain plus copies
         e2e_value = flops_step * K / (max(e2e_chain_share, 1e-6) * 1e-3) / 1e12
         h2d = sum(L["h"]["x"].numel() + L["h"]["dY"].numel() for L in layers) * 2
