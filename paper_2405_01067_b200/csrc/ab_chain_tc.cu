@@ -419,32 +419,65 @@ grad_kernel(const __grid_constant__ CUtensorMap tmAct0, const __grid_constant__ 
   }
 }
 
-// out[p][j] = sum_s partial[s][p][j]  (transpose_out: out[j][p])
-__global__ void reduce_partials_kernel(const float* __restrict__ partial, int slices, int P, int r,
-                                       float* __restrict__ out, int transpose_out) {
-  const int64_t total = (int64_t)P * r;
-  const int64_t step = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += step) {
-    int64_t pp, j;
-    if (transpose_out) { j = idx / P; pp = idx - j * P; } else { pp = idx / r; j = idx - pp * r; }
+// Sums the per-slice partials in ascending slice order (fixed order: identical bits every run).
+//   blocks [0, nA):  dA[p][j]  = sum_s pA[s][p][j]            (float4 per thread)
+//   blocks [nA, ..): dB[j][q]  = sum_s pB[s][q][j]            (32 x 32 tiles transposed through shared memory)
+__global__ void __launch_bounds__(256)
+reduce_partials_kernel(const float* __restrict__ pA, float* __restrict__ dA, int PA, int nA,
+                       const float* __restrict__ pB, float* __restrict__ dB, int PB, int slices, int r) {
+  if ((int)blockIdx.x < nA) {
+    const int64_t total4 = (int64_t)PA * r / 4;
+    const int64_t i4 = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (i4 >= total4) return;
+    const float4* src = reinterpret_cast<const float4*>(pA) + i4;
+    float4 acc = src[0];
+    for (int s = 1; s < slices; ++s) {
+      const float4 v = src[(int64_t)s * total4];
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    reinterpret_cast<float4*>(dA)[i4] = acc;
+    return;
+  }
+  __shared__ float tile[32][33];
+  const int t = blockIdx.x - nA;
+  const int tiles_j = (r + 31) / 32;
+  const int q0 = (t / tiles_j) * 32, j0 = (t % tiles_j) * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int i = ty; i < 32; i += 8) {
+    const int q = q0 + i, j = j0 + tx;
     float acc = 0.f;
-    for (int s = 0; s < slices; ++s) acc += partial[((int64_t)s * P + pp) * r + j];
-    out[idx] = acc;
+    if (q < PB && j < r)
+      for (int s = 0; s < slices; ++s) acc += pB[((int64_t)s * PB + q) * r + j];
+    tile[i][tx] = acc;
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int j = j0 + i, q = q0 + tx;
+    if (j < r && q < PB) dB[(int64_t)j * PB + q] = tile[tx][i];
   }
 }
 
-// dst[j][i] = src[i][j], bf16, src rows x cols with row stride ld
-__global__ void transpose_bf16_kernel(const bf16* __restrict__ src, int rows, int cols, int ld, bf16* __restrict__ dst) {
+// Both factor transposes of a backward call in one launch: At[j][i] = A[i][j] (A is m x r, row stride
+// ldA) for blocks [0, nA), Bt[j][i] = B[i][j] (B is r x n, row stride ldB) after that.
+__global__ void transpose_factors_kernel(const bf16* __restrict__ A, int m, int r, int ldA, bf16* __restrict__ At, int nA,
+                                         const bf16* __restrict__ B, int n, int ldB, bf16* __restrict__ Bt) {
   __shared__ bf16 tile[32][33];
-  const int bx = blockIdx.x * 32, by = blockIdx.y * 32;
-  for (int i = threadIdx.y; i < 32; i += 8) {
-    int rr = by + i, cc = bx + threadIdx.x;
-    tile[i][threadIdx.x] = (rr < rows && cc < cols) ? src[(size_t)rr * ld + cc] : __float2bfloat16(0.f);
+  const bool first = (int)blockIdx.x < nA;
+  const bf16* src = first ? A : B;
+  bf16* dst = first ? At : Bt;
+  const int rows = first ? m : r, cols = first ? r : n, ld = first ? ldA : ldB;
+  const int t = first ? blockIdx.x : blockIdx.x - nA;
+  const int tiles_c = (cols + 31) / 32;
+  const int by = (t / tiles_c) * 32, bx = (t % tiles_c) * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int i = ty; i < 32; i += 8) {
+    const int rr = by + i, cc = bx + tx;
+    tile[i][tx] = (rr < rows && cc < cols) ? src[(size_t)rr * ld + cc] : __float2bfloat16(0.f);
   }
   __syncthreads();
-  for (int i = threadIdx.y; i < 32; i += 8) {
-    int cc = bx + i, rr = by + threadIdx.x;
-    if (cc < cols && rr < rows) dst[(size_t)cc * rows + rr] = tile[threadIdx.x][i];
+  for (int i = ty; i < 32; i += 8) {
+    const int cc = bx + i, rr = by + tx;
+    if (cc < cols && rr < rows) dst[(size_t)cc * rows + rr] = tile[tx][i];
   }
 }
 
@@ -623,11 +656,11 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
     T = w.T;
   }
   if (dX || dB) {
-    dim3 tb(32, 8);
-    transpose_bf16_kernel<<<dim3((r + 31) / 32, (m + 31) / 32), tb, 0, st>>>(static_cast<const bf16*>(A), m, r, ldA, w.At);
-    AB_LAUNCH_OK();
-    if (dX) {
-      transpose_bf16_kernel<<<dim3((n + 31) / 32, (r + 31) / 32), tb, 0, st>>>(static_cast<const bf16*>(B), r, n, ldB, w.Bt);
+    {
+      const int nA = ((m + 31) / 32) * ((r + 31) / 32);
+      const int nB = dX ? ((r + 31) / 32) * ((n + 31) / 32) : 0;
+      transpose_factors_kernel<<<nA + nB, 256, 0, st>>>(static_cast<const bf16*>(A), m, r, ldA, w.At, nA,
+                                                        static_cast<const bf16*>(B), n, ldB, w.Bt);
       AB_LAUNCH_OK();
     }
     // dT = dY A (kept for dB), dX = dT B
@@ -657,12 +690,10 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
     const unsigned grid = (unsigned)((p.job[0].chunks + p.job[1].chunks) * gp.slices);
     grad_kernel<<<grid, 192, gp.smem, st>>>(tmAct[0], tmSmall[0], tmAct[1], tmSmall[1], p);
     AB_LAUNCH_OK();
-    if (dA) {
-      reduce_partials_kernel<<<148 * 4, 256, 0, st>>>(w.pA, gp.slices, m, r, dA, 0);
-      AB_LAUNCH_OK();
-    }
-    if (dB) {
-      reduce_partials_kernel<<<148 * 4, 256, 0, st>>>(w.pB, gp.slices, n, r, dB, 1);
+    {
+      const int nA = dA ? (int)(((int64_t)m * r / 4 + 255) / 256) : 0;
+      const int nB = dB ? ((n + 31) / 32) * ((r + 31) / 32) : 0;
+      reduce_partials_kernel<<<nA + nB, 256, 0, st>>>(w.pA, dA, m, nA, w.pB, dB, n, gp.slices, r);
       AB_LAUNCH_OK();
     }
   }
