@@ -1,16 +1,17 @@
 // Factored group synchronisation: the split of W = Abar Bbar (Algorithm 1, the decomposition that
 // follows the all-reduces and "W <- AB") without ever forming the m x n matrix.  W has rank <= r,
 // so everything reduces to r x r problems:
-//   G_A = Abar^T Abar = P_A L_A P_A^T,   G_B = Bbar Bbar^T = P_B L_B P_B^T      (eigen, r x r)
-//   Abar = U_A C_A, C_A = L_A^(1/2) P_A^T;   Bbar^T = U_B C_B, C_B = L_B^(1/2) P_B^T
-//   W = U_A M U_B^T,  M = C_A C_B^T  (r x r),   M = U_M S V_M^T                 (SVD, r x r)
-//   A' = Abar Z_A,  Z_A = P_A L_A^(-1/2) (M V_M) S^(-1/2);   B' = Z_B Bbar,  Z_B = S^(1/2) V_M^T L_B^(-1/2) P_B^T
-// Each r x r problem is solved by one CTA that keeps the matrix in shared memory and
-// orthogonalises its ROWS with one-sided Jacobi rotations (for a symmetric G the rows of the
-// result are lambda_i p_i^T; for M they are sigma_i v_i^T), so no kernel boundary and no
-// global traffic sits between rotations.  Eigenvalues of G_A / G_B below 1e-6 of the largest
-// are treated as zero (exactly right for factors truncated by the rank rule; otherwise the
-// factors need a condition number below about 300 -- all workloads here are far inside).
+//   G_A = Abar^T Abar = R_A^T R_A,   G_B = Bbar Bbar^T = R_B^T R_B      (Cholesky, r x r, upper R)
+//   Abar = Q_A R_A,  Bbar^T = Q_B R_B   with Q_A = Abar R_A^-1, Q_B = Bbar^T R_B^-1 orthonormal
+//   W = Q_A M Q_B^T,  M = R_A R_B^T  (r x r),   M = U_M S V_M^T         (SVD, r x r)
+//   A' = Abar Z_A,  Z_A = R_A^-1 (M V_M) S^(-1/2);   B' = Z_B Bbar,  Z_B = S^(1/2) V_M^T R_B^-T
+// One CTA per Gram matrix factors it in shared memory and inverts the triangle in place; one CTA
+// per M keeps it in shared memory and orthogonalises its ROWS with one-sided Jacobi rotations
+// (the rows of the result are sigma_i v_i^T), so no kernel boundary and no global traffic sits
+// between rotations.  Cholesky pivots below 1e-6 of the largest diagonal entry of G are treated
+// as zero: the row of R and the row and column of its inverse are dropped, which is exactly right
+// for factors truncated by the rank rule (zero columns of A, zero rows of B).  Otherwise the
+// factors need a condition number below about 300 -- all workloads here are far inside.
 #include <algorithm>
 #include <cstdio>
 #include <vector>
@@ -23,7 +24,8 @@ namespace {
 constexpr int kJMaxSweeps = 40;
 constexpr float kJDead2 = 1e-12f;    // rows below 1e-6 of the largest norm are zero rows
 constexpr float kJCount2 = 1e-8f;    // rows below 1e-4 of the largest norm do not hold up convergence
-constexpr float kEigThr = 1e-6f;     // relative eigenvalue cut of G_A, G_B
+constexpr float kEigThr = 1e-6f;     // relative pivot cut of G_A, G_B (and of sigma in the scalings)
+constexpr int kCThreads = 512;
 
 struct JacobiJob {
   const float* X;   // k x r input (row stride r)
@@ -241,6 +243,72 @@ jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
 #endif
 }
 
+struct CholJob {
+  const float* G;   // r x r symmetric positive semi-definite (row stride r)
+  float* R;         // r x r upper triangular, G = R^T R; zeros below the diagonal, dropped rows zero
+  float* Rinv;      // r x r upper triangular inverse of the kept part; dropped rows and columns zero
+  int* status;      // receives AB_OK (may be null)
+  int r;
+};
+
+// Right-looking Cholesky of one Gram matrix in shared memory, then the inverse of the triangle by
+// back substitution, one warp per column.  R lives in the upper triangle; column j of the inverse
+// is parked in the strict lower triangle of row j (contiguous), its diagonal in dinv[].
+__global__ void __launch_bounds__(kCThreads, 1) chol_inv_kernel(const CholJob* __restrict__ jobs) {
+  extern __shared__ __align__(16) float sm[];
+  const CholJob job = jobs[blockIdx.x];
+  const int r = job.r, ld = r + 1;
+  float* S = sm;                       // r x ld
+  float* dinv = S + (size_t)r * ld;    // r
+  __shared__ float maxdiag;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = kCThreads / 32;
+
+  if (tid == 0) maxdiag = 0.f;
+  for (int idx = tid; idx < r * r; idx += kCThreads) S[(idx / r) * ld + idx % r] = job.G[idx];
+  __syncthreads();
+  for (int i = tid; i < r; i += kCThreads)
+    atomicMax(reinterpret_cast<int*>(&maxdiag), __float_as_int(fmaxf(S[i * ld + i], 0.f)));
+  __syncthreads();
+  const float cut = kEigThr * maxdiag;
+
+  for (int j = 0; j < r; ++j) {
+    const float dj = S[j * ld + j];
+    const bool live = dj > cut && dj > 0.f;
+    const float inv = live ? 1.f / sqrtf(dj) : 0.f;
+    for (int k = j + 1 + tid; k < r; k += kCThreads) S[j * ld + k] *= inv;     // a dropped row becomes zero
+    __syncthreads();
+    if (tid == 0) { S[j * ld + j] = dj * inv; dinv[j] = inv; }                  // nobody reads the pivot below
+    for (int i = j + 1 + warp; i < r; i += nwarps) {
+      const float f = S[j * ld + i];
+      if (f != 0.f)
+        for (int k = i + lane; k < r; k += 32) S[i * ld + k] = fmaf(-f, S[j * ld + k], S[i * ld + k]);
+    }
+    __syncthreads();
+  }
+
+  // X = R^-1 restricted to the kept rows: X_jj = 1/R_jj, X_ij = -(sum_{i<k<=j} R_ik X_kj) / R_ii
+  for (int j = warp; j < r; j += nwarps) {
+    const float xjj = dinv[j];
+    for (int i = j - 1; i >= 0; --i) {
+      float acc = 0.f;
+      for (int k = i + 1 + lane; k < j; k += 32) acc = fmaf(S[i * ld + k], S[j * ld + k], acc);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (lane == 0) S[j * ld + i] = -dinv[i] * fmaf(S[i * ld + j], xjj, acc);
+      __syncwarp();
+    }
+  }
+  __syncthreads();
+  for (int idx = tid; idx < r * r; idx += kCThreads) {
+    const int i = idx / r, k = idx % r;
+    job.R[idx] = (k >= i) ? S[i * ld + k] : 0.f;
+    job.Rinv[idx] = (k > i) ? S[k * ld + i] : (k == i ? dinv[i] : 0.f);
+  }
+  if (tid == 0 && job.status) *job.status = AB_OK;
+}
+
+size_t chol_smem_bytes(int r) { return sizeof(float) * ((size_t)r * (r + 1) + r) + 64; }
+
 template <int EL, int TH>
 int launch_jacobi_t(const JacobiJob* jobs, int count, size_t smem, float tol, cudaStream_t st) {
   AB_CUDA_OK(cudaFuncSetAttribute(jacobi_rows_smem_kernel<EL, TH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -279,9 +347,10 @@ __global__ void fast_rank_rule_kernel(const float* const* __restrict__ sigma, co
 }
 
 struct FastWs {
-  std::vector<float*> Abar, Bbar, GA, GB, PA, PB, lamA, lamB, M, Vs, Y1, ZA, ZB;
+  std::vector<float*> Abar, Bbar, GA, GB, RA, RB, IA, IB, M, Vs, Y1, ZA, ZB;
   GemmDesc* descs;      // 9 L
-  JacobiJob* jobs;      // 3 L
+  CholJob* cjobs;       // 2 L
+  JacobiJob* jobs;      // L
   int* jstatus;         // 3 L
   const float** sig_ptrs;
   int** rout_ptrs;
@@ -299,11 +368,11 @@ FastWs fast_layout(const ab_sync_desc* d, int L, void* ws) {
   each(w.Abar, [](const ab_sync_desc& x) { return (size_t)x.m * x.r; });
   each(w.Bbar, [](const ab_sync_desc& x) { return (size_t)x.r * x.n; });
   auto rr = [](const ab_sync_desc& x) { return (size_t)x.r * x.r; };
-  auto r1 = [](const ab_sync_desc& x) { return (size_t)x.r; };
-  each(w.GA, rr); each(w.GB, rr); each(w.PA, rr); each(w.PB, rr); each(w.lamA, r1); each(w.lamB, r1);
+  each(w.GA, rr); each(w.GB, rr); each(w.RA, rr); each(w.RB, rr); each(w.IA, rr); each(w.IB, rr);
   each(w.M, rr); each(w.Vs, rr); each(w.Y1, rr); each(w.ZA, rr); each(w.ZB, rr);
   w.descs = ar.take_n<GemmDesc>((size_t)9 * L);
-  w.jobs = ar.take_n<JacobiJob>((size_t)3 * L);
+  w.cjobs = ar.take_n<CholJob>((size_t)2 * L);
+  w.jobs = ar.take_n<JacobiJob>((size_t)L);
   w.jstatus = ar.take_n<int>((size_t)3 * L);
   w.sig_ptrs = ar.take_n<const float*>(L);
   w.rout_ptrs = ar.take_n<int*>(L);
@@ -343,9 +412,10 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   for (int i = 0; i < L; ++i) {
     rmax = std::max(rmax, d[i].r); mmax = std::max(mmax, d[i].m); nmax = std::max(nmax, d[i].n);
   }
-  // ---- host-built tables: 9 GEMM descriptors and 3 Jacobi jobs per matrix, copied in one go each
+  // ---- host-built tables: 9 GEMM descriptors, 2 Cholesky jobs and 1 Jacobi job per matrix, copied in one go each
   std::vector<GemmDesc> g((size_t)9 * L);
-  std::vector<JacobiJob> jb((size_t)3 * L);
+  std::vector<CholJob> cj((size_t)2 * L);
+  std::vector<JacobiJob> jb((size_t)L);
   std::vector<const float*> sigp(L);
   std::vector<int*> routp(L);
   std::vector<int> rs(L);
@@ -355,19 +425,17 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
     // batch 0 (2L): Gram matrices
     g[0 * L + i] = mk(Ab, 1, r, Ab, r, 1, w.GA[i], r, r, r, m);           // G_A = Abar^T Abar
     g[1 * L + i] = mk(Bb, n, 1, Bb, 1, n, w.GB[i], r, r, r, n);           // G_B = Bbar Bbar^T
-    // batch 1 (L): M = diag(sqrt lamA) PA PB^T diag(sqrt lamB)
-    GemmDesc& gm = g[2 * L + i];
-    gm = mk(w.PA[i], r, 1, w.PB[i], 1, r, w.M[i], r, r, r, r);
-    gm.row_vec = w.lamA[i]; gm.row_mode = 1; gm.col_vec = w.lamB[i]; gm.col_mode = 1;
-    // batch 2 (2L): Y1 = M Vs^T ;  Z_B = diag(sqrt sig) Vs diag(lamB^-1/2) PB
+    // batch 1 (L): M = R_A R_B^T
+    g[2 * L + i] = mk(w.RA[i], r, 1, w.RB[i], 1, r, w.M[i], r, r, r, r);
+    // batch 2 (2L): Y1 = M Vs^T ;  Z_B = diag(sqrt sig) Vs R_B^-T
     g[3 * L + i] = mk(w.M[i], r, 1, w.Vs[i], 1, r, w.Y1[i], r, r, r, r);
     GemmDesc& gzb = g[4 * L + i];
-    gzb = mk(w.Vs[i], r, 1, w.PB[i], r, 1, w.ZB[i], r, r, r, r);
-    gzb.row_vec = d[i].sigma; gzb.row_mode = 1; gzb.k_vec = w.lamB[i]; gzb.k_mode = 2;
-    // batch 3 (L): Z_A = PA^T diag(lamA^-1/2) Y1 diag(sig^-1/2)
+    gzb = mk(w.Vs[i], r, 1, w.IB[i], 1, r, w.ZB[i], r, r, r, r);
+    gzb.row_vec = d[i].sigma; gzb.row_mode = 1;
+    // batch 3 (L): Z_A = R_A^-1 Y1 diag(sig^-1/2)
     GemmDesc& gza = g[5 * L + i];
-    gza = mk(w.PA[i], 1, r, w.Y1[i], r, 1, w.ZA[i], r, r, r, r);
-    gza.k_vec = w.lamA[i]; gza.k_mode = 2; gza.col_vec = d[i].sigma; gza.col_mode = 2;
+    gza = mk(w.IA[i], r, 1, w.Y1[i], r, 1, w.ZA[i], r, r, r, r);
+    gza.col_vec = d[i].sigma; gza.col_mode = 2;
     // batch 4 (L): A' = Abar Z_A (columns >= r' zero);  batch 5 (L): B' = Z_B Bbar (rows >= r' zero)
     GemmDesc& ga = g[6 * L + i];
     ga = mk(Ab, r, 1, w.ZA[i], r, 1, d[i].A_out, r, m, r, r);
@@ -377,13 +445,13 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
     gb.c_bf16 = out_bf16; gb.live_rows = d[i].r_out;
     // batch 6 (L, optional): W = Abar Bbar
     g[8 * L + i] = mk(Ab, r, 1, Bb, n, 1, d[i].W_out, n, d[i].W_out ? m : 0, d[i].W_out ? n : 0, r);
-    JacobiJob ja = {w.GA[i], w.PA[i], w.lamA[i], w.jstatus ? w.jstatus + 3 * i : nullptr, r, r};
-    JacobiJob jbb = {w.GB[i], w.PB[i], w.lamB[i], w.jstatus ? w.jstatus + 3 * i + 1 : nullptr, r, r};
-    JacobiJob jm = {w.M[i], w.Vs[i], d[i].sigma, w.jstatus ? w.jstatus + 3 * i + 2 : nullptr, r, r};
-    jb[i] = ja; jb[L + i] = jbb; jb[2 * L + i] = jm;
+    cj[i] = CholJob{w.GA[i], w.RA[i], w.IA[i], w.jstatus + 3 * i, r};
+    cj[L + i] = CholJob{w.GB[i], w.RB[i], w.IB[i], w.jstatus + 3 * i + 1, r};
+    jb[i] = JacobiJob{w.M[i], w.Vs[i], d[i].sigma, w.jstatus + 3 * i + 2, r, r};
     sigp[i] = d[i].sigma; routp[i] = d[i].r_out; rs[i] = r;
   }
   AB_CUDA_OK(cudaMemcpyAsync(w.descs, g.data(), g.size() * sizeof(GemmDesc), cudaMemcpyHostToDevice, st));
+  AB_CUDA_OK(cudaMemcpyAsync(w.cjobs, cj.data(), cj.size() * sizeof(CholJob), cudaMemcpyHostToDevice, st));
   AB_CUDA_OK(cudaMemcpyAsync(w.jobs, jb.data(), jb.size() * sizeof(JacobiJob), cudaMemcpyHostToDevice, st));
   AB_CUDA_OK(cudaMemcpyAsync(w.sig_ptrs, sigp.data(), L * sizeof(float*), cudaMemcpyHostToDevice, st));
   AB_CUDA_OK(cudaMemcpyAsync(w.rout_ptrs, routp.data(), L * sizeof(int*), cudaMemcpyHostToDevice, st));
@@ -400,9 +468,12 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   for (int i = 0; i < L; ++i) any_w = any_w || d[i].W_out != nullptr;
   if (any_w) AB_TRY(gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, st));                 // a8 (optional)
   AB_TRY(gemm_simt_batched(w.descs, 2 * L, rmax, rmax, st));                                // Gram
-  AB_TRY(launch_jacobi(w.jobs, 2 * L, rmax, smem, tol, st));                                // eigen of G_A, G_B
+  const size_t csm = chol_smem_bytes(rmax);
+  AB_CUDA_OK(cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csm));
+  chol_inv_kernel<<<2 * L, kCThreads, csm, st>>>(w.cjobs);                                  // R_A, R_B and inverses
+  AB_LAUNCH_OK();
   AB_TRY(gemm_simt_batched(w.descs + 2 * L, L, rmax, rmax, st));                            // M
-  AB_TRY(launch_jacobi(w.jobs + 2 * L, L, rmax, smem, tol, st));                            // SVD of M
+  AB_TRY(launch_jacobi(w.jobs, L, rmax, smem, tol, st));                                    // SVD of M
   fast_rank_rule_kernel<<<(L + 127) / 128, 128, 0, st>>>(w.sig_ptrs, w.rs, sigma_cutoff, w.rout_ptrs, w.jstatus,
                                                          dev_status, L);
   AB_LAUNCH_OK();
