@@ -14,12 +14,17 @@
 // factors need a condition number below about 300 -- all workloads here are far inside.
 #include <algorithm>
 #include <cstdio>
+#include <type_traits>
 #include <vector>
+
+#include <cooperative_groups.h>
 
 #include "ab_common.cuh"
 
 namespace ab {
 namespace {
+
+namespace cg = cooperative_groups;
 
 constexpr int kJMaxSweeps = 40;
 constexpr float kJDead2 = 1e-12f;    // rows below 1e-6 of the largest norm are zero rows
@@ -46,47 +51,86 @@ __device__ __forceinline__ void rr_pair2(int ne, int t, int idx, int& p, int& q)
   if (p > q) { int tmp = p; p = q; q = tmp; }
 }
 
-template <int kEL, int kJThreads>      // kEL elements per lane and row in registers: r <= 32 kEL
-__global__ void __launch_bounds__(kJThreads, 1)
-jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
+// One matrix per cluster of kC CTAs.  Rows are grouped in blocks of 4; block b lives in the shared
+// memory of CTA b % kC, and every CTA reads and writes any row through distributed shared memory.
+// Each row carries its squared norm in the padding element behind it.  In each round a warp takes
+// one pair of blocks, pulls its 8 rows into registers (r/32 elements per lane and row), rotates the
+// 16 cross pairs (4 steps of 4 disjoint pairs worked on side by side; in the first round of a
+// sweep also the pairs inside each block) and writes the rows back: shared memory is touched once
+// per 16 rotations.  Rounds end with a cluster barrier (a hardware barrier: every CTA of the
+// cluster runs the same number of them, since sweep and round counts depend only on values all
+// CTAs agree on).
+template <int kEL, int kC>      // kEL elements per lane and row in registers: r <= 32 kEL
+__global__ void __launch_bounds__((kC == 1 && kEL == 6) ? 768 : 512, 1)
+jacobi_rows_cluster_kernel(const JacobiJob* __restrict__ jobs, float tol) {
+  cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ __align__(16) float sm[];
-  const JacobiJob job = jobs[blockIdx.x];
+  const int crank = (kC == 1) ? 0 : (int)cluster.block_rank();
+  const JacobiJob job = jobs[blockIdx.x / kC];
   const int k = job.k, r = job.r, ld = r + 1;
-  float* X = sm;                       // k x ld
-  float* n2 = X + (size_t)k * ld;      // squared row norms, k
-  int* rank = reinterpret_cast<int*>(n2 + k);
-  __shared__ int rot_counted;
-  __shared__ float max_n2;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = kJThreads / 32;
-
-  for (int idx = tid; idx < k * r; idx += kJThreads) X[(idx / r) * ld + idx % r] = job.X[idx];
-  __syncthreads();
-
   const int nb = (k + 3) / 4;                  // blocks of 4 rows
+  const int nbl = (nb + kC - 1) / kC;          // blocks held by each CTA (same layout in all)
+  float* X = sm;                               // 4 nbl x ld; X[i * ld + r] = squared norm of local row i
+  float* zrow = X + (size_t)4 * nbl * ld;      // ld zeros: stands in for rows beyond k (rotations leave it zero)
+  float* lmax = zrow + ld;                     // kC: largest squared norm seen by each CTA
+  int* lflag = reinterpret_cast<int*>(lmax + kC);   // kC: "a rotation that counts was applied" per CTA
+  int* rank = lflag + kC;                      // 4 nbl
+  __shared__ int wflag;
+  __shared__ float wmax;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nthreads = blockDim.x, nwarps = nthreads >> 5;
+  auto csync = [&]() {                         // all CTAs that hold a part of this matrix
+    if constexpr (kC == 1) __syncthreads(); else cluster.sync();
+  };
+
+  auto row_ptr = [&](int row) -> float* {      // any row of the matrix, wherever it lives
+    const int b = row >> 2;
+    float* p = X + (size_t)(((b / kC) << 2) + (row & 3)) * ld;
+    if (kC == 1) return p;
+    return cluster.map_shared_rank(p, b % kC);
+  };
+  auto global_row = [&](int lr) { return (((lr >> 2) * kC + crank) << 2) + (lr & 3); };
+  const int nlocal = 4 * nbl;
+
+  for (int lr = warp; lr < nlocal; lr += nwarps) {
+    const int g = global_row(lr);
+    for (int t = lane; t < r; t += 32) X[lr * ld + t] = (g < k) ? job.X[(size_t)g * r + t] : 0.f;
+  }
+  for (int t = tid; t < ld; t += nthreads) zrow[t] = 0.f;
+  csync();                              // every CTA of the cluster is running and loaded
+
+  // exact squared norms of the local rows into their padding element; the cluster-wide maximum
+  auto refresh_norms = [&]() -> float {
+    if (tid == 0) { wmax = 0.f; wflag = 0; }
+    __syncthreads();
+    for (int lr = warp; lr < nlocal; lr += nwarps) {
+      float a = 0.f;
+      for (int t = lane; t < r; t += 32) { const float v = X[lr * ld + t]; a = fmaf(v, v, a); }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+      if (lane == 0) { X[lr * ld + r] = a; atomicMax(reinterpret_cast<int*>(&wmax), __float_as_int(a)); }
+    }
+    __syncthreads();
+    if (tid < kC) {
+      float* dst = (kC == 1) ? lmax : cluster.map_shared_rank(lmax, tid);
+      dst[crank] = wmax;
+    }
+    csync();
+    float m = 0.f;
+#pragma unroll
+    for (int c = 0; c < kC; ++c) m = fmaxf(m, lmax[c]);
+    return m;
+  };
+
   const int nbe = nb + (nb & 1);
   const int brounds = nbe > 2 ? nbe - 1 : 1;
   int sweeps = 0;
   bool converged = (k < 2);
   for (; sweeps < kJMaxSweeps && !converged; ++sweeps) {
-    // exact norms at the start of every sweep (the running updates drift)
-    if (tid == 0) { rot_counted = 0; max_n2 = 0.f; }
-    __syncthreads();
-    for (int i = warp; i < k; i += nwarps) {
-      float a = 0.f;
-      for (int t = lane; t < r; t += 32) { float v = X[i * ld + t]; a = fmaf(v, v, a); }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-      if (lane == 0) { n2[i] = a; atomicMax(reinterpret_cast<int*>(&max_n2), __float_as_int(a)); }
-    }
-    __syncthreads();
+    const float max_n2 = refresh_norms();      // the running updates drift: exact norms every sweep
     const float dead2 = kJDead2 * max_n2, count2 = kJCount2 * max_n2;
-    // Rows are grouped in blocks of 4.  In each round a warp takes one pair of blocks, pulls its 8
-    // rows into registers (r/32 elements per lane and row), rotates the 16 cross pairs (4 steps of
-    // 4 disjoint pairs worked on side by side; in the first round of a sweep also the pairs inside
-    // each block) and writes the rows back: shared memory is touched once per 16 rotations
-    // instead of three times per rotation.
     for (int round = 0; round < brounds; ++round) {
-      for (int task = warp; task < nbe / 2; task += nwarps) {
+      for (int task = crank + kC * warp; task < nbe / 2; task += kC * nwarps) {
         int bi, bj;
         rr_pair2(nbe, round, task, bi, bj);
         const bool has_j = bj < nb;
@@ -94,15 +138,27 @@ jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
         if (!has_j && round != 0) continue;
         float x[8][kEL];
         float nn[8];
+        // where each of the 8 rows lives: an offset into X for a single CTA (fewer registers and
+        // plain shared-memory addressing), a pointer that may lead to a peer's shared memory otherwise
+        typename std::conditional<kC == 1, int, float*>::type ref[8];
+        auto at = [&](int a) -> float* {
+          if constexpr (kC == 1) return X + ref[a]; else return ref[a];
+        };
 #pragma unroll
         for (int a = 0; a < 8; ++a) {
           const int row = (a < 4 ? bi * 4 + a : bj * 4 + (a - 4));
           const bool in = row < k && (a < 4 || has_j);
-          nn[a] = in ? n2[row] : 0.f;
+          if constexpr (kC == 1) ref[a] = in ? row * ld : 4 * nbl * ld;
+          else ref[a] = in ? row_ptr(row) : zrow;
+        }
+#pragma unroll
+        for (int a = 0; a < 8; ++a) {
+          const float* rp = at(a);
+          nn[a] = rp[r];
 #pragma unroll
           for (int e = 0; e < kEL; ++e) {
             const int t = lane + 32 * e;
-            x[a][e] = (in && t < r) ? X[row * ld + t] : 0.f;
+            x[a][e] = (t < r) ? rp[t] : 0.f;
           }
         }
         bool counted = false;
@@ -191,56 +247,117 @@ jacobi_rows_smem_kernel(const JacobiJob* __restrict__ jobs, float tol) {
         }
 #pragma unroll
         for (int a = 0; a < 8; ++a) {
-          const int row = (a < 4 ? bi * 4 + a : bj * 4 + (a - 4));
-          const bool in = row < k && (a < 4 || has_j);
-          if (in) {
+          float* rp = at(a);
 #pragma unroll
-            for (int e = 0; e < kEL; ++e) {
-              const int t = lane + 32 * e;
-              if (t < r) X[row * ld + t] = x[a][e];
-            }
-            if (lane == 0) n2[row] = nn[a];
+          for (int e = 0; e < kEL; ++e) {
+            const int t = lane + 32 * e;
+            if (t < r) rp[t] = x[a][e];
           }
+          if (lane == 0) rp[r] = nn[a];
         }
-        if (lane == 0 && counted) rot_counted = 1;
+        if (lane == 0 && counted) wflag = 1;
       }
-      __syncthreads();
+      csync();                          // all rows of this round are back in place
     }
-    converged = (rot_counted == 0);
-    __syncthreads();
+    if (tid < kC) {
+      int* dst = (kC == 1) ? lflag : cluster.map_shared_rank(lflag, tid);
+      dst[crank] = wflag;
+    }
+    csync();
+    int any = 0;
+#pragma unroll
+    for (int c = 0; c < kC; ++c) any |= lflag[c];
+    converged = (any == 0);
   }
 
-  // norms, descending order, unit rows
-  if (tid == 0) max_n2 = 0.f;
-  __syncthreads();
-  for (int i = warp; i < k; i += nwarps) {
-    float a = 0.f;
-    for (int t = lane; t < r; t += 32) { float v = X[i * ld + t]; a = fmaf(v, v, a); }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-    if (lane == 0) { n2[i] = a; atomicMax(reinterpret_cast<int*>(&max_n2), __float_as_int(a)); }
-  }
-  __syncthreads();
-  for (int i = tid; i < k; i += kJThreads) {
-    const float li = n2[i];
+  // norms, descending order, unit rows: each CTA finishes the rows it holds
+  const float max_n2 = refresh_norms();
+  for (int lr = tid; lr < nlocal; lr += nthreads) {
+    const int gi = global_row(lr);
+    if (gi >= k) continue;
+    const float li = X[lr * ld + r];
     int rk = 0;
-    for (int j = 0; j < k; ++j) { const float lj = n2[j]; rk += (lj > li) || (lj == li && j < i); }
-    rank[i] = rk;
+    for (int j = 0; j < k; ++j) { const float lj = row_ptr(j)[r]; rk += (lj > li) || (lj == li && j < gi); }
+    rank[lr] = rk;
   }
   __syncthreads();
   const float dead2 = kJDead2 * max_n2;
-  for (int i = warp; i < k; i += nwarps) {
-    const float a = n2[i];
+  for (int lr = warp; lr < nlocal; lr += nwarps) {
+    if (global_row(lr) >= k) continue;
+    const float a = X[lr * ld + r];
     const bool live = a > dead2 && a > 0.f;
     const float nrm = live ? sqrtf(a) : 0.f, inv = live ? 1.f / nrm : 0.f;
-    float* dst = job.rows + (size_t)rank[i] * r;
-    for (int t = lane; t < r; t += 32) dst[t] = X[i * ld + t] * inv;
-    if (lane == 0) job.norms[rank[i]] = nrm;
+    float* dst = job.rows + (size_t)rank[lr] * r;
+    for (int t = lane; t < r; t += 32) dst[t] = X[lr * ld + t] * inv;
+    if (lane == 0) job.norms[rank[lr]] = nrm;
   }
-  if (tid == 0 && job.status) *job.status = converged ? AB_OK : AB_ERR_NOT_CONVERGED;
+  if (crank == 0 && tid == 0 && job.status) *job.status = converged ? AB_OK : AB_ERR_NOT_CONVERGED;
 #ifdef AB_TRACE_SWEEPS
-  if (tid == 0) printf("jacobi job %d: k=%d r=%d sweeps=%d converged=%d\n", (int)blockIdx.x, k, r, sweeps, (int)converged);
+  if (crank == 0 && tid == 0) printf("jacobi job %d: k=%d r=%d sweeps=%d converged=%d\n", (int)(blockIdx.x / kC), k, r, sweeps, (int)converged);
 #endif
+  csync();                              // nobody leaves while a peer may still read its rows
+}
+
+size_t jacobi_smem_bytes(int k, int r, int C) {
+  const int nbl = ((k + 3) / 4 + C - 1) / C;
+  return sizeof(float) * ((size_t)(4 * nbl + 1) * (r + 1) + C) + sizeof(int) * ((size_t)C + 4 * nbl) + 64;
+}
+
+template <int EL, int C>
+cudaLaunchConfig_t jacobi_config(int count, int rmax, cudaStream_t st, cudaLaunchAttribute* attr) {
+  const int tasks = ((rmax + 3) / 4 + 1) / 2;                         // block pairs per round
+  const int max_warps = (C == 1 && EL == 6) ? 24 : 16;              // matches the kernel's launch bounds
+  const int warps = std::max(1, std::min(max_warps, (tasks + C - 1) / C));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(count * C));
+  cfg.blockDim = dim3((unsigned)(32 * warps));
+  cfg.dynamicSmemBytes = jacobi_smem_bytes(rmax, rmax, C);
+  cfg.stream = st;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cfg;
+}
+// Launches with clusters of C CTAs if `count` such clusters can be resident at once (or if C == 1).
+// Returns 1 when it declined, so that the caller tries a narrower cluster.
+template <int EL, int C>
+int try_launch_jacobi(const JacobiJob* jobs, int count, int rmax, float tol, cudaStream_t st) {
+  cudaLaunchAttribute attr[1];
+  cudaLaunchConfig_t cfg = jacobi_config<EL, C>(count, rmax, st, attr);
+  if (cfg.dynamicSmemBytes > 227u * 1024u) return C == 1 ? AB_ERR_UNSUPPORTED : 1;
+  AB_CUDA_OK(cudaFuncSetAttribute(jacobi_rows_cluster_kernel<EL, C>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)cfg.dynamicSmemBytes));
+  if (C > 1) {
+    // one CTA per SM: CTAs that share an SM would only take turns on its issue slots
+    int dev = 0, sms = 0, resident = 0;
+    AB_CUDA_OK(cudaGetDevice(&dev));
+    AB_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (rmax < 16 * C || (long long)count * C > sms) return 1;
+    if (cudaOccupancyMaxActiveClusters(&resident, jacobi_rows_cluster_kernel<EL, C>, &cfg) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return 1;
+    }
+    if (resident < count) return 1;
+  }
+  AB_CUDA_OK(cudaLaunchKernelEx(&cfg, jacobi_rows_cluster_kernel<EL, C>, jobs, tol));
+  AB_LAUNCH_OK();
+  return AB_OK;
+}
+// Clusters of 8 or 4 CTAs per matrix when that many SMs are free for every matrix, else one CTA each
+// (measured: a pair of CTAs gains nothing over one CTA with twice the warps; the round time is then
+// set by the latency of one warp's 16 rotations, not by issue slots).
+template <int EL>
+int launch_jacobi_el(const JacobiJob* jobs, int count, int rmax, float tol, cudaStream_t st) {
+  int s = try_launch_jacobi<EL, 8>(jobs, count, rmax, tol, st);
+  if (s == 1) s = try_launch_jacobi<EL, 4>(jobs, count, rmax, tol, st);
+  if (s == 1) s = try_launch_jacobi<EL, 1>(jobs, count, rmax, tol, st);
+  return s;
+}
+int launch_jacobi(const JacobiJob* jobs, int count, int rmax, float tol, cudaStream_t st) {
+  if (rmax <= 64) return launch_jacobi_el<2>(jobs, count, rmax, tol, st);
+  if (rmax <= 128) return launch_jacobi_el<4>(jobs, count, rmax, tol, st);
+  if (rmax <= 192) return launch_jacobi_el<6>(jobs, count, rmax, tol, st);
+  return launch_jacobi_el<8>(jobs, count, rmax, tol, st);
 }
 
 struct CholJob {
@@ -308,22 +425,6 @@ __global__ void __launch_bounds__(kCThreads, 1) chol_inv_kernel(const CholJob* _
 }
 
 size_t chol_smem_bytes(int r) { return sizeof(float) * ((size_t)r * (r + 1) + r) + 64; }
-
-template <int EL, int TH>
-int launch_jacobi_t(const JacobiJob* jobs, int count, size_t smem, float tol, cudaStream_t st) {
-  AB_CUDA_OK(cudaFuncSetAttribute(jacobi_rows_smem_kernel<EL, TH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  jacobi_rows_smem_kernel<EL, TH><<<count, TH, smem, st>>>(jobs, tol);
-  AB_LAUNCH_OK();
-  return AB_OK;
-}
-int launch_jacobi(const JacobiJob* jobs, int count, int rmax, size_t smem, float tol, cudaStream_t st) {
-  if (rmax <= 64) return launch_jacobi_t<2, 512>(jobs, count, smem, tol, st);
-  if (rmax <= 128) return launch_jacobi_t<4, 512>(jobs, count, smem, tol, st);
-  if (rmax <= 192) return launch_jacobi_t<6, 768>(jobs, count, smem, tol, st);
-  return launch_jacobi_t<8, 512>(jobs, count, smem, tol, st);
-}
-
-size_t jacobi_smem_bytes(int k, int r) { return sizeof(float) * ((size_t)k * (r + 1) + k) + sizeof(int) * k + 64; }
 
 // r' = #{ i < r : sigma_i >= cutoff * sigma_0 } (at least 1); folds the three solver statuses.
 __global__ void fast_rank_rule_kernel(const float* const* __restrict__ sigma, const int* __restrict__ rs,
@@ -397,7 +498,7 @@ GemmDesc mk(const float* A, int64_t sAm, int64_t sAk, const float* B, int64_t sB
 
 bool sync_factored_supported(const ab_sync_desc* d, int L) {
   for (int i = 0; i < L; ++i)
-    if (jacobi_smem_bytes(d[i].r, d[i].r) > 227 * 1024 || d[i].r > 256) return false;
+    if (chol_smem_bytes(d[i].r) > 227 * 1024 || d[i].r > 256) return false;
   return true;
 }
 
@@ -462,7 +563,6 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
     AB_TRY(group_average(d[i].A_copies, d[i].strideA, K, (int64_t)d[i].m * d[i].r, dt, AB_F32, w.Abar[i], st));
     AB_TRY(group_average(d[i].B_copies, d[i].strideB, K, (int64_t)d[i].r * d[i].n, dt, AB_F32, w.Bbar[i], st));
   }
-  const size_t smem = jacobi_smem_bytes(rmax, rmax);
   const float tol = 5e-7f * sqrtf((float)rmax) < 4e-6f ? 4e-6f : 5e-7f * sqrtf((float)rmax);
   bool any_w = false;
   for (int i = 0; i < L; ++i) any_w = any_w || d[i].W_out != nullptr;
@@ -473,7 +573,7 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   chol_inv_kernel<<<2 * L, kCThreads, csm, st>>>(w.cjobs);                                  // R_A, R_B and inverses
   AB_LAUNCH_OK();
   AB_TRY(gemm_simt_batched(w.descs + 2 * L, L, rmax, rmax, st));                            // M
-  AB_TRY(launch_jacobi(w.jobs, L, rmax, smem, tol, st));                                    // SVD of M
+  AB_TRY(launch_jacobi(w.jobs, L, rmax, tol, st));                                    // SVD of M
   fast_rank_rule_kernel<<<(L + 127) / 128, 128, 0, st>>>(w.sig_ptrs, w.rs, sigma_cutoff, w.rout_ptrs, w.jstatus,
                                                          dev_status, L);
   AB_LAUNCH_OK();
