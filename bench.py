@@ -78,7 +78,7 @@ class ClockSampler(threading.Thread):
                 for b, nm in names.items():
                     if bits & b:
                         self.reasons.add(nm)
-                time.sleep(0.05)
+                time.sleep(0.002)
         except Exception as e:  # clocks are evidence, not a dependency of the measurement
             self.reasons.add(f"nvml_unavailable:{type(e).__name__}")
 
@@ -393,7 +393,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=256 * 197, help="token rows per layer (default: batch 256 x 197)")

@@ -168,7 +168,7 @@ typedef struct {
 typedef enum {
   AB_SYNC_AUTO = 0,      /* factored when it applies, else dense */
   AB_SYNC_DENSE = 1,     /* form W, then the dense split of ab_svd_split */
-  AB_SYNC_FACTORED = 2   /* never form W: r x r eigen/SVD problems only (rank(W) <= r makes this exact) */
+  AB_SYNC_FACTORED = 2   /* never form W: r x r Cholesky/SVD problems only (rank(W) <= r makes this exact) */
 } ab_sync_path;
 
 /*
@@ -177,11 +177,12 @@ typedef enum {
  * Bbar, then the split of W as in ab_svd_split.  descs: HOST array of L descriptors (read
  * before the call returns).  Factor storage dt on both sides.  dev_status: device int[L].
  * path: an ab_sync_path.  The factored path uses that W = Abar Bbar has rank <= r: the
- * decomposition reduces to eigen-problems of Abar^T Abar and Bbar Bbar^T and the SVD of an
- * r x r core, each solved inside one CTA's shared memory; W itself is only written if W_out
- * asks for it.  It needs r <= 232 and factors whose condition number is below about 300
- * (eigenvalues of the two Gram matrices under 1e-6 of the largest are taken as zero, which is
- * exact for factors already truncated by the rank rule); AB_SYNC_FACTORED returns
+ * decomposition reduces to Cholesky factors of Abar^T Abar and Bbar Bbar^T and the SVD of an
+ * r x r core, each solved inside shared memory (one CTA, or a cluster of CTAs, per matrix); W
+ * itself is only written if W_out asks for it.  It needs r <= 236 (shared-memory capacity) and
+ * factors whose condition number is below about 300 (Cholesky pivots under 1e-6 of the largest
+ * diagonal entry of a Gram matrix are taken as zero, which is exact for factors already
+ * truncated by the rank rule); AB_SYNC_FACTORED returns
  * AB_ERR_UNSUPPORTED when r is too large, AB_SYNC_AUTO falls back to the dense path.
  * Workspace: ab_sync_workspace_bytes (covers either path).
  */
