@@ -497,9 +497,9 @@ GemmDesc mk(const float* A, int64_t sAm, int64_t sAk, const float* B, int64_t sB
 }  // namespace
 
 bool sync_factored_supported(const ab_sync_desc* d, int L) {
+  // dynamic shared memory of the two single-CTA kernels, with room for their few static words
+  const size_t cap = 227 * 1024 - 256;
   for (int i = 0; i < L; ++i)
-    // dynamic shared memory of the two single-CTA kernels, with room for their few static words
-    const size_t cap = 227 * 1024 - 256;
     if (chol_smem_bytes(d[i].r) > cap || jacobi_smem_bytes(d[i].r, d[i].r, 1) > cap) return false;
   return true;
 }
