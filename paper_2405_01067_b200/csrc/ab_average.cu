@@ -2,6 +2,8 @@
 // Each thread owns 16 input bytes per copy (4 fp32 or 8 bf16 values), keeps up to four copies'
 // loads in flight, adds them in fp32 in ascending k and scales by fl(1/K).  The sum order is
 // part of the contract (results are compared bit for bit).
+#include <algorithm>
+
 #include "ab_common.cuh"
 
 namespace ab {
@@ -45,34 +47,61 @@ __device__ __forceinline__ void store_vec(bf16* p, const float (&v)[N]) {
   else __stcs(reinterpret_cast<uint2*>(p), make_uint2(w[0], w[1]));
 }
 
+// Mean of element group i (V values) of K copies: the one place that fixes the order of the sums.
+template <typename TIn, typename TOut>
+__device__ __forceinline__ void mean_vec_at(const TIn* __restrict__ base, int64_t stride, int K, float inv,
+                                            TOut* __restrict__ out, int64_t i) {
+  constexpr int V = Vec<TIn>::N;
+  const TIn* p = base + i * V;
+  float s[V];
+  Vec<TIn>::load(p, s);
+  int k = 1;
+  for (; k + 3 <= K; k += 3) {       // three more copies in flight, added in ascending k
+    float a[V], b[V], c[V];
+    Vec<TIn>::load(p + (int64_t)k * stride, a);
+    Vec<TIn>::load(p + (int64_t)(k + 1) * stride, b);
+    Vec<TIn>::load(p + (int64_t)(k + 2) * stride, c);
+#pragma unroll
+    for (int j = 0; j < V; ++j) s[j] = __fadd_rn(__fadd_rn(__fadd_rn(s[j], a[j]), b[j]), c[j]);
+  }
+  for (; k < K; ++k) {
+    float a[V];
+    Vec<TIn>::load(p + (int64_t)k * stride, a);
+#pragma unroll
+    for (int j = 0; j < V; ++j) s[j] = __fadd_rn(s[j], a[j]);
+  }
+#pragma unroll
+  for (int j = 0; j < V; ++j) s[j] = __fmul_rn(s[j], inv);
+  store_vec<V>(out + i * V, s);
+}
+
 template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(256)
 average_vec_kernel(const TIn* __restrict__ base, int64_t stride, int K, int64_t nvec, float inv,
                    TOut* __restrict__ out) {
-  constexpr int V = Vec<TIn>::N;
   const int64_t step = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step) {
-    const TIn* p = base + i * V;
-    float s[V];
-    Vec<TIn>::load(p, s);
-    int k = 1;
-    for (; k + 3 <= K; k += 3) {       // three more copies in flight, added in ascending k
-      float a[V], b[V], c[V];
-      Vec<TIn>::load(p + (int64_t)k * stride, a);
-      Vec<TIn>::load(p + (int64_t)(k + 1) * stride, b);
-      Vec<TIn>::load(p + (int64_t)(k + 2) * stride, c);
-#pragma unroll
-      for (int j = 0; j < V; ++j) s[j] = __fadd_rn(__fadd_rn(__fadd_rn(s[j], a[j]), b[j]), c[j]);
-    }
-    for (; k < K; ++k) {
-      float a[V];
-      Vec<TIn>::load(p + (int64_t)k * stride, a);
-#pragma unroll
-      for (int j = 0; j < V; ++j) s[j] = __fadd_rn(s[j], a[j]);
-    }
-#pragma unroll
-    for (int j = 0; j < V; ++j) s[j] = __fmul_rn(s[j], inv);
-    store_vec<V>(out + i * V, s);
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += step)
+    mean_vec_at<TIn, TOut>(base, stride, K, inv, out, i);
+}
+
+// Many means in one launch (blockIdx.y = job), fp32 results: the vector body where the job's
+// pointers and stride allow it, single elements for the rest.  Same sums as the kernels above.
+template <typename TIn>
+__global__ void __launch_bounds__(256)
+average_batched_kernel(const AvgJob* __restrict__ jobs, int K, float inv) {
+  constexpr int V = Vec<TIn>::N;
+  const AvgJob j = jobs[blockIdx.y];
+  const TIn* base = static_cast<const TIn*>(j.base);
+  const bool vec_ok = ((reinterpret_cast<uintptr_t>(j.base) | reinterpret_cast<uintptr_t>(j.out)) & 15u) == 0 &&
+                      (j.stride % V == 0);
+  const int64_t nvec = vec_ok ? j.count / V : 0;
+  const int64_t step = (int64_t)gridDim.x * blockDim.x;
+  const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (int64_t i = t0; i < nvec; i += step) mean_vec_at<TIn, float>(base, j.stride, K, inv, j.out, i);
+  for (int64_t i = nvec * V + t0; i < j.count; i += step) {
+    float s = to_f32(base[i]);
+    for (int k = 1; k < K; ++k) s = __fadd_rn(s, to_f32(base[i + (int64_t)k * j.stride]));
+    j.out[i] = __fmul_rn(s, inv);
   }
 }
 
@@ -126,6 +155,19 @@ int group_average(const void* base, int64_t stride_elems, int K, int64_t count,
   if (in_dt == AB_F32 && out_dt == AB_BF16) return run<float, bf16>(base, stride_elems, K, count, out, st);
   if (in_dt == AB_BF16 && out_dt == AB_F32) return run<bf16, float>(base, stride_elems, K, count, out, st);
   return run<bf16, bf16>(base, stride_elems, K, count, out, st);
+}
+
+int group_average_batched(const AvgJob* d_jobs, int njobs, int K, int in_dt, int64_t max_count, cudaStream_t st) {
+  if (njobs <= 0 || max_count <= 0) return AB_OK;
+  const int64_t blocks = (max_count / 4 + 255) / 256 + 1;
+  const int64_t cap = std::max<int64_t>(1, (int64_t)148 * 8 / njobs);
+  dim3 grid((unsigned)std::min(blocks, cap), (unsigned)njobs);
+  if (grid.y > 65535u) return AB_ERR_UNSUPPORTED;
+  const float inv = 1.0f / (float)K;
+  if (in_dt == AB_F32) average_batched_kernel<float><<<grid, 256, 0, st>>>(d_jobs, K, inv);
+  else average_batched_kernel<bf16><<<grid, 256, 0, st>>>(d_jobs, K, inv);
+  AB_LAUNCH_OK();
+  return AB_OK;
 }
 
 }  // namespace ab

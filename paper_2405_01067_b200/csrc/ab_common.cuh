@@ -85,6 +85,7 @@ struct GemmDesc {
   int row_mode, col_mode, k_mode;
   float thr;
   const int* live_rows; const int* live_cols;
+  int upper_only;   // 1: tiles entirely below the diagonal are skipped (symmetric result, upper part used)
 };
 int gemm_simt_batched(const GemmDesc* d_descs, int count, int max_M, int max_N, cudaStream_t st);
 
@@ -123,6 +124,9 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
                   void* ws, size_t ws_bytes, cudaStream_t st);
 
 // ---- group mean (ab_average.cu) ----------------------------------------------------------------
+// One mean per job in a single launch; results are fp32.  d_jobs is device memory.
+struct AvgJob { const void* base; int64_t stride; int64_t count; float* out; };
+int group_average_batched(const AvgJob* d_jobs, int njobs, int K, int in_dt, int64_t max_count, cudaStream_t st);
 int group_average(const void* base, int64_t stride_elems, int K, int64_t count,
                   int in_dt, int out_dt, void* out, cudaStream_t st);
 

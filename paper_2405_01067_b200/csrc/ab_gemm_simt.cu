@@ -189,6 +189,7 @@ gemm_simt_batched_kernel(const GemmDesc* __restrict__ descs) {
   const GemmDesc d = descs[blockIdx.z];
   const int64_t m0 = (int64_t)blockIdx.y * BM_, n0 = (int64_t)blockIdx.x * BN_;
   if (m0 >= d.M || n0 >= d.N) return;
+  if (d.upper_only && n0 + BN_ <= m0) return;
   __shared__ __align__(16) float As[2][BK][BM_ + 4];
   __shared__ __align__(16) float Bs[2][BK][BN_ + 4];
   const int tid = threadIdx.x;

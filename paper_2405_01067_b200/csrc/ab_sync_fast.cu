@@ -361,7 +361,9 @@ int launch_jacobi(const JacobiJob* jobs, int count, int rmax, float tol, cudaStr
 }
 
 struct CholJob {
-  const float* G;   // r x r symmetric positive semi-definite (row stride r)
+  const float* G;   // nparts partial sums of an r x r symmetric positive semi-definite matrix (row stride r,
+                    // r * r apart); only the upper triangle is read
+  int nparts;
   float* R;         // r x r upper triangular, G = R^T R; zeros below the diagonal, dropped rows zero
   float* Rinv;      // r x r upper triangular inverse of the kept part; dropped rows and columns zero
   int* status;      // receives AB_OK (may be null)
@@ -381,7 +383,11 @@ __global__ void __launch_bounds__(kCThreads, 1) chol_inv_kernel(const CholJob* _
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = kCThreads / 32;
 
   if (tid == 0) maxdiag = 0.f;
-  for (int idx = tid; idx < r * r; idx += kCThreads) S[(idx / r) * ld + idx % r] = job.G[idx];
+  for (int idx = tid; idx < r * r; idx += kCThreads) {
+    float v = job.G[idx];
+    for (int q = 1; q < job.nparts; ++q) v += job.G[(size_t)q * r * r + idx];      // ascending part order
+    S[(idx / r) * ld + idx % r] = v;
+  }
   __syncthreads();
   for (int i = tid; i < r; i += kCThreads)
     atomicMax(reinterpret_cast<int*>(&maxdiag), __float_as_int(fmaxf(S[i * ld + i], 0.f)));
@@ -447,10 +453,21 @@ __global__ void fast_rank_rule_kernel(const float* const* __restrict__ sigma, co
   }
 }
 
+// The long index of a Gram product is cut into slices of about kGramSlice (at most kGramMaxParts).
+constexpr int kGramSlice = 768, kGramMaxParts = 8;
+int gram_parts(int len) { return std::max(1, std::min(kGramMaxParts, (len + kGramSlice - 1) / kGramSlice)); }
+int gram_k0(int len, int parts, int q) {      // start of slice q (a multiple of 16), len for q == parts
+  if (q >= parts) return len;
+  const int per = (((len + parts - 1) / parts) + 15) / 16 * 16;
+  return std::min(len, q * per);
+}
+
 struct FastWs {
   std::vector<float*> Abar, Bbar, GA, GB, RA, RB, IA, IB, M, Vs, Y1, ZA, ZB;
   GemmDesc* descs;      // 9 L
+  GemmDesc* gram_descs; // up to 2 kGramMaxParts L
   CholJob* cjobs;       // 2 L
+  AvgJob* ajobs;        // 2 L
   JacobiJob* jobs;      // L
   int* jstatus;         // 3 L
   const float** sig_ptrs;
@@ -469,10 +486,14 @@ FastWs fast_layout(const ab_sync_desc* d, int L, void* ws) {
   each(w.Abar, [](const ab_sync_desc& x) { return (size_t)x.m * x.r; });
   each(w.Bbar, [](const ab_sync_desc& x) { return (size_t)x.r * x.n; });
   auto rr = [](const ab_sync_desc& x) { return (size_t)x.r * x.r; };
-  each(w.GA, rr); each(w.GB, rr); each(w.RA, rr); each(w.RB, rr); each(w.IA, rr); each(w.IB, rr);
+  each(w.GA, [](const ab_sync_desc& x) { return (size_t)gram_parts(x.m) * x.r * x.r; });
+  each(w.GB, [](const ab_sync_desc& x) { return (size_t)gram_parts(x.n) * x.r * x.r; });
+  each(w.RA, rr); each(w.RB, rr); each(w.IA, rr); each(w.IB, rr);
   each(w.M, rr); each(w.Vs, rr); each(w.Y1, rr); each(w.ZA, rr); each(w.ZB, rr);
   w.descs = ar.take_n<GemmDesc>((size_t)9 * L);
+  w.gram_descs = ar.take_n<GemmDesc>((size_t)2 * kGramMaxParts * L);
   w.cjobs = ar.take_n<CholJob>((size_t)2 * L);
+  w.ajobs = ar.take_n<AvgJob>((size_t)2 * L);
   w.jobs = ar.take_n<JacobiJob>((size_t)L);
   w.jstatus = ar.take_n<int>((size_t)3 * L);
   w.sig_ptrs = ar.take_n<const float*>(L);
@@ -491,6 +512,7 @@ GemmDesc mk(const float* A, int64_t sAm, int64_t sAk, const float* B, int64_t sB
   g.row_mode = g.col_mode = g.k_mode = 0;
   g.thr = kEigThr;
   g.live_rows = g.live_cols = nullptr;
+  g.upper_only = 0;
   return g;
 }
 
@@ -518,6 +540,8 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   // ---- host-built tables: 9 GEMM descriptors, 2 Cholesky jobs and 1 Jacobi job per matrix, copied in one go each
   std::vector<GemmDesc> g((size_t)9 * L);
   std::vector<CholJob> cj((size_t)2 * L);
+  std::vector<GemmDesc> gg;
+  gg.reserve((size_t)2 * kGramMaxParts * L);
   std::vector<JacobiJob> jb((size_t)L);
   std::vector<const float*> sigp(L);
   std::vector<int*> routp(L);
@@ -525,9 +549,10 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   for (int i = 0; i < L; ++i) {
     const int m = d[i].m, n = d[i].n, r = d[i].r;
     float *Ab = w.Abar[i], *Bb = w.Bbar[i];
-    // batch 0 (2L): Gram matrices
-    g[0 * L + i] = mk(Ab, 1, r, Ab, r, 1, w.GA[i], r, r, r, m);           // G_A = Abar^T Abar
-    g[1 * L + i] = mk(Bb, n, 1, Bb, 1, n, w.GB[i], r, r, r, n);           // G_B = Bbar Bbar^T
+    // (slots 0 .. 2L of this table are unused: the Gram products G_A = Abar^T Abar and
+    // G_B = Bbar Bbar^T have a table of their own, one entry per slice of the long index)
+    g[0 * L + i] = mk(nullptr, 0, 0, nullptr, 0, 0, nullptr, 0, 0, 0, 0);
+    g[1 * L + i] = g[0 * L + i];
     // batch 1 (L): M = R_A R_B^T
     g[2 * L + i] = mk(w.RA[i], r, 1, w.RB[i], 1, r, w.M[i], r, r, r, r);
     // batch 2 (2L): Y1 = M Vs^T ;  Z_B = diag(sqrt sig) Vs R_B^-T
@@ -548,28 +573,51 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
     gb.c_bf16 = out_bf16; gb.live_rows = d[i].r_out;
     // batch 6 (L, optional): W = Abar Bbar
     g[8 * L + i] = mk(Ab, r, 1, Bb, n, 1, d[i].W_out, n, d[i].W_out ? m : 0, d[i].W_out ? n : 0, r);
-    cj[i] = CholJob{w.GA[i], w.RA[i], w.IA[i], w.jstatus + 3 * i, r};
-    cj[L + i] = CholJob{w.GB[i], w.RB[i], w.IB[i], w.jstatus + 3 * i + 1, r};
+    const int pa = gram_parts(m), pb = gram_parts(n);
+    cj[i] = CholJob{w.GA[i], pa, w.RA[i], w.IA[i], w.jstatus + 3 * i, r};
+    cj[L + i] = CholJob{w.GB[i], pb, w.RB[i], w.IB[i], w.jstatus + 3 * i + 1, r};
+    // Gram matrices in slices of the long index (equal work per CTA, partial sums added by the
+    // Cholesky kernel in ascending slice order), upper tiles only
+    for (int q = 0; q < pa; ++q) {
+      const int k0 = gram_k0(m, pa, q), k1 = gram_k0(m, pa, q + 1);
+      GemmDesc x = mk(Ab + (size_t)k0 * r, 1, r, Ab + (size_t)k0 * r, r, 1, w.GA[i] + (size_t)q * r * r, r, r, r, k1 - k0);
+      x.upper_only = 1;
+      gg.push_back(x);
+    }
+    for (int q = 0; q < pb; ++q) {
+      const int k0 = gram_k0(n, pb, q), k1 = gram_k0(n, pb, q + 1);
+      GemmDesc x = mk(Bb + k0, n, 1, Bb + k0, 1, n, w.GB[i] + (size_t)q * r * r, r, r, r, k1 - k0);
+      x.upper_only = 1;
+      gg.push_back(x);
+    }
     jb[i] = JacobiJob{w.M[i], w.Vs[i], d[i].sigma, w.jstatus + 3 * i + 2, r, r};
     sigp[i] = d[i].sigma; routp[i] = d[i].r_out; rs[i] = r;
   }
   AB_CUDA_OK(cudaMemcpyAsync(w.descs, g.data(), g.size() * sizeof(GemmDesc), cudaMemcpyHostToDevice, st));
+  AB_CUDA_OK(cudaMemcpyAsync(w.gram_descs, gg.data(), gg.size() * sizeof(GemmDesc), cudaMemcpyHostToDevice, st));
   AB_CUDA_OK(cudaMemcpyAsync(w.cjobs, cj.data(), cj.size() * sizeof(CholJob), cudaMemcpyHostToDevice, st));
   AB_CUDA_OK(cudaMemcpyAsync(w.jobs, jb.data(), jb.size() * sizeof(JacobiJob), cudaMemcpyHostToDevice, st));
   AB_CUDA_OK(cudaMemcpyAsync(w.sig_ptrs, sigp.data(), L * sizeof(float*), cudaMemcpyHostToDevice, st));
   AB_CUDA_OK(cudaMemcpyAsync(w.rout_ptrs, routp.data(), L * sizeof(int*), cudaMemcpyHostToDevice, st));
   AB_CUDA_OK(cudaMemcpyAsync(w.rs, rs.data(), L * sizeof(int), cudaMemcpyHostToDevice, st));
 
-  // ---- a7: means of the K copies (fp32)
-  for (int i = 0; i < L; ++i) {
-    AB_TRY(group_average(d[i].A_copies, d[i].strideA, K, (int64_t)d[i].m * d[i].r, dt, AB_F32, w.Abar[i], st));
-    AB_TRY(group_average(d[i].B_copies, d[i].strideB, K, (int64_t)d[i].r * d[i].n, dt, AB_F32, w.Bbar[i], st));
+  // ---- a7: means of the K copies (fp32), all matrices in one launch
+  {
+    std::vector<AvgJob> aj((size_t)2 * L);
+    int64_t longest = 0;
+    for (int i = 0; i < L; ++i) {
+      aj[2 * i] = AvgJob{d[i].A_copies, d[i].strideA, (int64_t)d[i].m * d[i].r, w.Abar[i]};
+      aj[2 * i + 1] = AvgJob{d[i].B_copies, d[i].strideB, (int64_t)d[i].r * d[i].n, w.Bbar[i]};
+      longest = std::max(longest, std::max(aj[2 * i].count, aj[2 * i + 1].count));
+    }
+    AB_CUDA_OK(cudaMemcpyAsync(w.ajobs, aj.data(), aj.size() * sizeof(AvgJob), cudaMemcpyHostToDevice, st));
+    AB_TRY(group_average_batched(w.ajobs, 2 * L, K, dt, longest, st));
   }
   const float tol = 5e-7f * sqrtf((float)rmax) < 4e-6f ? 4e-6f : 5e-7f * sqrtf((float)rmax);
   bool any_w = false;
   for (int i = 0; i < L; ++i) any_w = any_w || d[i].W_out != nullptr;
   if (any_w) AB_TRY(gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, st));                 // a8 (optional)
-  AB_TRY(gemm_simt_batched(w.descs, 2 * L, rmax, rmax, st));                                // Gram
+  AB_TRY(gemm_simt_batched(w.gram_descs, (int)gg.size(), rmax, rmax, st));                  // Gram slices
   const size_t csm = chol_smem_bytes(rmax);
   AB_CUDA_OK(cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csm));
   chol_inv_kernel<<<2 * L, kCThreads, csm, st>>>(w.cjobs);                                  // R_A, R_B and inverses
