@@ -370,9 +370,9 @@ struct CholJob {
   int r;
 };
 
-// Right-looking Cholesky of one Gram matrix in shared memory, then the inverse of the triangle by
-// back substitution, one warp per column.  R lives in the upper triangle; column j of the inverse
-// is parked in the strict lower triangle of row j (contiguous), its diagonal in dinv[].
+// Right-looking Cholesky of one Gram matrix in shared memory (r <= 256), then the inverse of the
+// triangle by back substitution, one warp per column.  R lives in the upper triangle; column j of
+// the inverse is parked in the strict lower triangle of row j (contiguous), its diagonal in dinv[].
 __global__ void __launch_bounds__(kCThreads, 1) chol_inv_kernel(const CholJob* __restrict__ jobs) {
   extern __shared__ __align__(16) float sm[];
   const CholJob job = jobs[blockIdx.x];
@@ -409,16 +409,37 @@ __global__ void __launch_bounds__(kCThreads, 1) chol_inv_kernel(const CholJob* _
     __syncthreads();
   }
 
-  // X = R^-1 restricted to the kept rows: X_jj = 1/R_jj, X_ij = -(sum_{i<k<=j} R_ik X_kj) / R_ii
+  // X = R^-1 restricted to the kept rows, one warp per column j, by back substitution in update
+  // form: lane l owns rows l, l + 32, ... of the column.  b starts as e_j; going down from k = j,
+  // x_k = b_k / R_kk is final (one shuffle hands it to all lanes) and every row i < k takes
+  // b_i -= R_ik x_k -- no reduction across lanes, and only the upper triangle (R) is read.
   for (int j = warp; j < r; j += nwarps) {
-    const float xjj = dinv[j];
-    for (int i = j - 1; i >= 0; --i) {
-      float acc = 0.f;
-      for (int k = i + 1 + lane; k < j; k += 32) acc = fmaf(S[i * ld + k], S[j * ld + k], acc);
+    float b[8], dk[8];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      if (lane == 0) S[j * ld + i] = -dinv[i] * fmaf(S[i * ld + j], xjj, acc);
-      __syncwarp();
+    for (int e = 0; e < 8; ++e) {
+      const int i = 32 * e + lane;
+      b[e] = (i == j) ? 1.f : 0.f;
+      dk[e] = (i < r) ? dinv[i] : 0.f;
+    }
+#pragma unroll
+    for (int e = 7; e >= 0; --e) {
+      if (32 * e > j) continue;                  // uniform over the warp
+      const int ltop = (j - 32 * e < 31) ? j - 32 * e : 31;
+      for (int l = ltop; l >= 0; --l) {
+        const int k = 32 * e + l;
+        const float xk = __shfl_sync(0xffffffffu, b[e] * dk[e], l);
+        if (lane == l) b[e] = xk;
+#pragma unroll
+        for (int e2 = 0; e2 <= e; ++e2) {
+          const int i = 32 * e2 + lane;
+          if (i < k) b[e2] = fmaf(-S[i * ld + k], xk, b[e2]);
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int i = 32 * e + lane;
+      if (i < j) S[j * ld + i] = b[e];           // column j of X, parked in row j below the diagonal
     }
   }
   __syncthreads();
