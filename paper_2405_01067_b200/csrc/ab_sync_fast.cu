@@ -29,6 +29,8 @@ namespace cg = cooperative_groups;
 constexpr int kJMaxSweeps = 40;
 constexpr float kJDead2 = 1e-12f;    // rows below 1e-6 of the largest norm are zero rows
 constexpr float kJCount2 = 1e-8f;    // rows below 1e-4 of the largest norm do not hold up convergence
+constexpr float kJEarly2 = 9e-8f;    // a sweep whose largest rotated cosine was below 3e-4 is the last one: one-sided
+                                     // Jacobi converges quadratically, so what it leaves is of the order 1e-7 < tol
 constexpr float kEigThr = 1e-6f;     // relative pivot cut of G_A, G_B (and of sigma in the scalings)
 constexpr int kCThreads = 512;
 
@@ -73,7 +75,7 @@ jacobi_rows_cluster_kernel(const JacobiJob* __restrict__ jobs, float tol) {
   float* X = sm;                               // 4 nbl x ld; X[i * ld + r] = squared norm of local row i
   float* zrow = X + (size_t)4 * nbl * ld;      // ld zeros: stands in for rows beyond k (rotations leave it zero)
   float* lmax = zrow + ld;                     // kC: largest squared norm seen by each CTA
-  int* lflag = reinterpret_cast<int*>(lmax + kC);   // kC: "a rotation that counts was applied" per CTA
+  int* lflag = reinterpret_cast<int*>(lmax + kC);   // kC: per CTA, the largest squared cosine it rotated (float bits)
   int* rank = lflag + kC;                      // 4 nbl
   __shared__ int wflag;
   __shared__ float wmax;
@@ -151,17 +153,23 @@ jacobi_rows_cluster_kernel(const JacobiJob* __restrict__ jobs, float tol) {
           if constexpr (kC == 1) ref[a] = in ? row * ld : 4 * nbl * ld;
           else ref[a] = in ? row_ptr(row) : zrow;
         }
+        const bool full = (r == 32 * kEL);       // every lane element exists: no per-element checks
 #pragma unroll
         for (int a = 0; a < 8; ++a) {
           const float* rp = at(a);
           nn[a] = rp[r];
+          if (full) {
 #pragma unroll
-          for (int e = 0; e < kEL; ++e) {
-            const int t = lane + 32 * e;
-            x[a][e] = (t < r) ? rp[t] : 0.f;
+            for (int e = 0; e < kEL; ++e) x[a][e] = rp[lane + 32 * e];
+          } else {
+#pragma unroll
+            for (int e = 0; e < kEL; ++e) {
+              const int t = lane + 32 * e;
+              x[a][e] = (t < r) ? rp[t] : 0.f;
+            }
           }
         }
-        bool counted = false;
+        unsigned counted = 0u;                  // largest squared cosine among the pairs rotated here (float bits)
 #pragma unroll
         for (int stp = 0; stp < 7; ++stp) {     // fully unrolled: every register index below is a constant
           if (stp >= 4 && round != 0) break;
@@ -189,13 +197,24 @@ jacobi_rows_cluster_kernel(const JacobiJob* __restrict__ jobs, float tol) {
                   for (int e = 0; e < kEL; ++e) g[u] = fmaf(x[a][e], x[bb][e], g[u]);
                 }
           }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u) g[u] += __shfl_xor_sync(0xffffffffu, g[u], o);
+          // four sums across the warp in 6 shuffles: each exchange halves what a lane still carries
+          // (two of the four values after the first, one after the second); the lanes of octet u
+          // (lanes 8u .. 8u+7) end up with the whole of g[u]
+          float gsum;
+          {
+            const bool h16 = (lane & 16) != 0, h8 = (lane & 8) != 0;
+            float k0 = h16 ? g[2] : g[0], k1 = h16 ? g[3] : g[1];
+            const float s0 = h16 ? g[0] : g[2], s1 = h16 ? g[1] : g[3];
+            k0 += __shfl_xor_sync(0xffffffffu, s0, 16);
+            k1 += __shfl_xor_sync(0xffffffffu, s1, 16);
+            gsum = h8 ? k1 : k0;
+            const float sd = h8 ? k0 : k1;
+            gsum += __shfl_xor_sync(0xffffffffu, sd, 8);
+            gsum += __shfl_xor_sync(0xffffffffu, gsum, 4);
+            gsum += __shfl_xor_sync(0xffffffffu, gsum, 2);
+            gsum += __shfl_xor_sync(0xffffffffu, gsum, 1);
           }
-          // rotation parameters: lane u (u < 4) works out pair u, then the results are broadcast --
-          // the parameter arithmetic would otherwise be repeated by all 32 lanes for all 4 pairs
+          // rotation parameters: the lanes of octet u work out pair u, then the results are broadcast
           float appv[4], aqqv[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
@@ -203,8 +222,8 @@ jacobi_rows_cluster_kernel(const JacobiJob* __restrict__ jobs, float tol) {
 #pragma unroll
             for (int a = 0; a < 8; ++a) { if (a == pa[u]) appv[u] = nn[a]; if (a == pb[u]) aqqv[u] = nn[a]; }
           }
-          const int lu = lane & 3;
-          const float my_g = lu == 0 ? g[0] : lu == 1 ? g[1] : lu == 2 ? g[2] : g[3];
+          const int lu = lane >> 3;
+          const float my_g = gsum;
           const float my_app = lu == 0 ? appv[0] : lu == 1 ? appv[1] : lu == 2 ? appv[2] : appv[3];
           const float my_aqq = lu == 0 ? aqqv[0] : lu == 1 ? aqqv[1] : lu == 2 ? aqqv[2] : aqqv[3];
           const bool my_act = my_app > dead2 && my_aqq > dead2 && my_app > 0.f && my_aqq > 0.f &&
@@ -220,12 +239,13 @@ jacobi_rows_cluster_kernel(const JacobiJob* __restrict__ jobs, float tol) {
             my_dn = t1 * my_g;
           }
           const bool my_counted = my_act && my_app > count2 && my_aqq > count2;
-          if (__any_sync(0xffffffffu, my_counted)) counted = true;
+          const float my_cos2 = my_counted ? __fdividef(my_g * my_g, my_app * my_aqq) : 0.f;
+          counted = max(counted, __reduce_max_sync(0xffffffffu, __float_as_uint(my_cos2)));
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
-            c[u] = __shfl_sync(0xffffffffu, my_c, u);
-            sn[u] = __shfl_sync(0xffffffffu, my_s, u);
-            const float dn = __shfl_sync(0xffffffffu, my_dn, u);
+            c[u] = __shfl_sync(0xffffffffu, my_c, 8 * u);
+            sn[u] = __shfl_sync(0xffffffffu, my_s, 8 * u);
+            const float dn = __shfl_sync(0xffffffffu, my_dn, 8 * u);
 #pragma unroll
             for (int a = 0; a < 8; ++a) { if (a == pa[u]) nn[a] = appv[u] - dn; if (a == pb[u]) nn[a] = aqqv[u] + dn; }
           }
@@ -248,14 +268,19 @@ jacobi_rows_cluster_kernel(const JacobiJob* __restrict__ jobs, float tol) {
 #pragma unroll
         for (int a = 0; a < 8; ++a) {
           float* rp = at(a);
+          if (full) {
 #pragma unroll
-          for (int e = 0; e < kEL; ++e) {
-            const int t = lane + 32 * e;
-            if (t < r) rp[t] = x[a][e];
+            for (int e = 0; e < kEL; ++e) rp[lane + 32 * e] = x[a][e];
+          } else {
+#pragma unroll
+            for (int e = 0; e < kEL; ++e) {
+              const int t = lane + 32 * e;
+              if (t < r) rp[t] = x[a][e];
+            }
           }
           if (lane == 0) rp[r] = nn[a];
         }
-        if (lane == 0 && counted) wflag = 1;
+        if (lane == 0 && counted) atomicMax(&wflag, (int)counted);
       }
       csync();                          // all rows of this round are back in place
     }
@@ -266,8 +291,11 @@ jacobi_rows_cluster_kernel(const JacobiJob* __restrict__ jobs, float tol) {
     csync();
     int any = 0;
 #pragma unroll
-    for (int c = 0; c < kC; ++c) any |= lflag[c];
-    converged = (any == 0);
+    for (int c = 0; c < kC; ++c) any = max(any, lflag[c]);
+    converged = (__int_as_float(any) <= kJEarly2);     // nothing rotated, or only by angles whose square is noise
+#ifdef AB_TRACE_SWEEPS
+    if (crank == 0 && tid == 0) printf("  job %d sweep %d: largest rotated cos^2 %.3e\n", (int)(blockIdx.x / kC), sweeps, __int_as_float(any));
+#endif
   }
 
   // norms, descending order, unit rows: each CTA finishes the rows it holds
