@@ -362,6 +362,59 @@ def test_group_sync_factored_truncated_factors_and_bf16(ab):
         assert np.linalg.norm(host(A_out[0]) @ host(B_out[0]) - W) / np.linalg.norm(W) <= tol
 
 
+def _factored_case(seed, m, n, r, K):
+    st = synth.streams(seed, ["AB"])
+    sig = np.exp(-np.arange(r) / max(8.0, r / 3.0))           # sigma_min about 5 % of sigma_max
+    A, B = synth.planted_factors(st["AB"], m, n, sig)
+    ea, eb = synth.group_noise(seed, K, (m, r), (r, n))
+    return synth.group_copies(A, ea), synth.group_copies(B, eb)
+
+
+@pytest.mark.parametrize("m,n,r,K,count", [
+    (70, 45, 10, 3, 1),       # nothing aligned, odd number of row blocks, one CTA per matrix
+    (100, 60, 24, 2, 3),      # ranks that are not multiples of 32
+    (200, 136, 64, 4, 2),     # 2 register elements per lane, clusters of 4 CTAs
+    (160, 320, 96, 4, 2),     # 4 elements, clusters of 4
+    (384, 256, 128, 2, 2),    # 4 elements, clusters of 8
+    (256, 300, 224, 2, 1),    # 8 elements, clusters of 8
+    (96, 80, 64, 2, 40),      # more matrices than clusters fit: one CTA per matrix
+])
+def test_group_sync_factored_shapes(ab, m, n, r, K, count):
+    """The factored route over the shapes that pick its different kernels (register elements per lane,
+    cluster width, vector and scalar load paths, ragged tiles), against the checker's own sync."""
+    cases = [_factored_case(100 * r + i, m, n, r, K) for i in range(min(count, 3))]
+    Aks = [cases[i % len(cases)][0] for i in range(count)]
+    Bks = [cases[i % len(cases)][1] for i in range(count)]
+    devs = [(dev(a), dev(b)) for a, b in cases]
+    plan = ab.SyncPlan([devs[i % len(cases)][0] for i in range(count)], [devs[i % len(cases)][1] for i in range(count)],
+                       0.1, want_W=True)
+    A_out, B_out, sigma, r_out, status = ab.ab_group_sync(plan, path=ab.AB_SYNC_FACTORED)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(status) == 0
+    for i in range(count):
+        if i >= len(cases):                     # repeats of a recipe must give the same bits
+            j = i % len(cases)
+            assert torch.equal(A_out[i], A_out[j]) and torch.equal(B_out[i], B_out[j]) and torch.equal(sigma[i], sigma[j])
+            continue
+        Abar, Bbar = orc.group_average_f32(Aks[i]), orc.group_average_f32(Bks[i])
+        ref = orc.group_sync(Abar[None], Bbar[None], r, 0.1)
+        s = ref["sigma"]
+        assert orc.rel_frob(host(plan.W_out[i]), ref["W"]) <= 1e-6
+        r_gpu = int(r_out[i].item())
+        near = np.any(np.abs(s[:r] - 0.1 * s[0]) <= 1e-3 * s[0])
+        assert abs(r_gpu - ref["r"]) <= (1 if near else 0), (i, r_gpu, ref["r"])
+        k = min(r_gpu, ref["r"])
+        sg = host(sigma[i])
+        assert np.all(np.abs(sg[:k] - s[:k]) <= 1e-4 * s[:k])
+        U, s2, Vt = np.linalg.svd(ref["W"], full_matrices=False)
+        Wr = (U[:, :r_gpu] * s2[:r_gpu]) @ Vt[:r_gpu]
+        Ah, Bh = host(A_out[i]), host(B_out[i])
+        assert np.linalg.norm(Ah @ Bh - Wr) / np.linalg.norm(ref["W"]) <= 1e-4
+        assert np.count_nonzero(Ah[:, r_gpu:]) == 0 and np.count_nonzero(Bh[r_gpu:]) == 0
+        bal = np.linalg.norm(Ah[:, :r_gpu].T @ Ah[:, :r_gpu] - np.diag(sg[:r_gpu])) / s[0]
+        assert bal <= 1e-3, (i, bal)
+
+
 # ------------------------------------------------------------------ full-size workloads
 
 def _oracle_backward_chunked(x, dY, A, B, rows=8192):
