@@ -202,7 +202,9 @@ def vit_model_sync(ab, torch, steps=5):
     def ev():
         return torch.cuda.Event(enable_timing=True)
     res = {}
-    for name, fn in (("mean", lambda: ab.ab_group_average(arena, out=mean_out)), ("sync", lambda: ab.ab_group_sync(plan))):
+    plan_now = ab.SyncPlan([v[0] for v in views], [v[1] for v in views], 0.1, want_W=False, strided=True)
+    for name, fn in (("mean", lambda: ab.ab_group_average(arena, out=mean_out)), ("sync", lambda: ab.ab_group_sync(plan)),
+                     ("sync_now", lambda: ab.ab_group_sync(plan_now))):
         for _ in range(2):
             fn()
         torch.cuda.synchronize()
@@ -217,10 +219,54 @@ def vit_model_sync(ab, torch, steps=5):
     pk = measured_peaks()
     mean_bytes = (K + 1) * 4.0 * total
     return dict(workload="vit_b16_full_sync_72_matrices_fp32_K8_cutoff0.1", ms_per_model=res["sync"],
+                ms_per_model_without_W=res["sync_now"], ms_per_matrix=res["sync"] / len(shapes),
                 mean_ms=res["mean"], mean_gbs=mean_bytes / (res["mean"] * 1e-3) / 1e9,
                 mean_frac_of_measured_hbm=mean_bytes / (res["mean"] * 1e-3) / 1e9 / pk["hbm"],
                 mean_frac_of_nominal_8tbs=mean_bytes / (res["mean"] * 1e-3) / 1e9 / 8000.0,
                 kept_ranks=sorted(set(plan.r_out.tolist())), device_status_errors=bad)
+
+
+def backward_variants(ab, torch, layers, N, iters=10):
+    """The two frozen-factor steps of the method on the same workload: a B-group trains B (forward, then
+    dT, dX and dB; A frozen, no dA), an A-group trains A (forward with T kept, then dA only -- its dX is
+    counted with the B-side variant of the layer below in a real model, and is not computed here).
+    Returns ms per step (both layers) and the algorithmic TFLOP/s of what each variant computes."""
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def b_group():
+        for L in layers:
+            g = L["g"]
+            ab.ab_layer_forward(g["x"], g["A"], g["B"], y=g["y"], ws=g["ws_f"])
+            ab.ab_layer_backward(g["x"], g["dY"], g["A"], g["B"], want=("dX", "dB"), dX=g["dX"], dB=g["dB"], ws=g["ws_b"])
+
+    def a_group():
+        for L in layers:
+            g = L["g"]
+            ab.ab_layer_forward(g["x"], g["A"], g["B"], y=g["y"], T_save=g["T"], ws=g["ws_f"])
+            ab.ab_layer_backward(g["x"], g["dY"], g["A"], g["B"], T_saved=g["T"], want=("dA",), dA=g["dA"], ws=g["ws_b"])
+
+    out = {}
+    for name, fn in (("b_group", b_group), ("a_group", a_group)):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = ev(), ev()
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        flop = 0.0
+        for L in layers:
+            m, r = L["g"]["A"].shape
+            n = L["g"]["B"].shape[1]
+            fwd = 2.0 * N * r * (m + n)
+            flop += fwd + (2.0 * N * r * (m + n) + 2.0 * N * r * n if name == "b_group" else 2.0 * N * r * m)
+        out[name] = dict(ms_per_step=ms, tflops=flop / (ms * 1e-3) / 1e12,
+                         computes="forward, dT, dX, dB" if name == "b_group" else "forward (T kept), dA")
+    return out
 
 
 def run_ours(args):
@@ -378,6 +424,8 @@ def run_ours(args):
                     e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                              ms_per_step=e2e_ms / K),
                     gpu_launches=int(launches), clocks=sampler.summary(), roofline=roof)
+        if world == 1:
+            line["frozen_factor_variants"] = backward_variants(ab, torch, layers, N)
         if world == 1 and not args.no_model_sync:
             del layers, plan
             torch.cuda.empty_cache()
@@ -394,7 +442,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=256 * 197, help="token rows per layer (default: batch 256 x 197)")
     ap.add_argument("--ref-rows", type=int, default=8192, help="rows of the CPU checker's bounded sample")

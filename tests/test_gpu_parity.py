@@ -463,6 +463,22 @@ def test_full_size_vit_mlp(ab, layer):
     _full_size_chain(ab, synth.vit_mlp(layer, seed=1, N=256 * 197, K=1))
 
 
+def test_full_size_frozen_factor_variants(ab):
+    """The steps of an A-group (dA only) and of a B-group (dX and dB, no dA) at the benchmark's size give
+    the bits of the full backward, which the test above holds against the checker."""
+    d = synth.vit_mlp(1, seed=1, N=256 * 197, K=1)
+    x, dY, A, B = (dev(d[k], True) for k in ("x", "dY", "A", "B"))
+    y, T = ab.ab_layer_forward(x, A, B, save_T=True)
+    full = ab.ab_layer_backward(x, dY, A, B, T_saved=T)
+    b_group = ab.ab_layer_backward(x, dY, A, B, want=("dX", "dB"))
+    a_group = ab.ab_layer_backward(x, dY, A, B, T_saved=T, want=("dA",))
+    a_group_recomputed = ab.ab_layer_backward(x, dY, A, B, want=("dA",))       # T rebuilt from x
+    torch.cuda.synchronize()
+    assert b_group[1] is None and a_group[0] is None and a_group[2] is None
+    assert torch.equal(full[0], b_group[0]) and torch.equal(full[2], b_group[2])
+    assert torch.equal(full[1], a_group[1]) and torch.equal(full[1], a_group_recomputed[1])
+
+
 def test_full_size_resnet_conv(ab):
     """ResNet-50 layer3 3x3 convolution as GEMM, 25,088 im2col rows, rank 128, then the rank-truncation
     split of the recombined W."""
