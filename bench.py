@@ -226,6 +226,76 @@ def vit_model_sync(ab, torch, steps=5):
                 kept_ranks=sorted(set(plan.r_out.tolist())), device_status_errors=bad)
 
 
+def other_workloads(ab, torch, iters=10):
+    """The remaining layer shapes of the evaluation, one line each: forward + backward (dX, dA, dB) of one
+    factorised layer, event-timed after warm-up, with the algorithmic FLOP and the minimum HBM bytes
+    (each activation once: x twice, dY, y, dX) and the ceiling those give: min(tensor peak, intensity x HBM
+    peak).  ResNet-50 layer3 3x3 conv as GEMM on materialised im2col rows; VGG16 512 x 4608 at ranks 8..64
+    (the skinny, HBM-bound regime); the small fp32 layer (launch-latency bound, reported in us)."""
+    from paper_2405_01067_b200 import synth
+    pk = measured_peaks()
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = ev(), ev()
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    def layer(d, bf16):
+        dt = torch.bfloat16 if bf16 else torch.float32
+        g = {k: torch.from_numpy(np.ascontiguousarray(d[k], dtype=np.float32)).to(dt).cuda() for k in ("x", "dY", "A", "B")}
+        N, n = g["x"].shape
+        m, r = g["A"].shape
+        code = ab.AB_BF16 if bf16 else ab.AB_F32
+        ws_f = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_FORWARD, N, m, n, r, 1, code), "cuda")
+        ws_b = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_BACKWARD, N, m, n, r, 1, code), "cuda")
+        y = torch.empty((N, m), dtype=dt, device="cuda")
+        T = torch.empty((N, r), dtype=dt, device="cuda")
+        dX = torch.empty((N, n), dtype=dt, device="cuda")
+        dA = torch.empty((m, r), dtype=torch.float32, device="cuda")
+        dB = torch.empty((r, n), dtype=torch.float32, device="cuda")
+
+        def fn():
+            ab.ab_layer_forward(g["x"], g["A"], g["B"], y=y, T_save=T, ws=ws_f)
+            ab.ab_layer_backward(g["x"], g["dY"], g["A"], g["B"], T_saved=T, dX=dX, dA=dA, dB=dB, ws=ws_b)
+        ms = timed(fn)
+        flop = 6.0 * N * r * (m + n)
+        nbytes = (2.0 if bf16 else 4.0) * N * (3 * n + 2 * m)
+        tf = flop / (ms * 1e-3) / 1e12
+        ceil_tf = min(pk["tc_sustained"], flop / nbytes * pk["hbm"] / 1e3)
+        return dict(N=N, m=m, n=n, r=r, ms=ms, tflops=tf, algorithmic_gbs=nbytes / (ms * 1e-3) / 1e9,
+                    ceiling_tflops=ceil_tf, frac_of_ceiling=tf / ceil_tf,
+                    bound="hbm" if ceil_tf < pk["tc_sustained"] else "tensor")
+
+    out = {}
+    d = synth.resnet_conv(2)
+    out["resnet50_layer3_conv3x3_r128"] = layer(d, True)
+    A32, B32 = torch.from_numpy(d["A"]).cuda(), torch.from_numpy(d["B"]).cuda()
+    W = ab.ab_recombine(A32, B32)
+    ms = timed(lambda: ab.ab_svd_split(W, d["r"], 0.0))
+    out["resnet50_layer3_conv3x3_r128"]["recombined_W_split_ms"] = ms
+    del d, A32, B32, W
+    out["vgg16_512x4608"] = {}
+    for r in (8, 16, 32, 64):
+        out["vgg16_512x4608"][f"r{r}"] = layer(synth.vgg_conv(r, 4), True)
+        torch.cuda.empty_cache()
+    d = synth.linear_fp32(0)
+    A, B, _, _, _ = ab.ab_svd_split(torch.from_numpy(d["W"]).cuda(), d["r"], 0.0)   # its factors are the split of its W
+    d["A"], d["B"] = A.cpu().numpy(), B.cpu().numpy()
+    one = layer(d, False)
+    out["linear_256x512_fp32_r32"] = dict(N=one["N"], us_fwd_bwd=one["ms"] * 1e3, note="launch-latency bound")
+    return out
+
+
 def backward_variants(ab, torch, layers, N, iters=10):
     """The two frozen-factor steps of the method on the same workload: a B-group trains B (forward, then
     dT, dX and dB; A frozen, no dA), an A-group trains A (forward with T kept, then dA only -- its dX is
@@ -430,6 +500,8 @@ def run_ours(args):
             del layers, plan
             torch.cuda.empty_cache()
             line["group_sync_model"] = vit_model_sync(ab, torch)
+        if world == 1 and not args.no_other_workloads:
+            line["other_workloads"] = other_workloads(ab, torch)
         if world == 1 and not args.no_cpu_baseline:
             cb = cpu_baseline(inputs, min(N, args.ref_rows))
             line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
@@ -448,6 +520,8 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=8192, help="rows of the CPU checker's bounded sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-model-sync", action="store_true", help="skip the full-ViT group-sync measurement")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the ResNet-50 / VGG16 / small fp32 layer measurements")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

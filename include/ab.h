@@ -70,7 +70,7 @@ size_t ab_workspace_bytes(int op, int64_t N, int m, int n, int r, int K, int dt)
  *   x [N,n], A [m,r] (row stride ldA >= r), B [r,n] (row stride ldB >= n), y [N,m], all of
  *   storage type dt.  T_save: NULL, or [N,r] of type dt that receives T = x B^T for the
  *   backward call.  The rank-r intermediate stays on chip when dt = AB_BF16, r is a
- *   multiple of 16 with 16 <= r <= 256 and m, n are multiples of 8; other shapes take a
+ *   multiple of 8 with 8 <= r <= 256 and m, n are multiples of 8; other shapes take a
  *   slower general kernel (same results to rounding).  N = 0 is a no-op.
  *   Device status: the first int of ws receives AB_OK, or AB_ERR_TIMEOUT if a bounded
  *   on-chip wait of the fused kernel expired (outputs are then undefined).  The same holds

@@ -424,15 +424,19 @@ grad_kernel(const __grid_constant__ CUtensorMap tmAct0, const __grid_constant__ 
 //   blocks [nA, ..): dB[j][q]  = sum_s pB[s][q][j]            (32 x 32 tiles transposed through shared memory)
 __global__ void __launch_bounds__(256)
 reduce_partials_kernel(const float* __restrict__ pA, float* __restrict__ dA, int PA, int nA,
-                       const float* __restrict__ pB, float* __restrict__ dB, int PB, int slices, int r) {
+                       const float* __restrict__ pB, float* __restrict__ dB, int PB, int slices, int r, int rp) {
+  // r: columns of the results; rp: row length of the partials (r rounded up to 16)
   if ((int)blockIdx.x < nA) {
     const int64_t total4 = (int64_t)PA * r / 4;
     const int64_t i4 = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (i4 >= total4) return;
-    const float4* src = reinterpret_cast<const float4*>(pA) + i4;
-    float4 acc = src[0];
+    const int64_t prow = (i4 * 4) / r;
+    const int col = (int)((i4 * 4) % r);
+    const float* src = pA + prow * rp + col;
+    const int64_t slice_stride = (int64_t)PA * rp;
+    float4 acc = *reinterpret_cast<const float4*>(src);
     for (int s = 1; s < slices; ++s) {
-      const float4 v = src[(int64_t)s * total4];
+      const float4 v = *reinterpret_cast<const float4*>(src + s * slice_stride);
       acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
     }
     reinterpret_cast<float4*>(dA)[i4] = acc;
@@ -447,7 +451,7 @@ reduce_partials_kernel(const float* __restrict__ pA, float* __restrict__ dA, int
     const int q = q0 + i, j = j0 + tx;
     float acc = 0.f;
     if (q < PB && j < r)
-      for (int s = 0; s < slices; ++s) acc += pB[((int64_t)s * PB + q) * r + j];
+      for (int s = 0; s < slices; ++s) acc += pB[((int64_t)s * PB + q) * rp + j];
     tile[i][tx] = acc;
   }
   __syncthreads();
@@ -531,7 +535,11 @@ int make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint
 }
 
 struct RowPlan { int natoms, ns, slot_bytes, ns2; size_t smem; };
-RowPlan row_plan(int r) {
+// Ranks that are multiples of 8 but not of 16 run as the next multiple of 16: the tensor maps keep the
+// true extents, so the extra rows / columns of every factor tile arrive as zeros.
+int pad16(int r) { return (r + 15) & ~15; }
+
+RowPlan row_plan(int r) {      // r: padded rank
   RowPlan pl;
   pl.natoms = (r + 63) / 64;
   pl.slot_bytes = kAtomBytes + r * 128;
@@ -574,8 +582,8 @@ BwdWs bwd_ws(void* ws, int64_t N, int m, int n, int r) {
   w.Bt = ar.take_n<bf16>((size_t)n * r);
   w.T = ar.take_n<bf16>((size_t)N * r);
   w.dT = ar.take_n<bf16>((size_t)N * r);
-  w.pA = ar.take_n<float>((size_t)gp.slices * m * r);
-  w.pB = ar.take_n<float>((size_t)gp.slices * n * r);
+  w.pA = ar.take_n<float>((size_t)gp.slices * m * pad16(r));
+  w.pB = ar.take_n<float>((size_t)gp.slices * n * pad16(r));
   w.bytes = align_up(ar.used, 256);
   return w;
 }
@@ -583,11 +591,12 @@ BwdWs bwd_ws(void* ws, int64_t N, int m, int n, int r) {
 // S = In F1^T (saved to Sg if not null), Out = S F2^T (skipped if Out is null)
 int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1, const void* F2, int ldF2, int P,
                      void* Out, void* Sg, int r, int* status, cudaStream_t st) {
-  RowPlan pl = row_plan(r);
+  const int rp = pad16(r);
+  RowPlan pl = row_plan(rp);
   if (pl.ns < 2 || pl.ns2 < 2) return AB_ERR_UNSUPPORTED;
   CUtensorMap tmIn, tmF1, tmF2, tmOut, tmS;
   AB_TRY(make_map(&tmIn, In, (uint64_t)N, K1, K1, 64, 128));
-  AB_TRY(make_map(&tmF1, F1, r, K1, ldF1, 64, r));
+  AB_TRY(make_map(&tmF1, F1, r, K1, ldF1, 64, rp));
   const bool second = Out != nullptr && P > 0;
   // unused maps still have to be valid objects: alias them to the first operand
   if (second) {
@@ -600,7 +609,7 @@ int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1
   if (Sg) AB_TRY(make_map(&tmS, Sg, (uint64_t)N, r, r, 64, 128));
   else tmS = tmIn;
   RowChainParams p;
-  p.K1 = K1; p.P = second ? P : 0; p.r = r; p.nk1 = (K1 + 63) / 64; p.nchunks = second ? (P + kChunk - 1) / kChunk : 0;
+  p.K1 = K1; p.P = second ? P : 0; p.r = rp; p.nk1 = (K1 + 63) / 64; p.nchunks = second ? (P + kChunk - 1) / kChunk : 0;
   p.natoms = pl.natoms; p.ns = pl.ns; p.slot_bytes = pl.slot_bytes; p.ns2 = pl.ns2; p.save_s = Sg ? 1 : 0;
   p.status = status;
   AB_CUDA_OK(cudaFuncSetAttribute(row_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
@@ -615,17 +624,17 @@ int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1
 bool chain_tc_supported(int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
                         const void* x, const void* A, const void* B, const void* y) {
   if (dt != AB_BF16) return false;
-  if (r % 16 != 0 || r < 16 || r > 256) return false;
+  if (r % 8 != 0 || r < 8 || r > 256) return false;
   if (m % 8 != 0 || n % 8 != 0 || ldA % 8 != 0 || ldB % 8 != 0) return false;
   if (N > (int64_t)1 << 30) return false;
   if (!aligned(x, 16) || !aligned(A, 16) || !aligned(B, 16) || !aligned(y, 16)) return false;
   if (!device_is_sm100() || !encode_fn()) return false;
-  return row_plan(r).ns >= 2 && row_plan(r).ns2 >= 2;
+  return row_plan(pad16(r)).ns >= 2 && row_plan(pad16(r)).ns2 >= 2;
 }
 
 size_t chain_tc_forward_ws(int64_t, int, int, int) { return 256; }
 size_t chain_tc_backward_ws(int64_t N, int m, int n, int r) {
-  if (r % 16 != 0 || r < 16 || r > 256) return 0;
+  if (r % 8 != 0 || r < 8 || r > 256) return 0;
   return bwd_ws(nullptr, N, m, n, r).bytes;
 }
 
@@ -668,6 +677,7 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
   }
   if (dA || dB) {
     GradPlan gp = grad_plan(N, m, n, r);
+    const int rp = pad16(r);
     GradParams p;
     CUtensorMap tmAct[2], tmSmall[2];
     int nj = 0;
@@ -684,7 +694,7 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
       ++nj;
     }
     if (nj == 1) { tmAct[1] = tmAct[0]; tmSmall[1] = tmSmall[0]; p.job[1] = p.job[0]; p.job[1].chunks = 0; }
-    p.njobs = nj; p.r = r; p.natoms = gp.natoms; p.ns = gp.ns; p.slot_bytes = gp.slot_bytes;
+    p.njobs = nj; p.r = rp; p.natoms = gp.natoms; p.ns = gp.ns; p.slot_bytes = gp.slot_bytes;
     p.slices = gp.slices; p.rows_per_slice = gp.rows_per_slice; p.N = (int)N; p.status = w.status;
     AB_CUDA_OK(cudaFuncSetAttribute(grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gp.smem));
     const unsigned grid = (unsigned)((p.job[0].chunks + p.job[1].chunks) * gp.slices);
@@ -693,7 +703,7 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
     {
       const int nA = dA ? (int)(((int64_t)m * r / 4 + 255) / 256) : 0;
       const int nB = dB ? ((n + 31) / 32) * ((r + 31) / 32) : 0;
-      reduce_partials_kernel<<<nA + nB, 256, 0, st>>>(w.pA, dA, m, nA, w.pB, dB, n, gp.slices, r);
+      reduce_partials_kernel<<<nA + nB, 256, 0, st>>>(w.pA, dA, m, nA, w.pB, dB, n, gp.slices, r, rp);
       AB_LAUNCH_OK();
     }
   }

@@ -73,7 +73,9 @@ def test_chain_fp32(ab, N, m, n, r, save_T):
 
 @pytest.mark.parametrize("N,m,n,r", [(300, 256, 128, 32), (257, 384, 512, 192), (1000, 768, 256, 256),
                                      (77, 40, 56, 8), (513, 136, 264, 48), (128, 128, 128, 16),
-                                     (640, 512, 1024, 64), (100, 50, 70, 7)])
+                                     (640, 512, 1024, 64), (100, 50, 70, 7),
+                                     # ranks that are multiples of 8 only: the tensor-core chain on a padded rank
+                                     (700, 512, 1152, 8), (300, 264, 200, 24), (515, 328, 384, 72), (260, 256, 512, 200)])
 @pytest.mark.parametrize("save_T", [False, True])
 def test_chain_bf16(ab, N, m, n, r, save_T):
     d = synth.chain_case(200 + N + r, m, n, r, N, bf16=True)
