@@ -118,6 +118,15 @@ size_t svd_batch_ws(const SvdItem* items, int L);
 int svd_batch(const SvdItem* items, int L, float sigma_cutoff, void* ws, size_t ws_bytes, cudaStream_t st);
 
 // ---- factored group sync (ab_sync_fast.cu) ------------------------------------------------------
+// One-sided Jacobi on the rows of `count` s x s matrices (s <= 256) kept in shared memory, one CTA or
+// one cluster of CTAs per matrix (ab_sync_fast.cu).  X: count matrices, s * s apart.  rows: the
+// orthogonalised rows scaled to unit length, sorted by descending norm; norms: those norms.  status:
+// one int per matrix, status_stride_bytes apart (AB_OK / AB_ERR_NOT_CONVERGED).  scratch: device memory
+// of rows_jacobi_scratch_bytes(count).
+bool rows_jacobi_fits(int count, int s);
+size_t rows_jacobi_scratch_bytes(int count);
+int rows_jacobi(const float* X, float* rows, float* norms, int* status, size_t status_stride_bytes, int count, int s,
+                void* scratch, cudaStream_t st);
 bool sync_factored_supported(const ab_sync_desc* d, int L);
 size_t sync_factored_ws(const ab_sync_desc* d, int L);
 int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int dt, int* dev_status,

@@ -362,6 +362,69 @@ norms_sort_kernel(const float* __restrict__ Xall, int s, float* __restrict__ lam
   }
 }
 
+// After the in-shared-memory solver: rows (unit length, sorted by descending lam) whose lam is below
+// 1e-4 of the largest carry directions of rounding noise, not eigenvectors.  Each of them is made
+// orthogonal to every row before it (Gram-Schmidt, two passes) and rescaled, so that the rows stay an
+// orthonormal set and W v picks up nothing of the resolved directions; a row that does not survive the
+// projection becomes zero (it then contributes nothing to either factor).  Only the first r_need rows
+// are ever used.  One CTA per matrix.
+__global__ void __launch_bounds__(256)
+complete_basis_kernel(float* __restrict__ rows_all, const float* __restrict__ lam_all, int s, int r_need) {
+  extern __shared__ float cb_sm[];
+  float* v = cb_sm;            // s
+  float* coef = cb_sm + s;     // s
+  __shared__ float red[8];
+  __shared__ int k_first;
+  float* rows = rows_all + (size_t)blockIdx.x * s * s;
+  const float* lam = lam_all + (size_t)blockIdx.x * s;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    int k = 0;
+    const float thr = 1e-4f * lam[0];
+    while (k < s && lam[k] >= thr && lam[k] > 0.f) ++k;
+    k_first = k;
+  }
+  __syncthreads();
+  const int k_end = r_need < s ? r_need : s;
+  for (int k = k_first; k < k_end; ++k) {
+    for (int u = tid; u < s; u += 256) v[u] = rows[(size_t)k * s + u];
+    __syncthreads();
+    for (int pass = 0; pass < 2; ++pass) {
+      for (int j = warp; j < k; j += 8) {
+        float a = 0.f;
+        for (int u = lane; u < s; u += 32) a = fmaf(rows[(size_t)j * s + u], v[u], a);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if (lane == 0) coef[j] = a;
+      }
+      __syncthreads();
+      for (int u = tid; u < s; u += 256) {
+        float a = v[u];
+        for (int j = 0; j < k; ++j) a = fmaf(-coef[j], rows[(size_t)j * s + u], a);
+        v[u] = a;
+      }
+      __syncthreads();
+    }
+    float a = 0.f;
+    for (int u = tid; u < s; u += 256) a = fmaf(v[u], v[u], a);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (lane == 0) red[warp] = a;
+    __syncthreads();
+    float n2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) n2 += red[i];
+    const float inv = n2 > 1e-6f ? rsqrtf(n2) : 0.f;       // the row started at unit length (or zero)
+    for (int u = tid; u < s; u += 256) rows[(size_t)k * s + u] = v[u] * inv;
+    __syncthreads();                                         // the next row reads this one from global memory
+  }
+}
+
+__global__ void identity_perm_kernel(int* __restrict__ perm, int s, int total) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < total) perm[i] = i % s;
+}
+
 // Vr[k][:] = Vt[perm[k]][:] scaled to unit length, k < r_cap (thousands of fp32 rotations leave
 // the rows orthogonal but let their norms wander by ~1e-6)
 __global__ void __launch_bounds__(256)
@@ -487,6 +550,7 @@ struct Layout {
   std::map<int, std::vector<int>> groups;     // s -> item indices
   std::map<int, float*> X, Vt;
   std::map<int, JState*> st;
+  std::map<int, void*> jobs;                  // scratch of the in-shared-memory solver
   std::vector<ItemWs> item;
   size_t bytes;
 };
@@ -500,6 +564,7 @@ Layout make_layout(const SvdItem* items, int L, void* ws) {
     lo.X[g.first] = ar.take_n<float>(cnt * s * s);
     lo.Vt[g.first] = ar.take_n<float>(cnt * s * s);
     lo.st[g.first] = ar.take_n<JState>(cnt);
+    lo.jobs[g.first] = ar.take_n<char>(rows_jacobi_scratch_bytes((int)cnt));
   }
   lo.item.resize(L);
   for (int i = 0; i < L; ++i) {
@@ -568,6 +633,21 @@ int svd_batch(const SvdItem* items, int L, float sigma_cutoff, void* ws, size_t 
   for (auto& g : lo.groups) {
     const int s = g.first, count = (int)g.second.size();
     Plan p = make_plan(items[g.second[0]]);
+    if (rows_jacobi_fits(count, s)) {
+      // small enough to stay in shared memory for the whole iteration: the rows of G rotated until
+      // orthogonal are lambda_i v_i^T, so the unit rows are the eigenvectors, already sorted
+      AB_CUDA_OK(cudaMemsetAsync(lo.st[s], 0, sizeof(JState) * count, stream));
+      AB_TRY(rows_jacobi(lo.X[s], lo.Vt[s], lo.item[g.second[0]].lam, &lo.st[s]->status, sizeof(JState), count, s,
+                         lo.jobs[s], stream));
+      int r_need = 0;
+      for (int idx : g.second) r_need = std::max(r_need, make_plan(items[idx]).r_cap);
+      complete_basis_kernel<<<count, 256, 2 * (size_t)s * sizeof(float), stream>>>(lo.Vt[s], lo.item[g.second[0]].lam, s,
+                                                                                  r_need);
+      AB_LAUNCH_OK();
+      identity_perm_kernel<<<(count * s + 255) / 256, 256, 0, stream>>>(lo.item[g.second[0]].perm, s, count * s);
+      AB_LAUNCH_OK();
+      continue;
+    }
     dim3 ig(64, (unsigned)count);
     init_state_kernel<<<ig, 256, 0, stream>>>(lo.Vt[s], lo.st[s], s, count);
     AB_LAUNCH_OK();

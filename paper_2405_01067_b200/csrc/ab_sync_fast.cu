@@ -379,6 +379,10 @@ int launch_jacobi_el(const JacobiJob* jobs, int count, int rmax, float tol, cuda
   int s = try_launch_jacobi<EL, 8>(jobs, count, rmax, tol, st);
   if (s == 1) s = try_launch_jacobi<EL, 4>(jobs, count, rmax, tol, st);
   if (s == 1) s = try_launch_jacobi<EL, 1>(jobs, count, rmax, tol, st);
+  if (s == AB_ERR_UNSUPPORTED) {            // too large for one CTA's shared memory: two CTAs hold half each
+    s = try_launch_jacobi<EL, 2>(jobs, count, rmax, tol, st);
+    if (s == 1) s = AB_ERR_UNSUPPORTED;
+  }
   return s;
 }
 int launch_jacobi(const JacobiJob* jobs, int count, int rmax, float tol, cudaStream_t st) {
@@ -567,6 +571,31 @@ GemmDesc mk(const float* A, int64_t sAm, int64_t sAk, const float* B, int64_t sB
 
 }  // namespace
 
+float rows_jacobi_tol(int s) { return 5e-7f * sqrtf((float)s) < 4e-6f ? 4e-6f : 5e-7f * sqrtf((float)s); }
+
+bool rows_jacobi_fits(int count, int s) {
+  if (s < 1 || s > 256 || count < 1) return false;
+  if (jacobi_smem_bytes(s, s, 1) <= 227 * 1024 - 256) return true;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return false;
+  return (long long)count * 2 <= sms && s >= 32;
+}
+
+size_t rows_jacobi_scratch_bytes(int count) { return align_up((size_t)count * sizeof(JacobiJob), 256); }
+
+int rows_jacobi(const float* X, float* rows, float* norms, int* status, size_t status_stride_bytes, int count, int s,
+                void* scratch, cudaStream_t st) {
+  std::vector<JacobiJob> jb((size_t)count);
+  for (int j = 0; j < count; ++j) {
+    int* stj = reinterpret_cast<int*>(reinterpret_cast<char*>(status) + (size_t)j * status_stride_bytes);
+    jb[j] = JacobiJob{X + (size_t)j * s * s, rows + (size_t)j * s * s, norms + (size_t)j * s, stj, s, s};
+  }
+  AB_CUDA_OK(cudaMemcpyAsync(scratch, jb.data(), jb.size() * sizeof(JacobiJob), cudaMemcpyHostToDevice, st));
+  return launch_jacobi(static_cast<const JacobiJob*>(scratch), count, s, rows_jacobi_tol(s), st);
+}
+
 bool sync_factored_supported(const ab_sync_desc* d, int L) {
   // dynamic shared memory of the two single-CTA kernels, with room for their few static words
   const size_t cap = 227 * 1024 - 256;
@@ -662,7 +691,7 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
     AB_CUDA_OK(cudaMemcpyAsync(w.ajobs, aj.data(), aj.size() * sizeof(AvgJob), cudaMemcpyHostToDevice, st));
     AB_TRY(group_average_batched(w.ajobs, 2 * L, K, dt, longest, st));
   }
-  const float tol = 5e-7f * sqrtf((float)rmax) < 4e-6f ? 4e-6f : 5e-7f * sqrtf((float)rmax);
+  const float tol = rows_jacobi_tol(rmax);
   bool any_w = false;
   for (int i = 0; i < L; ++i) any_w = any_w || d[i].W_out != nullptr;
   if (any_w) AB_TRY(gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, st));                 // a8 (optional)
