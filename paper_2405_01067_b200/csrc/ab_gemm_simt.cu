@@ -1,7 +1,7 @@
 // Strided GEMMs on the fp32 pipes: the path for fp32 storage (where a reduced-precision
 // tensor-core pass would miss the 1e-4 bound) and for shapes the fused tensor-core chain does
 // not take.  Two kernels:
-//  - gemm_simt_kernel: any mix of fp32 / bf16 operands.  64x64 output tile per CTA, 16-deep k
+//  - gemm_simt_kernel: any mix of fp32 / bf16 operands (all-fp32 problems go to the second kernel).  64x64 output tile per CTA, 16-deep k
 //    slabs staged in shared memory, 4x4 accumulators per thread.  Each 16-term partial dot
 //    product is formed in fp32 and added to a running fp64 sum, so long reductions keep ~1e-7
 //    relative accuracy; the order of additions is fixed by the shape alone.
@@ -183,10 +183,8 @@ struct TileIo {
 };
 
 template <int BM_, int BN_>
-__global__ void __launch_bounds__((BM_ / 8) * (BN_ / 8), 512 / ((BM_ / 8) * (BN_ / 8)))
-gemm_simt_batched_kernel(const GemmDesc* __restrict__ descs) {
+__device__ __forceinline__ void gemm_tile_8x8(const GemmDesc& d) {
   constexpr int NT = (BM_ / 8) * (BN_ / 8);
-  const GemmDesc d = descs[blockIdx.z];
   const int64_t m0 = (int64_t)blockIdx.y * BM_, n0 = (int64_t)blockIdx.x * BN_;
   if (m0 >= d.M || n0 >= d.N) return;
   if (d.upper_only && n0 + BN_ <= m0) return;
@@ -281,6 +279,29 @@ gemm_simt_batched_kernel(const GemmDesc* __restrict__ descs) {
 }
 
 template <int BM_, int BN_>
+__global__ void __launch_bounds__((BM_ / 8) * (BN_ / 8), 512 / ((BM_ / 8) * (BN_ / 8)))
+gemm_simt_batched_kernel(const GemmDesc* __restrict__ descs) {
+  const GemmDesc d = descs[blockIdx.z];
+  gemm_tile_8x8<BM_, BN_>(d);
+}
+
+// The same tile code for one problem whose descriptor travels as a kernel argument.
+template <int BM_, int BN_>
+__global__ void __launch_bounds__((BM_ / 8) * (BN_ / 8), 512 / ((BM_ / 8) * (BN_ / 8)))
+gemm_simt_one_kernel(const __grid_constant__ GemmDesc d) {
+  gemm_tile_8x8<BM_, BN_>(d);
+}
+
+template <int BM_, int BN_>
+int launch_one(const GemmDesc& d, cudaStream_t st) {
+  dim3 grid((unsigned)((d.N + BN_ - 1) / BN_), (unsigned)((d.M + BM_ - 1) / BM_), 1u);
+  if (grid.y > 65535u) return AB_ERR_UNSUPPORTED;
+  gemm_simt_one_kernel<BM_, BN_><<<grid, (BM_ / 8) * (BN_ / 8), 0, st>>>(d);
+  AB_LAUNCH_OK();
+  return AB_OK;
+}
+
+template <int BM_, int BN_>
 int launch_batched(const GemmDesc* d_descs, int count, int max_M, int max_N, cudaStream_t st) {
   dim3 grid((unsigned)((max_N + BN_ - 1) / BN_), (unsigned)((max_M + BM_ - 1) / BM_), (unsigned)count);
   if (grid.y > 65535u || grid.z > 65535u) return AB_ERR_UNSUPPORTED;
@@ -306,6 +327,24 @@ int gemm_simt(const void* A, int a_dt, int64_t sAm, int64_t sAk,
               void* C, int c_dt, int64_t ldc,
               int64_t M, int64_t N, int64_t K, cudaStream_t st) {
   if (M <= 0 || N <= 0) return AB_OK;
+  if (a_dt == AB_F32 && b_dt == AB_F32 && c_dt == AB_F32 && M < ((int64_t)1 << 22) && N < ((int64_t)1 << 31) &&
+      K < ((int64_t)1 << 31)) {
+    // all-fp32 problems take the register-tiled kernel (fp32 sums in ascending k)
+    GemmDesc d;
+    d.A = static_cast<const float*>(A); d.B = static_cast<const float*>(B); d.C = C;
+    d.sAm = sAm; d.sAk = sAk; d.sBk = sBk; d.sBn = sBn; d.ldc = ldc;
+    d.M = (int)M; d.N = (int)N; d.K = (int)K; d.c_bf16 = 0;
+    d.row_vec = d.col_vec = d.k_vec = nullptr;
+    d.row_mode = d.col_mode = d.k_mode = 0;
+    d.thr = 0.f;
+    d.live_rows = d.live_cols = nullptr;
+    d.upper_only = 0;
+    const bool bigM = M >= 512, bigN = N >= 512;
+    if (bigM && bigN) return launch_one<128, 128>(d, st);
+    if (bigM) return launch_one<128, 64>(d, st);
+    if (bigN) return launch_one<64, 128>(d, st);
+    return launch_one<64, 64>(d, st);
+  }
   // rows beyond 65535 tiles are covered by splitting M into bands
   const int64_t band = (int64_t)65535 * BM;
   for (int64_t mo = 0; mo < M; mo += band) {
