@@ -435,6 +435,7 @@ reduce_partials_kernel(const float* __restrict__ pA, float* __restrict__ dA, int
     const float* src = pA + prow * rp + col;
     const int64_t slice_stride = (int64_t)PA * rp;
     float4 acc = *reinterpret_cast<const float4*>(src);
+#pragma unroll 4
     for (int s = 1; s < slices; ++s) {
       const float4 v = *reinterpret_cast<const float4*>(src + s * slice_stride);
       acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
@@ -451,6 +452,7 @@ reduce_partials_kernel(const float* __restrict__ pA, float* __restrict__ dA, int
     const int q = q0 + i, j = j0 + tx;
     float acc = 0.f;
     if (q < PB && j < r)
+#pragma unroll 4
       for (int s = 0; s < slices; ++s) acc += pB[((int64_t)s * PB + q) * rp + j];
     tile[i][tx] = acc;
   }
