@@ -53,7 +53,7 @@ struct RowChainParams {
 struct Bars {
   uint64_t full[kMaxStages], empty[kMaxStages];
   uint64_t full2[kMaxStages2], empty2[kMaxStages2];
-  uint64_t t_full, s_ready;
+  uint64_t t_full, s_ready, unit_done;
   uint64_t acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   int abort_any;   // set by any role that gave up
@@ -280,6 +280,258 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
   __syncthreads();
   if (*reinterpret_cast<volatile int*>(&bars->abort_any)) {
     // give loads that are still in flight time to land before the shared memory is released
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// row_chain_units_kernel: the same chain for many row blocks per CTA.  A persistent CTA owns a
+// contiguous range of 128-row blocks and works through it in units of two blocks (one block when
+// the range is odd).  Both blocks of a unit share every factor tile that is loaded -- each slab of
+// F1 feeds two first-product MMAs, each tile of F2 two second-product MMAs -- so a row costs half
+// the factor bytes; what paces the single-block kernel is exactly those bytes (1.5 MB of factors
+// against 0.2 MB of activations per block at the ViT shapes).  In a two-block unit the two
+// accumulators belong to the two blocks (the epilogue of one overlaps the MMAs of the other); in a
+// one-block unit they alternate between chunks as in row_chain_kernel.
+struct UnitParams {
+  int K1, P, r, nk1, nchunks, natoms;
+  int ns, slot_bytes;      // first product: slots of two 128-row In tiles + one F1 slab
+  int ns2, ring2_bytes;    // second product: 32 KB slots at the start of shared memory
+  int save_s;
+  int tiles;               // 128-row blocks in all
+  int* status;
+};
+
+__global__ void __launch_bounds__(192, 1)
+row_chain_units_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ CUtensorMap tmF1,
+                       const __grid_constant__ CUtensorMap tmF2, const __grid_constant__ CUtensorMap tmOut,
+                       const __grid_constant__ CUtensorMap tmS, const UnitParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // [ second-product ring | S of block 0 | S of block 1 | two staging tiles | barriers ]; the first
+  // product's ring lies over the first three regions, which it has to itself while it runs
+  uint8_t* ring = smem;
+  uint8_t* S0 = smem + p.ring2_bytes;
+  uint8_t* stg = S0 + 2 * p.natoms * kAtomBytes;
+  Bars* bars = reinterpret_cast<Bars*>(stg + 2 * kAtomBytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t_begin = (int)((int64_t)blockIdx.x * p.tiles / gridDim.x);
+  const int t_end = (int)((int64_t)(blockIdx.x + 1) * p.tiles / gridDim.x);
+  const int rot1 = blockIdx.x % p.nk1;
+  const int rot2 = p.nchunks > 0 ? (blockIdx.x * 5) % p.nchunks : 0;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.ns; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
+    for (int i = 0; i < p.ns2; ++i) { mbar_init(&bars->full2[i], 1); mbar_init(&bars->empty2[i], 1); }
+    mbar_init(&bars->t_full, 1);
+    mbar_init(&bars->s_ready, kEpiThreads);
+    mbar_init(&bars->unit_done, 2);             // the MMA issuer's commit and the epilogue's store issuer
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 4); }
+    bars->abort_any = 0;
+    bars->epi_abort = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&tmIn); tma_prefetch_desc(&tmF1); tma_prefetch_desc(&tmF2);
+    tma_prefetch_desc(&tmOut); tma_prefetch_desc(&tmS);
+  }
+  if (warp == 1) tmem_alloc(&bars->tmem_base, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
+  // TMEM: block b of a unit keeps its S accumulator at column 256 b while the first product runs;
+  // accumulator b of the second product takes the same 256 columns afterwards.
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int i1 = 0, i2 = 0, u = 0;
+      bool ok = true;
+      for (int t = t_begin; t < t_end && ok; ++u) {
+        const int nt = (t_end - t >= 2) ? 2 : 1;
+        const int row0 = t * 128;
+        // the shared memory of the last unit is free once its MMAs are done and its stores have been read
+        if (u > 0 && !mbar_wait(&bars->unit_done, (u - 1) & 1)) { raise_timeout(bars, p.status); ok = false; break; }
+        for (int ks = 0; ks < p.nk1 && ok; ++ks, ++i1) {
+          const int slot = i1 % p.ns, ph = (i1 / p.ns) & 1;
+          if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
+          uint8_t* dst = smem + (size_t)slot * p.slot_bytes;
+          mbar_arrive_expect_tx(&bars->full[slot], nt * kAtomBytes + p.r * 128);
+          const int kr = (ks + rot1) % p.nk1;
+          tma_load_2d(dst, &tmIn, &bars->full[slot], kr * 64, row0);
+          if (nt == 2) tma_load_2d(dst + kAtomBytes, &tmIn, &bars->full[slot], kr * 64, row0 + 128);
+          tma_load_2d(dst + 2 * kAtomBytes, &tmF1, &bars->full[slot], kr * 64, 0);
+        }
+        // the second product's slots lie over the first product's: wait until its MMAs have read them
+        if (ok && !mbar_wait(&bars->t_full, u & 1)) { raise_timeout(bars, p.status); ok = false; }
+        for (int c = 0; c < p.nchunks && ok; ++c) {
+          for (int j = 0; j < p.natoms; ++j, ++i2) {
+            const int slot = i2 % p.ns2, ph = (i2 / p.ns2) & 1;
+            if (!mbar_wait(&bars->empty2[slot], ph ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
+            mbar_arrive_expect_tx(&bars->full2[slot], kAtom2Bytes);
+            tma_load_2d(ring + (size_t)slot * kAtom2Bytes, &tmF2, &bars->full2[slot], j * 64,
+                        ((c + rot2) % p.nchunks) * kChunk);
+          }
+        }
+        t += nt;
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc1 = instr_desc_bf16(128, p.r, 0, 0);
+      const uint32_t idesc2 = instr_desc_bf16(128, kChunk, 0, 0);
+      int i1 = 0, i2 = 0, u = 0;
+      int q[2] = {0, 0};                       // uses of each accumulator so far
+      bool ok = true;
+      for (int t = t_begin; t < t_end && ok; ++u) {
+        const int nt = (t_end - t >= 2) ? 2 : 1;
+        for (int ks = 0; ks < p.nk1; ++ks, ++i1) {
+          const int slot = i1 % p.ns, ph = (i1 / p.ns) & 1;
+          if (!mbar_wait(&bars->full[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + (size_t)slot * p.slot_bytes);
+          const uint64_t da0 = smem_desc_sw128(sa, 16), da1 = smem_desc_sw128(sa + kAtomBytes, 16);
+          const uint64_t db = smem_desc_sw128(sa + 2 * kAtomBytes, 16);
+          int ksteps = (p.K1 - ((ks + rot1) % p.nk1) * 64 + 15) >> 4;
+          if (ksteps > 4) ksteps = 4;
+          for (int kk = 0; kk < ksteps; ++kk) {
+            tc_mma_bf16(tmem_base, da0 + 2 * kk, db + 2 * kk, idesc1, (ks | kk) != 0);
+            if (nt == 2) tc_mma_bf16(tmem_base + 256, da1 + 2 * kk, db + 2 * kk, idesc1, (ks | kk) != 0);
+          }
+          tc_commit(&bars->empty[slot]);
+        }
+        if (!ok) break;
+        tc_commit(&bars->t_full);
+        if (p.nchunks > 0) {
+          if (!mbar_wait(&bars->s_ready, u & 1)) { raise_timeout(bars, p.status); ok = false; break; }
+          tc_fence_after();
+        }
+        for (int c = 0; c < p.nchunks && ok; ++c) {
+          for (int tt = 0; tt < nt && ok; ++tt) {
+            const int b = (nt == 2) ? tt : (c & 1);
+            if (!mbar_wait(&bars->acc_empty[b], (q[b] & 1) ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
+            tc_fence_after();
+            const uint32_t tacc = tmem_base + kChunk * b;
+            const uint8_t* Sb = S0 + (size_t)tt * p.natoms * kAtomBytes;
+            for (int j = 0; j < p.natoms; ++j) {
+              const int idx = i2 + j, slot = idx % p.ns2, ph = (idx / p.ns2) & 1;
+              if (!mbar_wait(&bars->full2[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
+              tc_fence_after();
+              const uint64_t da = smem_desc_sw128(smem_u32(Sb + j * kAtomBytes), 16);
+              const uint64_t db = smem_desc_sw128(smem_u32(ring + (size_t)slot * kAtom2Bytes), 16);
+              int ksteps = (p.r - j * 64) >> 4;
+              if (ksteps > 4) ksteps = 4;
+              for (int kk = 0; kk < ksteps; ++kk) tc_mma_bf16(tacc, da + 2 * kk, db + 2 * kk, idesc2, (j | kk) != 0);
+              if (tt == nt - 1) tc_commit(&bars->empty2[slot]);     // the last block of the unit is done with this tile
+            }
+            if (ok) { tc_commit(&bars->acc_full[b]); ++q[b]; }
+          }
+          i2 += p.natoms;
+        }
+        if (ok) tc_commit(&bars->unit_done);
+        t += nt;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int qw = warp & 3;                // TMEM lane quarter this warp may read
+    const int row = qw * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(qw * 32) << 16;
+    const bool issuer = (threadIdx.x == 64);
+    int q[2] = {0, 0};
+    int nstores = 0, u = 0;
+    bool ok = true;
+    for (int t = t_begin; t < t_end && ok; ++u) {
+      const int nt = (t_end - t >= 2) ? 2 : 1;
+      const int row0 = t * 128;
+      ok = epi_wait(bars, &bars->t_full, u & 1, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      for (int tt = 0; tt < nt; ++tt) {
+        uint8_t* Sb = S0 + (size_t)tt * p.natoms * kAtomBytes;
+        for (int c0 = 0; c0 < p.r; c0 += 64) {
+          uint32_t v[4][16];
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            if (c0 + g * 16 < p.r) tmem_ld16_nowait(tmem_base + 256 * tt + lane_base + c0 + g * 16, v[g]);
+          tmem_wait_ld();
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            if (c0 + g * 16 < p.r) store_bf16x16_swizzled(Sb + (c0 >> 6) * kAtomBytes + row * 128, row, c0 + g * 16, v[g]);
+        }
+      }
+      tc_fence_before();
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->s_ready);
+      if (p.save_s) {
+        named_bar_sync(1, kEpiThreads);
+        if (issuer) {
+          for (int tt = 0; tt < nt; ++tt)
+            for (int j = 0; j < p.natoms; ++j)
+              tma_store_2d(&tmS, S0 + ((size_t)tt * p.natoms + j) * kAtomBytes, j * 64, row0 + tt * 128);
+          tma_store_commit();
+        }
+      }
+      for (int c = 0; c < p.nchunks && ok; ++c) {
+        for (int tt = 0; tt < nt && ok; ++tt) {
+          const int b = (nt == 2) ? tt : (c & 1);
+          ok = epi_wait(bars, &bars->acc_full[b], q[b] & 1, p.status);
+          if (!ok) break;
+          ++q[b];
+          tc_fence_after();
+          const uint32_t tacc = tmem_base + kChunk * b + lane_base;
+          for (int h = 0; h < kChunk / 64; ++h) {
+            const int col = ((c + rot2) % p.nchunks) * kChunk + h * 64;
+            const bool live = col < p.P;
+            uint32_t v[4][16];
+            if (live) {
+#pragma unroll
+              for (int g = 0; g < 4; ++g) tmem_ld16_nowait(tacc + h * 64 + g * 16, v[g]);
+              tmem_wait_ld();
+            }
+            if (h == kChunk / 64 - 1) {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&bars->acc_empty[b]);
+            }
+            if (!live) continue;
+            uint8_t* buf = stg + (nstores & 1) * kAtomBytes;
+            ++nstores;
+            if (issuer) tma_store_wait_read<1>();
+            named_bar_sync(1, kEpiThreads);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) store_bf16x16_swizzled(buf + row * 128, row, g * 16, v[g]);
+            fence_proxy_async_smem();
+            named_bar_sync(1, kEpiThreads);
+            if (issuer) {
+              tma_store_2d(&tmOut, buf, col, row0 + tt * 128);
+              tma_store_commit();
+            }
+          }
+        }
+      }
+      // every epilogue thread has passed the last barrier, so all TMEM reads of the unit are done; once
+      // the stores issued so far have read their shared memory the next unit may overwrite S
+      if (issuer && ok) {
+        tma_store_wait_read<0>();
+        mbar_arrive(&bars->unit_done);
+      }
+      t += nt;
+    }
+    if (issuer) tma_store_wait_all();
+  }
+
+  // ------------------------------------------------------------ common exit
+  tc_fence_before();
+  __syncthreads();
+  if (*reinterpret_cast<volatile int*>(&bars->abort_any)) {
     const uint64_t t0 = globaltimer_ns();
     while (globaltimer_ns() - t0 < 200000ull) { }
     __syncthreads();
@@ -554,6 +806,30 @@ RowPlan row_plan(int r) {      // r: padded rank
   return pl;
 }
 
+struct UnitPlan { int natoms, ns, slot_bytes, ns2, ring2_bytes; size_t smem; bool ok; };
+UnitPlan unit_plan(int r) {    // r: padded rank
+  UnitPlan pl;
+  pl.natoms = (r + 63) / 64;
+  pl.slot_bytes = 2 * kAtomBytes + r * 128;
+  const int fixed = 2 * pl.natoms * kAtomBytes + 2 * kAtomBytes + (int)sizeof(Bars) + 1024;
+  pl.ns2 = (kSmemLimit - fixed) / kAtom2Bytes;
+  if (pl.ns2 > kMaxStages2) pl.ns2 = kMaxStages2;
+  pl.ring2_bytes = pl.ns2 > 0 ? pl.ns2 * kAtom2Bytes : 0;
+  pl.ns = (pl.ring2_bytes + 2 * pl.natoms * kAtomBytes) / pl.slot_bytes;
+  if (pl.ns > kMaxStages) pl.ns = kMaxStages;
+  pl.smem = (size_t)fixed + (size_t)pl.ring2_bytes;
+  pl.ok = pl.ns2 >= pl.natoms && pl.ns2 >= 2 && pl.ns >= 2;
+  return pl;
+}
+
+int sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return 0;
+  return sms;
+}
+
 struct GradPlan { int natoms, ns, slot_bytes, slices, rows_per_slice; size_t smem; };
 GradPlan grad_plan(int64_t N, int m, int n, int r) {
   GradPlan pl;
@@ -610,6 +886,23 @@ int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1
   }
   if (Sg) AB_TRY(make_map(&tmS, Sg, (uint64_t)N, r, r, 64, 128));
   else tmS = tmIn;
+  // More row blocks than SMs: persistent CTAs that take two blocks at a time and load each factor
+  // tile once for both.
+  {
+    const int64_t tiles = (N + 127) / 128;
+    const int sms = sm_count();
+    const UnitPlan up = unit_plan(rp);
+    if (second && sms > 0 && tiles > sms && up.ok) {
+      UnitParams q;
+      q.K1 = K1; q.P = P; q.r = rp; q.nk1 = (K1 + 63) / 64; q.nchunks = (P + kChunk - 1) / kChunk; q.natoms = up.natoms;
+      q.ns = up.ns; q.slot_bytes = up.slot_bytes; q.ns2 = up.ns2; q.ring2_bytes = up.ring2_bytes;
+      q.save_s = Sg ? 1 : 0; q.tiles = (int)tiles; q.status = status;
+      AB_CUDA_OK(cudaFuncSetAttribute(row_chain_units_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)up.smem));
+      row_chain_units_kernel<<<(unsigned)sms, 192, up.smem, st>>>(tmIn, tmF1, tmF2, tmOut, tmS, q);
+      AB_LAUNCH_OK();
+      return AB_OK;
+    }
+  }
   RowChainParams p;
   p.K1 = K1; p.P = second ? P : 0; p.r = rp; p.nk1 = (K1 + 63) / 64; p.nchunks = second ? (P + kChunk - 1) / kChunk : 0;
   p.natoms = pl.natoms; p.ns = pl.ns; p.slot_bytes = pl.slot_bytes; p.ns2 = pl.ns2; p.save_s = Sg ? 1 : 0;

@@ -82,6 +82,14 @@ def test_chain_bf16(ab, N, m, n, r, save_T):
     check_chain(ab, d, True, save_T)
 
 
+@pytest.mark.parametrize("N,m,n,r", [(47361, 256, 320, 64), (19244, 384, 256, 192), (40000, 136, 200, 24)])
+def test_chain_many_row_blocks(ab, N, m, n, r):
+    """More 128-row blocks than SMs: persistent CTAs that take the blocks two at a time (and a single one
+    where a CTA's share is odd), ragged last block, T kept."""
+    d = synth.chain_case(300 + r, m, n, r, N, bf16=True)
+    check_chain(ab, d, True, save_T=True)
+
+
 def test_chain_strided_factors(ab):
     d = synth.chain_case(5, 96, 80, 24, 150, bf16=False)
     Abig = torch.zeros((96, 40), device="cuda")
@@ -478,7 +486,10 @@ def test_full_size_frozen_factor_variants(ab):
     torch.cuda.synchronize()
     assert b_group[1] is None and a_group[0] is None and a_group[2] is None
     assert torch.equal(full[0], b_group[0]) and torch.equal(full[2], b_group[2])
-    assert torch.equal(full[1], a_group[1]) and torch.equal(full[1], a_group_recomputed[1])
+    assert torch.equal(full[1], a_group[1])
+    # T rebuilt by the first-product-only launch walks the slabs of B in another order than the forward
+    # did: same T up to the rounding of its fp32 sums, hence a few bf16 last-place differences
+    assert orc.rel_frob(host(a_group_recomputed[1]), host(full[1])) <= 1e-4
 
 
 def test_full_size_resnet_conv(ab):
