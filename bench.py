@@ -36,7 +36,7 @@ LAYERS = ((3072, 768), (768, 3072))
 K_GROUPS = 4
 # dram__bytes_read.sum + dram__bytes_write.sum of one row_chain_kernel launch (forward, 50,432 rows),
 # from the ncu capture summarised under profiles/; None until the kernel of that capture is current.
-ROW_CHAIN_DRAM_BYTES_PER_LAUNCH = 350.0e6   # forward of W1: 79.7 MB read + 270.3 MB written
+ROW_CHAIN_DRAM_BYTES_PER_LAUNCH = 349.2e6   # forward of W1: 79.4 MB read + 269.9 MB written (ncu capture under profiles/)
 
 
 def chain_flops(N, layers=LAYERS, r=R):
@@ -474,7 +474,7 @@ def run_ours(args):
         # (both layers have m+n = 3840), 2 N (m+n) bytes.
         fwd_flops = 2.0 * N * R * 3840
         fwd_tflops = fwd_flops / (fwd_ms * 1e-3) / 1e12
-        roof = dict(bound="tensor", kernel="row_chain_kernel (one launch = ab_layer_forward of one layer)",
+        roof = dict(bound="tensor", kernel="row_chain_units_kernel (one launch = ab_layer_forward of one layer at this size)",
                     achieved=fwd_tflops, peak=pk["tc_sustained"], unit="TFLOP/s", frac=fwd_tflops / pk["tc_sustained"],
                     traffic=ROW_CHAIN_DRAM_BYTES_PER_LAUNCH, us_per_launch=fwd_ms * 1e3,
                     peak_source=f"bf16_tflops_sustained of {pk['source']}",

@@ -327,9 +327,11 @@ int gemm_simt(const void* A, int a_dt, int64_t sAm, int64_t sAk,
               void* C, int c_dt, int64_t ldc,
               int64_t M, int64_t N, int64_t K, cudaStream_t st) {
   if (M <= 0 || N <= 0) return AB_OK;
+  const int64_t tiles64 = ((M + 63) / 64) * ((N + 63) / 64);
   if (a_dt == AB_F32 && b_dt == AB_F32 && c_dt == AB_F32 && M < ((int64_t)1 << 22) && N < ((int64_t)1 << 31) &&
-      K < ((int64_t)1 << 31)) {
-    // all-fp32 problems take the register-tiled kernel (fp32 sums in ascending k)
+      K < ((int64_t)1 << 31) && tiles64 >= 296) {
+    // all-fp32 problems with enough tiles to fill the SMs twice take the register-tiled kernel (fp32
+    // sums in ascending k); smaller ones are latency-bound and do better with 256 threads per tile
     GemmDesc d;
     d.A = static_cast<const float*>(A); d.B = static_cast<const float*>(B); d.C = C;
     d.sAm = sAm; d.sAk = sAk; d.sBk = sBk; d.sBn = sBn; d.ldc = ldc;
