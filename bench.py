@@ -296,6 +296,29 @@ def other_workloads(ab, torch, iters=10):
     return out
 
 
+def optimizer_step(ab, torch, iters=10):
+    """AdamW update of a whole ViT-B/16 factor set (31.85 M fp32 master values, moments in fp32, bf16 copy
+    written): a pure HBM stream of 30 bytes per value."""
+    count = 31850496
+    p = torch.randn(count, device="cuda")
+    g = torch.randn(count, device="cuda")
+    m = torch.zeros(count, device="cuda")
+    v = torch.zeros(count, device="cuda")
+    lp = torch.empty(count, dtype=torch.bfloat16, device="cuda")
+    for k in range(3):
+        ab.ab_adamw_step(p, g, m, v, 1e-3, k + 1, param_bf16=lp)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for k in range(iters):
+        ab.ab_adamw_step(p, g, m, v, 1e-3, k + 4, param_bf16=lp)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    gbs = 30.0 * count / (ms * 1e-3) / 1e9
+    return dict(values=count, ms=ms, gbs=gbs, frac_of_measured_hbm=gbs / measured_peaks()["hbm"])
+
+
 def backward_variants(ab, torch, layers, N, iters=10):
     """The two frozen-factor steps of the method on the same workload: a B-group trains B (forward, then
     dT, dX and dB; A frozen, no dA), an A-group trains A (forward with T kept, then dA only -- its dX is
@@ -502,6 +525,7 @@ def run_ours(args):
             line["group_sync_model"] = vit_model_sync(ab, torch)
         if world == 1 and not args.no_other_workloads:
             line["other_workloads"] = other_workloads(ab, torch)
+            line["adamw_update_vit_factors"] = optimizer_step(ab, torch)
         if world == 1 and not args.no_cpu_baseline:
             cb = cpu_baseline(inputs, min(N, args.ref_rows))
             line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}

@@ -119,6 +119,28 @@ int ab_layer_backward(const void* x, const void* dY, const void* A, const void* 
                       void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * One AdamW update of a factor from the gradient ab_layer_backward left (the paper trains with
+ * AdamW, Section "Experiments"; decoupled weight decay):
+ *   p <- p (1 - lr wd);  m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;
+ *   p <- p - lr (m / (1-b1^step)) / (sqrt(v / (1-b2^step)) + eps).
+ * param, m, v: fp32 [count], updated in place; grad: fp32 [count]; param_bf16: NULL, or bf16
+ * [count] that receives the updated values rounded to nearest even (the copy the tensor-core
+ * chain reads).  step >= 1.  lr is the rate of this step: multiply ab_lr_rebound_factor in
+ * while a rebound is running.  All pointers device memory; one launch on the stream.
+ */
+int ab_adamw_step(float* param, const float* grad, float* m, float* v, void* param_bf16, int64_t count,
+                  float lr, float beta1, float beta2, float eps, float weight_decay, int step,
+                  void* cuda_stream);
+
+/*
+ * Learning-rate rebound (Section "Methodology", "learning rate rebound"): whenever the parameters
+ * change shape the rate drops to near zero and climbs back to its scheduled value over
+ * rebound_steps steps.  The paper does not give the shape of the climb; this is the linear
+ * one: floor + (1 - floor) * min(1, steps_since_change / rebound_steps).  Host function.
+ */
+float ab_lr_rebound_factor(int steps_since_change, int rebound_steps, float floor);
+
+/*
  * Mean of K group copies (Algorithm 1: A <- allReduce(A / worldSize), likewise B), the K
  * workers being K arenas in one device's memory: copy k starts at base + k*stride_elems
  * (elements of in_dt).  In fp32 and in a fixed order:

@@ -205,6 +205,27 @@ def group_sync(A_copies, B_copies, r_max, sigma_cutoff):
     return dict(Abar=Abar, Bbar=Bbar, W=W, A=A, B=B, sigma=s, r=r)
 
 
+def adamw_step(p, g, m, v, lr, step, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=1e-2):
+    """One AdamW update with decoupled weight decay (the optimizer of the paper's experiments), float64:
+    p <- p (1 - lr wd); m <- b1 m + (1 - b1) g; v <- b2 v + (1 - b2) g^2;
+    p <- p - lr (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps).  Returns new (p, m, v)."""
+    p, g, m, v = _f64(p), _f64(g), _f64(m), _f64(v)
+    p = p * (1.0 - lr * weight_decay)
+    m = beta1 * m + (1.0 - beta1) * g
+    v = beta2 * v + (1.0 - beta2) * g * g
+    mhat = m / (1.0 - beta1 ** step)
+    vhat = v / (1.0 - beta2 ** step)
+    return p - lr * mhat / (np.sqrt(vhat) + eps), m, v
+
+
+def lr_rebound_factor(steps_since_change, rebound_steps, floor=0.0):
+    """Learning-rate rebound (Methodology): the rate restarts at `floor` of its scheduled value when the
+    parameters change shape and climbs back linearly over rebound_steps steps (the paper gives no shape)."""
+    if rebound_steps <= 0 or steps_since_change >= rebound_steps:
+        return 1.0
+    return floor + (1.0 - floor) * max(0, steps_since_change) / rebound_steps
+
+
 def rel_frob(a, b):
     """||a - b||_F / ||b||_F in float64 (0 when both are zero)."""
     a, b = _f64(a), _f64(b)

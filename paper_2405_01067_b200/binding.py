@@ -23,7 +23,7 @@ AB_SYNC_AUTO, AB_SYNC_DENSE, AB_SYNC_FACTORED = 0, 1, 2
 
 EXPORTS = ["ab_status_string", "ab_version", "ab_launch_count", "ab_workspace_bytes", "ab_layer_forward", "ab_layer_backward",
            "ab_group_average", "ab_recombine", "ab_svd_split", "ab_group_sync", "ab_sync_workspace_bytes",
-           "ab_layer_forward_static", "ab_static_scratch_elems"]
+           "ab_layer_forward_static", "ab_static_scratch_elems", "ab_adamw_step", "ab_lr_rebound_factor"]
 
 
 class AbError(RuntimeError):
@@ -75,6 +75,10 @@ def lib() -> ctypes.CDLL:
     L.ab_layer_forward_static.restype = c_int
     L.ab_layer_forward_static.argtypes = [c_void_p] * 4 + [c_int64] + [c_int] * 6 + [c_void_p]
     L.ab_static_scratch_elems.restype = c_size_t
+    L.ab_adamw_step.restype = c_int
+    L.ab_adamw_step.argtypes = [c_void_p] * 5 + [c_int64] + [c_float] * 5 + [c_int, c_void_p]
+    L.ab_lr_rebound_factor.restype = c_float
+    L.ab_lr_rebound_factor.argtypes = [c_int, c_int, c_float]
     _lib = L
     return L
 
@@ -179,6 +183,25 @@ def ab_layer_backward(x, dY, A, B, T_saved=None, want=("dX", "dA", "dB"), dX=Non
                                  N, m, n, r, A.stride(0), B.stride(0), dt, _ptr(ws), ws.numel(), _stream(stream))
     _check(st, "ab_layer_backward")
     return dX, dA, dB
+
+
+def ab_adamw_step(param, grad, m, v, lr, step, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=1e-2, param_bf16=None,
+                  stream=None):
+    """One AdamW update in place (param, m, v fp32; grad fp32); param_bf16 optionally receives the rounded copy."""
+    _dev_ok(param, grad, m, v, param_bf16)
+    for t in (param, grad, m, v):
+        if t.dtype != torch.float32 or not t.is_contiguous():
+            raise ValueError("ab_adamw_step takes contiguous fp32 tensors")
+    if param_bf16 is not None and (param_bf16.dtype != torch.bfloat16 or param_bf16.numel() != param.numel()):
+        raise ValueError("param_bf16 must be a bf16 tensor of the same size")
+    st = lib().ab_adamw_step(_ptr(param), _ptr(grad), _ptr(m), _ptr(v), _ptr(param_bf16), param.numel(), lr, beta1, beta2,
+                             eps, weight_decay, step, _stream(stream))
+    _check(st, "ab_adamw_step")
+    return param
+
+
+def ab_lr_rebound_factor(steps_since_change: int, rebound_steps: int, floor: float = 0.0) -> float:
+    return float(lib().ab_lr_rebound_factor(steps_since_change, rebound_steps, floor))
 
 
 def ab_group_average(copies, out=None, out_dtype=None, stream=None):

@@ -165,6 +165,24 @@ int ab_layer_backward(const void* x, const void* dY, const void* A, const void* 
   return general_backward(x, dY, A, B, T_saved, dX, dA, dB, N, m, n, r, ldA, ldB, dt, ws, ws_bytes, st);
 }
 
+int ab_adamw_step(float* param, const float* grad, float* m, float* v, void* param_bf16, int64_t count,
+                  float lr, float beta1, float beta2, float eps, float weight_decay, int step,
+                  void* cuda_stream) {
+  if (count < 0 || step < 1) return AB_ERR_INVALID_ARG;
+  if (count == 0) return AB_OK;
+  if (!param || !grad || !m || !v) return AB_ERR_INVALID_ARG;
+  if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps > 0.f)) return AB_ERR_INVALID_ARG;
+  if (!have_device()) return AB_ERR_CUDA;
+  return adamw_step(param, grad, m, v, static_cast<bf16*>(param_bf16), count, lr, beta1, beta2, eps, weight_decay,
+                    step, static_cast<cudaStream_t>(cuda_stream));
+}
+
+float ab_lr_rebound_factor(int steps_since_change, int rebound_steps, float floor) {
+  if (rebound_steps <= 0 || steps_since_change >= rebound_steps) return 1.f;
+  if (steps_since_change < 0) steps_since_change = 0;
+  return floor + (1.f - floor) * ((float)steps_since_change / (float)rebound_steps);
+}
+
 int ab_group_average(const void* base, int64_t stride_elems, int K, int64_t count,
                      int in_dt, int out_dt, void* out, void* cuda_stream) {
   if (!dtype_ok(in_dt) || !dtype_ok(out_dt)) return AB_ERR_INVALID_ARG;

@@ -133,6 +133,10 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
                   void* ws, size_t ws_bytes, cudaStream_t st);
 
 // ---- group mean (ab_average.cu) ----------------------------------------------------------------
+// AdamW step on fp32 master values (ab_optim.cu); p_lp: optional bf16 copy of the result.
+int adamw_step(float* p, const float* g, float* m, float* v, bf16* p_lp, int64_t count, float lr, float beta1,
+               float beta2, float eps, float weight_decay, int step, cudaStream_t st);
+
 // One mean per job in a single launch; results are fp32.  d_jobs is device memory.
 struct AvgJob { const void* base; int64_t stride; int64_t count; float* out; };
 int group_average_batched(const AvgJob* d_jobs, int njobs, int K, int in_dt, int64_t max_count, cudaStream_t st);

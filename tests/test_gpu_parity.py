@@ -425,6 +425,30 @@ def test_group_sync_factored_shapes(ab, m, n, r, K, count):
         assert bal <= 1e-3, (i, bal)
 
 
+@pytest.mark.parametrize("count", [1, 7, 4096 + 3, 3072 * 192])
+@pytest.mark.parametrize("with_bf16", [False, True])
+def test_adamw_step(ab, count, with_bf16):
+    """Three AdamW updates (the last with a rebound factor in the rate) against the checker; the bf16 copy is
+    the fp32 result rounded to nearest even."""
+    rng = np.random.default_rng(count)
+    p0 = rng.standard_normal(count).astype(np.float32)
+    p, m, v = dev(p0), torch.zeros(count, device="cuda"), torch.zeros(count, device="cuda")
+    lp = torch.empty(count, dtype=torch.bfloat16, device="cuda") if with_bf16 else None
+    rp, rm, rv = p0.astype(np.float64), np.zeros(count), np.zeros(count)
+    for step in (1, 2, 3):
+        g = rng.standard_normal(count).astype(np.float32)
+        lr = 1e-2 * (ab.ab_lr_rebound_factor(step, 4, 0.1) if step == 3 else 1.0)
+        ab.ab_adamw_step(p, dev(g), m, v, lr, step, 0.9, 0.99, 1e-8, 0.1, param_bf16=lp)
+        rp, rm, rv = orc.adamw_step(rp, g, rm, rv, lr, step, 0.9, 0.99, 1e-8, 0.1)
+    torch.cuda.synchronize()
+    assert abs(ab.ab_lr_rebound_factor(3, 4, 0.1) - orc.lr_rebound_factor(3, 4, 0.1)) < 1e-7
+    # fp32 arithmetic on values of order one: a few units of 6e-8, also where terms cancel
+    assert np.allclose(host(p), rp, rtol=2e-6, atol=5e-7)
+    assert np.allclose(host(m), rm, rtol=2e-6, atol=5e-7) and np.allclose(host(v), rv, rtol=2e-6, atol=5e-7)
+    if with_bf16:
+        assert torch.equal(lp, p.to(torch.bfloat16))
+
+
 # ------------------------------------------------------------------ full-size workloads
 
 def _oracle_backward_chunked(x, dY, A, B, rows=8192):
