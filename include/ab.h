@@ -206,7 +206,10 @@ typedef enum {
  * diagonal entry of a Gram matrix are taken as zero, which is exact for factors already
  * truncated by the rank rule); AB_SYNC_FACTORED returns
  * AB_ERR_UNSUPPORTED when r is too large, AB_SYNC_AUTO falls back to the dense path.
- * Workspace: ab_sync_workspace_bytes (covers either path).
+ * Workspace: ab_sync_workspace_bytes (covers either path).  When a W_out is given, the factored
+ * path runs that product on a helper stream of the library (one per device, lowest priority,
+ * created on first use) beside its Jacobi kernel and joins it before the call's last kernel, so
+ * the caller's stream order still covers everything the call writes.
  */
 int ab_group_sync(const ab_sync_desc* descs, int L, int K, float sigma_cutoff, int dt,
                   int* dev_status, void* ws, size_t ws_bytes, void* cuda_stream, int path);

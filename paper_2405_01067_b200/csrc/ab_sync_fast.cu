@@ -14,6 +14,7 @@
 // factors need a condition number below about 300 -- all workloads here are far inside.
 #include <algorithm>
 #include <cstdio>
+#include <mutex>
 #include <type_traits>
 #include <vector>
 
@@ -571,6 +572,28 @@ GemmDesc mk(const float* A, int64_t sAm, int64_t sAk, const float* B, int64_t sB
 
 }  // namespace
 
+// One helper stream per device (lowest priority, created on first use, kept for the life of the
+// process): the optional product W = Abar Bbar depends only on the means, so it runs there beside the
+// Cholesky and Jacobi kernels, which leave half of the SMs idle.
+cudaStream_t side_stream() {
+  static std::mutex mu;
+  static cudaStream_t streams[64] = {};
+  static bool tried[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!tried[dev]) {
+    tried[dev] = true;
+    int lo = 0, hi = 0;
+    if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess ||
+        cudaStreamCreateWithPriority(&streams[dev], cudaStreamNonBlocking, lo) != cudaSuccess) {
+      (void)cudaGetLastError();
+      streams[dev] = nullptr;
+    }
+  }
+  return streams[dev];
+}
+
 float rows_jacobi_tol(int s) { return 5e-7f * sqrtf((float)s) < 4e-6f ? 4e-6f : 5e-7f * sqrtf((float)s); }
 
 bool rows_jacobi_fits(int count, int s) {
@@ -694,14 +717,35 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   const float tol = rows_jacobi_tol(rmax);
   bool any_w = false;
   for (int i = 0; i < L; ++i) any_w = any_w || d[i].W_out != nullptr;
-  if (any_w) AB_TRY(gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, st));                 // a8 (optional)
+  // a8 (optional): forked off where the Jacobi kernel starts (the kernels before it fill every SM
+  // themselves), joined at the end
+  cudaStream_t side = any_w ? side_stream() : nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+  if (side) {
+    if (cudaEventCreateWithFlags(&fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&join, cudaEventDisableTiming) != cudaSuccess) {
+      (void)cudaGetLastError();
+      if (fork) cudaEventDestroy(fork);
+      if (join) cudaEventDestroy(join);
+      fork = join = nullptr;
+      side = nullptr;
+    }
+  }
+  if (any_w && !side) AB_TRY(gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, st));
   AB_TRY(gemm_simt_batched(w.gram_descs, (int)gg.size(), rmax, rmax, st));                  // Gram slices
   const size_t csm = chol_smem_bytes(rmax);
   AB_CUDA_OK(cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csm));
   chol_inv_kernel<<<2 * L, kCThreads, csm, st>>>(w.cjobs);                                  // R_A, R_B and inverses
   AB_LAUNCH_OK();
   AB_TRY(gemm_simt_batched(w.descs + 2 * L, L, rmax, rmax, st));                            // M
+  int side_rc = AB_OK;
+  if (side && cudaEventRecord(fork, st) != cudaSuccess) side_rc = AB_ERR_CUDA;
   AB_TRY(launch_jacobi(w.jobs, L, rmax, tol, st));                                    // SVD of M
+  if (side) {
+    if (side_rc == AB_OK && cudaStreamWaitEvent(side, fork, 0) != cudaSuccess) side_rc = AB_ERR_CUDA;
+    if (side_rc == AB_OK) side_rc = gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, side);
+    if (side_rc == AB_OK && cudaEventRecord(join, side) != cudaSuccess) side_rc = AB_ERR_CUDA;
+  }
   fast_rank_rule_kernel<<<(L + 127) / 128, 128, 0, st>>>(w.sig_ptrs, w.rs, sigma_cutoff, w.rout_ptrs, w.jstatus,
                                                          dev_status, L);
   AB_LAUNCH_OK();
@@ -709,6 +753,12 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   AB_TRY(gemm_simt_batched(w.descs + 5 * L, L, rmax, rmax, st));                            // Z_A
   AB_TRY(gemm_simt_batched(w.descs + 6 * L, L, mmax, rmax, st));                            // A'
   AB_TRY(gemm_simt_batched(w.descs + 7 * L, L, rmax, nmax, st));                            // B'
+  if (side) {
+    if (side_rc == AB_OK && cudaStreamWaitEvent(st, join, 0) != cudaSuccess) side_rc = AB_ERR_CUDA;
+    cudaEventDestroy(fork);      // released once the recorded work is done
+    cudaEventDestroy(join);
+    if (side_rc != AB_OK) { (void)cudaGetLastError(); return side_rc; }
+  }
   return AB_OK;
 }
 }  // namespace ab
