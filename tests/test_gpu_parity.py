@@ -372,6 +372,26 @@ def test_group_sync_factored_truncated_factors_and_bf16(ab):
         assert np.linalg.norm(host(A_out[0]) @ host(B_out[0]) - W) / np.linalg.norm(W) <= tol
 
 
+def test_group_sync_dense_many_matrices_of_short_side_256(ab):
+    """40 matrices whose short side is 256 through the dense route: too many for clusters of 4 or 8 CTAs
+    and too large for one CTA's shared memory, so each Gram matrix is solved by a pair of CTAs."""
+    cases = [_factored_case(900 + i, 256, 300, 64, 2) for i in range(2)]
+    devs = [(dev(a), dev(b)) for a, b in cases]
+    L = 40
+    plan = ab.SyncPlan([devs[i % 2][0] for i in range(L)], [devs[i % 2][1] for i in range(L)], 0.0)
+    A_out, B_out, sigma, r_out, status = ab.ab_group_sync(plan, path=ab.AB_SYNC_DENSE)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(status) == 0
+    for i in range(2):
+        W = orc.recombine(orc.group_average_f32(cases[i][0]), orc.group_average_f32(cases[i][1]))
+        s = np.linalg.svd(W, compute_uv=False)
+        assert int(r_out[i].item()) == 64
+        assert np.all(np.abs(host(sigma[i]) - s[:64]) <= 1e-4 * s[:64])
+        assert np.linalg.norm(host(A_out[i]) @ host(B_out[i]) - W) / np.linalg.norm(W) <= 1e-4
+    for i in range(2, L):
+        assert torch.equal(A_out[i], A_out[i % 2]) and torch.equal(sigma[i], sigma[i % 2])
+
+
 def _factored_case(seed, m, n, r, K):
     st = synth.streams(seed, ["AB"])
     sig = np.exp(-np.arange(r) / max(8.0, r / 3.0))           # sigma_min about 5 % of sigma_max
