@@ -14,6 +14,7 @@
 // factors need a condition number below about 300 -- all workloads here are far inside.
 #include <algorithm>
 #include <cstdio>
+#include <cstring>
 #include <mutex>
 #include <type_traits>
 #include <vector>
@@ -694,26 +695,34 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
     jb[i] = JacobiJob{w.M[i], w.Vs[i], d[i].sigma, w.jstatus + 3 * i + 2, r, r};
     sigp[i] = d[i].sigma; routp[i] = d[i].r_out; rs[i] = r;
   }
-  AB_CUDA_OK(cudaMemcpyAsync(w.descs, g.data(), g.size() * sizeof(GemmDesc), cudaMemcpyHostToDevice, st));
-  AB_CUDA_OK(cudaMemcpyAsync(w.gram_descs, gg.data(), gg.size() * sizeof(GemmDesc), cudaMemcpyHostToDevice, st));
-  AB_CUDA_OK(cudaMemcpyAsync(w.cjobs, cj.data(), cj.size() * sizeof(CholJob), cudaMemcpyHostToDevice, st));
-  AB_CUDA_OK(cudaMemcpyAsync(w.jobs, jb.data(), jb.size() * sizeof(JacobiJob), cudaMemcpyHostToDevice, st));
-  AB_CUDA_OK(cudaMemcpyAsync(w.sig_ptrs, sigp.data(), L * sizeof(float*), cudaMemcpyHostToDevice, st));
-  AB_CUDA_OK(cudaMemcpyAsync(w.rout_ptrs, routp.data(), L * sizeof(int*), cudaMemcpyHostToDevice, st));
-  AB_CUDA_OK(cudaMemcpyAsync(w.rs, rs.data(), L * sizeof(int), cudaMemcpyHostToDevice, st));
+  // All tables sit back to back in the workspace (descs ... rs): one host image, one copy.
+  std::vector<AvgJob> aj((size_t)2 * L);
+  int64_t longest = 0;
+  for (int i = 0; i < L; ++i) {
+    aj[2 * i] = AvgJob{d[i].A_copies, d[i].strideA, (int64_t)d[i].m * d[i].r, w.Abar[i]};
+    aj[2 * i + 1] = AvgJob{d[i].B_copies, d[i].strideB, (int64_t)d[i].r * d[i].n, w.Bbar[i]};
+    longest = std::max(longest, std::max(aj[2 * i].count, aj[2 * i + 1].count));
+  }
+  {
+    char* base = reinterpret_cast<char*>(w.descs);
+    const size_t span = (size_t)(reinterpret_cast<char*>(w.rs + L) - base);
+    std::vector<char> img(span, 0);
+    auto put = [&](const void* dev_ptr, const void* src, size_t bytes) {
+      std::memcpy(img.data() + (reinterpret_cast<const char*>(dev_ptr) - base), src, bytes);
+    };
+    put(w.descs, g.data(), g.size() * sizeof(GemmDesc));
+    put(w.gram_descs, gg.data(), gg.size() * sizeof(GemmDesc));
+    put(w.cjobs, cj.data(), cj.size() * sizeof(CholJob));
+    put(w.ajobs, aj.data(), aj.size() * sizeof(AvgJob));
+    put(w.jobs, jb.data(), jb.size() * sizeof(JacobiJob));
+    put(w.sig_ptrs, sigp.data(), L * sizeof(float*));
+    put(w.rout_ptrs, routp.data(), L * sizeof(int*));
+    put(w.rs, rs.data(), L * sizeof(int));
+    AB_CUDA_OK(cudaMemcpyAsync(base, img.data(), span, cudaMemcpyHostToDevice, st));
+  }
 
   // ---- a7: means of the K copies (fp32), all matrices in one launch
-  {
-    std::vector<AvgJob> aj((size_t)2 * L);
-    int64_t longest = 0;
-    for (int i = 0; i < L; ++i) {
-      aj[2 * i] = AvgJob{d[i].A_copies, d[i].strideA, (int64_t)d[i].m * d[i].r, w.Abar[i]};
-      aj[2 * i + 1] = AvgJob{d[i].B_copies, d[i].strideB, (int64_t)d[i].r * d[i].n, w.Bbar[i]};
-      longest = std::max(longest, std::max(aj[2 * i].count, aj[2 * i + 1].count));
-    }
-    AB_CUDA_OK(cudaMemcpyAsync(w.ajobs, aj.data(), aj.size() * sizeof(AvgJob), cudaMemcpyHostToDevice, st));
-    AB_TRY(group_average_batched(w.ajobs, 2 * L, K, dt, longest, st));
-  }
+  AB_TRY(group_average_batched(w.ajobs, 2 * L, K, dt, longest, st));
   const float tol = rows_jacobi_tol(rmax);
   bool any_w = false;
   for (int i = 0; i < L; ++i) any_w = any_w || d[i].W_out != nullptr;
