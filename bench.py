@@ -465,7 +465,8 @@ def run_ours(args):
     sampler.stop_flag = True
     launches = ab.ab_launch_count() - launches0
     total_ms = t_begin.elapsed_time(t_end)
-    chain_ms = sum(mk[0].elapsed_time(mk[1]) for mk in marks)
+    chain_each = sorted(mk[0].elapsed_time(mk[1]) for mk in marks)
+    chain_ms = sum(chain_each)
     sync_ms = sum(mk[1].elapsed_time(mk[2]) for mk in marks)
     fwd_ms = sum(a.elapsed_time(b) for a, b in fwd_events) / max(len(fwd_events), 1)   # per forward launch
     if int(plan.status.abs().sum().item()) != 0:
@@ -522,7 +523,8 @@ def run_ours(args):
                     config=dict(workload="vit_b16_mlp_pair_r192", rows=N, layers=[list(s) for s in LAYERS], r=R,
                                 K=K_GROUPS, sync="mean + recombine (W written) + truncated-SVD split of both layers every step, factored route",
                                 l2="inputs larger than L2 (about 0.8 GB of activations read per step)"),
-                    chain_ms_per_step=chain_ms / K, group_sync_ms_per_step=sync_ms / K,
+                    chain_ms_per_step=chain_ms / K, chain_ms_median=chain_each[len(chain_each) // 2],
+                    chain_ms_min=chain_each[0], group_sync_ms_per_step=sync_ms / K,
                     pct_of_nominal_bf16_peak=100.0 * per_gpu / NOMINAL_BF16_TFLOPS,
                     e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                              ms_per_step=e2e_ms / K, ms_per_step_with_group_sync=e2e_sync_ms / K),
