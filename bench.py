@@ -120,9 +120,19 @@ def cpu_baseline(inputs, rows, sync_scale=8):
         s = synth.vit_sync_matrix(1, i, m, n, K=K_GROUPS, scale=sync_scale)
         orc.group_sync(synth.group_copies(s["A"], s["noise_A"]), synth.group_copies(s["B"], s["noise_B"]), s["r"], 0.0)
     t_sync = time.perf_counter() - t0
+    # for scale: the library SVD (LAPACK, float64) of one full-size recombined matrix of each shape
+    lapack = {}
+    rng = np.random.default_rng(0)
+    for (m, n) in ((768, 768), (3072, 768)):
+        W = rng.standard_normal((m, n // 4)) @ rng.standard_normal((n // 4, n))
+        t0 = time.perf_counter()
+        np.linalg.svd(W, full_matrices=False)
+        lapack[f"{m}x{n}"] = time.perf_counter() - t0
     return dict(value=chain_flops(rows) / t_chain / 1e12, unit=UNIT, cores=int(cores), kind="oracle",
                 sample=f"chain: first {rows} of 50432 rows of both layers, float64, {t_chain:.2f} s; "
-                       f"sync: both matrices at 1/{sync_scale} scale, own Jacobi SVD, {t_sync:.2f} s",
+                       f"sync: both matrices at 1/{sync_scale} scale, own Jacobi SVD, {t_sync:.2f} s; "
+                       f"LAPACK SVD of one full-size matrix: 768x768 {lapack['768x768']:.2f} s, "
+                       f"3072x768 {lapack['3072x768']:.2f} s",
                 chain_s=t_chain, sync_sample_s=t_sync)
 
 
