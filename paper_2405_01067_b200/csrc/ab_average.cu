@@ -2,6 +2,11 @@
 // Each thread owns 16 input bytes per copy (4 fp32 or 8 bf16 values), keeps up to four copies'
 // loads in flight, adds them in fp32 in ascending k and scales by fl(1/K).  The sum order is
 // part of the contract (results are compared bit for bit).
+// Launch shape: one 16-byte group per thread, i.e. as many 256-thread blocks as the data has
+// groups.  On a 1.15 GB stream (8 copies of 31.85 M fp32 values) that draws 6.9-7.0 TB/s, against
+// 6.0 TB/s for a grid of 8 blocks per SM walking the data with a grid-sized stride and 6.7 TB/s
+// for 16 or 32 blocks per SM; all K loads in flight at once, two groups per thread, 256-bit
+// loads and other cache hints measured the same or worse.
 #include <algorithm>
 
 #include "ab_common.cuh"
@@ -84,19 +89,27 @@ average_vec_kernel(const TIn* __restrict__ base, int64_t stride, int K, int64_t 
     mean_vec_at<TIn, TOut>(base, stride, K, inv, out, i);
 }
 
-// Many means in one launch (blockIdx.y = job), fp32 results: the vector body where the job's
-// pointers and stride allow it, single elements for the rest.  Same sums as the kernels above.
+// Many means in one launch, fp32 results.  The grid is flat: job j owns the blocks
+// [first_block_j, first_block_{j+1}), one 16-byte group per thread, and a block finds its job by
+// bisection over the table.  The vector body runs where the job's pointers and stride allow it,
+// single elements cover the rest.  Same sums as the kernels above.
 template <typename TIn>
 __global__ void __launch_bounds__(256)
-average_batched_kernel(const AvgJob* __restrict__ jobs, int K, float inv) {
+average_batched_kernel(const AvgJob* __restrict__ jobs, int njobs, int K, float inv) {
   constexpr int V = Vec<TIn>::N;
-  const AvgJob j = jobs[blockIdx.y];
+  int lo = 0, hi = njobs - 1;
+  while (lo < hi) {                         // last job whose first block is <= blockIdx.x
+    const int mid = (lo + hi + 1) >> 1;
+    if (jobs[mid].first_block <= (int64_t)blockIdx.x) lo = mid; else hi = mid - 1;
+  }
+  const AvgJob j = jobs[lo];
+  const int64_t nblocks = (lo + 1 < njobs ? jobs[lo + 1].first_block : (int64_t)gridDim.x) - j.first_block;
   const TIn* base = static_cast<const TIn*>(j.base);
   const bool vec_ok = ((reinterpret_cast<uintptr_t>(j.base) | reinterpret_cast<uintptr_t>(j.out)) & 15u) == 0 &&
                       (j.stride % V == 0);
   const int64_t nvec = vec_ok ? j.count / V : 0;
-  const int64_t step = (int64_t)gridDim.x * blockDim.x;
-  const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t step = nblocks * blockDim.x;
+  const int64_t t0 = ((int64_t)blockIdx.x - j.first_block) * blockDim.x + threadIdx.x;
   for (int64_t i = t0; i < nvec; i += step) mean_vec_at<TIn, float>(base, j.stride, K, inv, j.out, i);
   for (int64_t i = nvec * V + t0; i < j.count; i += step) {
     float s = to_f32(base[i]);
@@ -129,7 +142,7 @@ int run(const void* base_, int64_t stride, int K, int64_t count, void* out_, cud
   int sms = 148;
   if (nvec > 0) {
     int64_t blocks = (nvec + 255) / 256;
-    int64_t cap = (int64_t)sms * 8;
+    int64_t cap = (int64_t)1 << 30;          // beyond that the kernel's stride loop takes over
     unsigned grid = (unsigned)(blocks < cap ? blocks : cap);
     average_vec_kernel<TIn, TOut><<<grid, 256, 0, st>>>(base, stride, K, nvec, inv, out);
     AB_LAUNCH_OK();
@@ -157,15 +170,18 @@ int group_average(const void* base, int64_t stride_elems, int K, int64_t count,
   return run<bf16, bf16>(base, stride_elems, K, count, out, st);
 }
 
-int group_average_batched(const AvgJob* d_jobs, int njobs, int K, int in_dt, int64_t max_count, cudaStream_t st) {
-  if (njobs <= 0 || max_count <= 0) return AB_OK;
-  const int64_t blocks = (max_count / 4 + 255) / 256 + 1;
-  const int64_t cap = std::max<int64_t>(1, (int64_t)148 * 8 / njobs);
-  dim3 grid((unsigned)std::min(blocks, cap), (unsigned)njobs);
-  if (grid.y > 65535u) return AB_ERR_UNSUPPORTED;
+int64_t average_job_blocks(int64_t count, int in_dt) {
+  const int64_t v = in_dt == AB_F32 ? 4 : 8;
+  const int64_t groups = (count + v - 1) / v;
+  return std::max<int64_t>(1, (groups + 255) / 256);
+}
+
+int group_average_batched(const AvgJob* d_jobs, int njobs, int K, int in_dt, int64_t total_blocks, cudaStream_t st) {
+  if (njobs <= 0 || total_blocks <= 0) return AB_OK;
+  if (total_blocks > ((int64_t)1 << 30)) return AB_ERR_UNSUPPORTED;
   const float inv = 1.0f / (float)K;
-  if (in_dt == AB_F32) average_batched_kernel<float><<<grid, 256, 0, st>>>(d_jobs, K, inv);
-  else average_batched_kernel<bf16><<<grid, 256, 0, st>>>(d_jobs, K, inv);
+  if (in_dt == AB_F32) average_batched_kernel<float><<<(unsigned)total_blocks, 256, 0, st>>>(d_jobs, njobs, K, inv);
+  else average_batched_kernel<bf16><<<(unsigned)total_blocks, 256, 0, st>>>(d_jobs, njobs, K, inv);
   AB_LAUNCH_OK();
   return AB_OK;
 }

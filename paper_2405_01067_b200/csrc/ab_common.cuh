@@ -138,8 +138,11 @@ int adamw_step(float* p, const float* g, float* m, float* v, bf16* p_lp, int64_t
                float beta2, float eps, float weight_decay, int step, cudaStream_t st);
 
 // One mean per job in a single launch; results are fp32.  d_jobs is device memory.
-struct AvgJob { const void* base; int64_t stride; int64_t count; float* out; };
-int group_average_batched(const AvgJob* d_jobs, int njobs, int K, int in_dt, int64_t max_count, cudaStream_t st);
+// One mean of a batched launch.  first_block: the job's first block in the flat grid (running sum of
+// average_job_blocks over the jobs before it); the launch gets the sum over all jobs.
+struct AvgJob { const void* base; int64_t stride; int64_t count; float* out; int64_t first_block; };
+int64_t average_job_blocks(int64_t count, int in_dt);
+int group_average_batched(const AvgJob* d_jobs, int njobs, int K, int in_dt, int64_t total_blocks, cudaStream_t st);
 int group_average(const void* base, int64_t stride_elems, int K, int64_t count,
                   int in_dt, int out_dt, void* out, cudaStream_t st);
 

@@ -63,8 +63,10 @@ int adamw_step(float* p, const float* g, float* m, float* v, bf16* p_lp, int64_t
   a.c1 = (float)(1.0 / (1.0 - pow((double)beta1, (double)step)));
   a.c2 = (float)(1.0 / (1.0 - pow((double)beta2, (double)step)));
   const int vec_ok = aligned(p, 16) && aligned(g, 16) && aligned(m, 16) && aligned(v, 16) && (!p_lp || aligned(p_lp, 8));
-  const int64_t blocks = (count / 4 + 255) / 256 + 1;
-  const unsigned grid = (unsigned)(blocks < 148 * 8 ? blocks : 148 * 8);
+  // one float4 per thread: a grid as long as the data streams faster than a few blocks per SM striding over it
+  const int64_t blocks = ((vec_ok ? count / 4 : count) + 255) / 256 + 1;
+  const int64_t cap = (int64_t)1 << 30;
+  const unsigned grid = (unsigned)(blocks < cap ? blocks : cap);
   adamw_kernel<<<grid, 256, 0, st>>>(p, g, m, v, p_lp, count, vec_ok, a);
   AB_LAUNCH_OK();
   return AB_OK;

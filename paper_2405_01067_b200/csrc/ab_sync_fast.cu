@@ -697,11 +697,14 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   }
   // All tables sit back to back in the workspace (descs ... rs): one host image, one copy.
   std::vector<AvgJob> aj((size_t)2 * L);
-  int64_t longest = 0;
+  int64_t avg_blocks = 0;            // flat grid of the batched mean: one 16-byte group per thread
   for (int i = 0; i < L; ++i) {
-    aj[2 * i] = AvgJob{d[i].A_copies, d[i].strideA, (int64_t)d[i].m * d[i].r, w.Abar[i]};
-    aj[2 * i + 1] = AvgJob{d[i].B_copies, d[i].strideB, (int64_t)d[i].r * d[i].n, w.Bbar[i]};
-    longest = std::max(longest, std::max(aj[2 * i].count, aj[2 * i + 1].count));
+    aj[2 * i] = AvgJob{d[i].A_copies, d[i].strideA, (int64_t)d[i].m * d[i].r, w.Abar[i], 0};
+    aj[2 * i + 1] = AvgJob{d[i].B_copies, d[i].strideB, (int64_t)d[i].r * d[i].n, w.Bbar[i], 0};
+    for (int h = 0; h < 2; ++h) {
+      aj[2 * i + h].first_block = avg_blocks;
+      avg_blocks += average_job_blocks(aj[2 * i + h].count, dt);
+    }
   }
   {
     char* base = reinterpret_cast<char*>(w.descs);
@@ -722,7 +725,7 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   }
 
   // ---- a7: means of the K copies (fp32), all matrices in one launch
-  AB_TRY(group_average_batched(w.ajobs, 2 * L, K, dt, longest, st));
+  AB_TRY(group_average_batched(w.ajobs, 2 * L, K, dt, avg_blocks, st));
   const float tol = rows_jacobi_tol(rmax);
   bool any_w = false;
   for (int i = 0; i < L; ++i) any_w = any_w || d[i].W_out != nullptr;
