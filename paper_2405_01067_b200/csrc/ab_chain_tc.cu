@@ -47,6 +47,7 @@ struct RowChainParams {
   int slot_bytes;
   int ns2;       // stages of the second product's ring (one 128 x 64 atom of F2 each)
   int save_s;    // 1: copy S to global through tmS
+  int clear_status;   // 1: this is the first kernel of a call and zeroes the status word (see clear_status_word)
   int* status;
 };
 
@@ -63,6 +64,15 @@ struct Bars {
 __device__ __forceinline__ void raise_timeout(Bars* b, int* status) {
   *reinterpret_cast<volatile int*>(&b->abort_any) = 1;
   atomicExch(status, (int)AB_ERR_TIMEOUT);
+}
+
+// The status word of a call starts at zero.  The first kernel of the call clears it itself (block 0,
+// right after dep_wait) instead of a memset in the stream, which would sit between this kernel and the
+// one before it and undo the overlap of dep_wait.  Block 0 runs in the first wave and gets here within
+// microseconds of the launch; a kernel raises AB_ERR_TIMEOUT only after a wait of about a second, so
+// the clear cannot wipe a raised error.
+__device__ __forceinline__ void clear_status_word(int enabled, int* status) {
+  if (enabled && blockIdx.x == 0 && threadIdx.x == 0) atomicExch(status, 0);
 }
 
 // epilogue-wide wait: every epilogue thread calls it; the verdict is uniform
@@ -126,6 +136,9 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
+  dep_wait();            // nothing above touches global memory
+  dep_launch();
+  clear_status_word(p.clear_status, p.status);
   // T (r <= 256 columns) is read out into S before the second product starts, so the two
   // 256-column accumulators of the second product reuse its columns.
   const uint32_t tT = tmem_base;
@@ -305,6 +318,7 @@ struct UnitParams {
   int ns2, ring2_bytes;    // second product: 32 KB slots at the start of shared memory
   int save_s;
   int tiles;               // 128-row blocks in all
+  int clear_status;
   int* status;
 };
 
@@ -345,6 +359,9 @@ row_chain_units_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
+  dep_wait();            // nothing above touches global memory
+  dep_launch();
+  clear_status_word(p.clear_status, p.status);
   // TMEM: block b of a unit keeps its S accumulator at column 256 b while the first product runs;
   // accumulator b of the second product takes the same 256 columns afterwards.
 
@@ -555,6 +572,7 @@ struct GradParams {
   int r, natoms, ns, slot_bytes;
   int slices, rows_per_slice;   // rows_per_slice is a multiple of 64
   int N;
+  int clear_status;
   int* status;
 };
 
@@ -595,6 +613,9 @@ grad_kernel(const __grid_constant__ CUtensorMap tmAct0, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
+  dep_wait();            // nothing above touches global memory
+  dep_launch();
+  clear_status_word(p.clear_status, p.status);
 
   if (warp == 0) {
     if (lane == 0) {
@@ -678,6 +699,8 @@ __global__ void __launch_bounds__(256)
 reduce_partials_kernel(const float* __restrict__ pA, float* __restrict__ dA, int PA, int nA,
                        const float* __restrict__ pB, float* __restrict__ dB, int PB, int slices, int r, int rp) {
   // r: columns of the results; rp: row length of the partials (r rounded up to 16)
+  dep_wait();
+  dep_launch();
   if ((int)blockIdx.x < nA) {
     const int64_t total4 = (int64_t)PA * r / 4;
     const int64_t i4 = (int64_t)blockIdx.x * 256 + threadIdx.x;
@@ -718,8 +741,12 @@ reduce_partials_kernel(const float* __restrict__ pA, float* __restrict__ dA, int
 // Both factor transposes of a backward call in one launch: At[j][i] = A[i][j] (A is m x r, row stride
 // ldA) for blocks [0, nA), Bt[j][i] = B[i][j] (B is r x n, row stride ldB) after that.
 __global__ void transpose_factors_kernel(const bf16* __restrict__ A, int m, int r, int ldA, bf16* __restrict__ At, int nA,
-                                         const bf16* __restrict__ B, int n, int ldB, bf16* __restrict__ Bt) {
+                                         const bf16* __restrict__ B, int n, int ldB, bf16* __restrict__ Bt,
+                                         int* status_to_clear) {
   __shared__ bf16 tile[32][33];
+  dep_wait();
+  dep_launch();
+  clear_status_word(status_to_clear != nullptr, status_to_clear);
   const bool first = (int)blockIdx.x < nA;
   const bf16* src = first ? A : B;
   bf16* dst = first ? At : Bt;
@@ -741,6 +768,30 @@ __global__ void transpose_factors_kernel(const bf16* __restrict__ A, int m, int 
 
 // ---------------------------------------------------------------------------------------------
 // host side
+// Launch with programmatic stream serialisation (see dep_wait): only for kernels that call dep_wait()
+// before their first access to global memory.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dep(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#define AB_LAUNCH_DEP(...)                         \
+  do {                                             \
+    if (launch_dep(__VA_ARGS__) != cudaSuccess) {  \
+      cudaGetLastError();                          \
+      return AB_ERR_CUDA;                          \
+    }                                              \
+  } while (0)
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -868,7 +919,7 @@ BwdWs bwd_ws(void* ws, int64_t N, int m, int n, int r) {
 
 // S = In F1^T (saved to Sg if not null), Out = S F2^T (skipped if Out is null)
 int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1, const void* F2, int ldF2, int P,
-                     void* Out, void* Sg, int r, int* status, cudaStream_t st) {
+                     void* Out, void* Sg, int r, int* status, bool clear_status, cudaStream_t st) {
   const int rp = pad16(r);
   RowPlan pl = row_plan(rp);
   if (pl.ns < 2 || pl.ns2 < 2) return AB_ERR_UNSUPPORTED;
@@ -896,9 +947,9 @@ int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1
       UnitParams q;
       q.K1 = K1; q.P = P; q.r = rp; q.nk1 = (K1 + 63) / 64; q.nchunks = (P + kChunk - 1) / kChunk; q.natoms = up.natoms;
       q.ns = up.ns; q.slot_bytes = up.slot_bytes; q.ns2 = up.ns2; q.ring2_bytes = up.ring2_bytes;
-      q.save_s = Sg ? 1 : 0; q.tiles = (int)tiles; q.status = status;
+      q.save_s = Sg ? 1 : 0; q.tiles = (int)tiles; q.clear_status = clear_status ? 1 : 0; q.status = status;
       AB_CUDA_OK(cudaFuncSetAttribute(row_chain_units_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)up.smem));
-      row_chain_units_kernel<<<(unsigned)sms, 192, up.smem, st>>>(tmIn, tmF1, tmF2, tmOut, tmS, q);
+      AB_LAUNCH_DEP(row_chain_units_kernel, dim3((unsigned)sms), dim3(192), up.smem, st, tmIn, tmF1, tmF2, tmOut, tmS, q);
       AB_LAUNCH_OK();
       return AB_OK;
     }
@@ -906,10 +957,11 @@ int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1
   RowChainParams p;
   p.K1 = K1; p.P = second ? P : 0; p.r = rp; p.nk1 = (K1 + 63) / 64; p.nchunks = second ? (P + kChunk - 1) / kChunk : 0;
   p.natoms = pl.natoms; p.ns = pl.ns; p.slot_bytes = pl.slot_bytes; p.ns2 = pl.ns2; p.save_s = Sg ? 1 : 0;
+  p.clear_status = clear_status ? 1 : 0;
   p.status = status;
   AB_CUDA_OK(cudaFuncSetAttribute(row_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
   const unsigned grid = (unsigned)((N + 127) / 128);
-  row_chain_kernel<<<grid, 192, pl.smem, st>>>(tmIn, tmF1, tmF2, tmOut, tmS, p);
+  AB_LAUNCH_DEP(row_chain_kernel, dim3(grid), dim3(192), pl.smem, st, tmIn, tmF1, tmF2, tmOut, tmS, p);
   AB_LAUNCH_OK();
   return AB_OK;
 }
@@ -939,8 +991,7 @@ int chain_tc_forward(const void* x, const void* A, const void* B, void* y, void*
   if (!ws || ws_bytes < 256) return AB_ERR_WORKSPACE;
   if (T_save && !aligned(T_save, 16)) return AB_ERR_INVALID_ARG;
   int* status = static_cast<int*>(ws);
-  AB_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
-  return launch_row_chain(x, N, n, B, ldB, A, ldA, m, y, T_save, r, status, st);
+  return launch_row_chain(x, N, n, B, ldB, A, ldA, m, y, T_save, r, status, true, st);
 }
 
 int chain_tc_backward(const void* x, const void* dY, const void* A, const void* B,
@@ -953,22 +1004,24 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
   if ((dX && !aligned(dX, 16)) || (T_saved && !aligned(T_saved, 16)) || (dA && !aligned(dA, 16)) ||
       (dB && !aligned(dB, 16)))
     return AB_ERR_INVALID_ARG;
-  AB_CUDA_OK(cudaMemsetAsync(w.status, 0, sizeof(int), st));
+  bool first = true;     // the first kernel of the call zeroes the status word
   const bf16* T = static_cast<const bf16*>(T_saved);
   if (dA && !T) {   // recompute T = x B^T (first product only)
-    AB_TRY(launch_row_chain(x, N, n, B, ldB, nullptr, 0, 0, nullptr, w.T, r, w.status, st));
+    AB_TRY(launch_row_chain(x, N, n, B, ldB, nullptr, 0, 0, nullptr, w.T, r, w.status, first, st));
+    first = false;
     T = w.T;
   }
   if (dX || dB) {
     {
       const int nA = ((m + 31) / 32) * ((r + 31) / 32);
       const int nB = dX ? ((r + 31) / 32) * ((n + 31) / 32) : 0;
-      transpose_factors_kernel<<<nA + nB, 256, 0, st>>>(static_cast<const bf16*>(A), m, r, ldA, w.At, nA,
-                                                        static_cast<const bf16*>(B), n, ldB, w.Bt);
+      AB_LAUNCH_DEP(transpose_factors_kernel, dim3(nA + nB), dim3(256), 0, st, static_cast<const bf16*>(A), m, r, ldA, w.At,
+                 nA, static_cast<const bf16*>(B), n, ldB, w.Bt, first ? w.status : static_cast<int*>(nullptr));
       AB_LAUNCH_OK();
+      first = false;
     }
     // dT = dY A (kept for dB), dX = dT B
-    AB_TRY(launch_row_chain(dY, N, m, w.At, m, w.Bt, r, n, dX, dB ? w.dT : nullptr, r, w.status, st));
+    AB_TRY(launch_row_chain(dY, N, m, w.At, m, w.Bt, r, n, dX, dB ? w.dT : nullptr, r, w.status, false, st));
   }
   if (dA || dB) {
     GradPlan gp = grad_plan(N, m, n, r);
@@ -990,18 +1043,21 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
     }
     if (nj == 1) { tmAct[1] = tmAct[0]; tmSmall[1] = tmSmall[0]; p.job[1] = p.job[0]; p.job[1].chunks = 0; }
     p.njobs = nj; p.r = rp; p.natoms = gp.natoms; p.ns = gp.ns; p.slot_bytes = gp.slot_bytes;
-    p.slices = gp.slices; p.rows_per_slice = gp.rows_per_slice; p.N = (int)N; p.status = w.status;
+    p.slices = gp.slices; p.rows_per_slice = gp.rows_per_slice; p.N = (int)N; p.clear_status = first ? 1 : 0; p.status = w.status;
     AB_CUDA_OK(cudaFuncSetAttribute(grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gp.smem));
     const unsigned grid = (unsigned)((p.job[0].chunks + p.job[1].chunks) * gp.slices);
-    grad_kernel<<<grid, 192, gp.smem, st>>>(tmAct[0], tmSmall[0], tmAct[1], tmSmall[1], p);
+    AB_LAUNCH_DEP(grad_kernel, dim3(grid), dim3(192), gp.smem, st, tmAct[0], tmSmall[0], tmAct[1], tmSmall[1], p);
     AB_LAUNCH_OK();
     {
       const int nA = dA ? (int)(((int64_t)m * r / 4 + 255) / 256) : 0;
       const int nB = dB ? ((n + 31) / 32) * ((r + 31) / 32) : 0;
-      reduce_partials_kernel<<<nA + nB, 256, 0, st>>>(w.pA, dA, m, nA, w.pB, dB, n, gp.slices, r, rp);
+      AB_LAUNCH_DEP(reduce_partials_kernel, dim3(nA + nB), dim3(256), 0, st, static_cast<const float*>(w.pA), dA, m, nA,
+                 static_cast<const float*>(w.pB), dB, n, gp.slices, r, rp);
       AB_LAUNCH_OK();
     }
+    first = false;
   }
+  if (first) AB_CUDA_OK(cudaMemsetAsync(w.status, 0, sizeof(int), st));   // nothing was asked for
   return AB_OK;
 }
 

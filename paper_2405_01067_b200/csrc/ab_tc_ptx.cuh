@@ -51,6 +51,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   }
 }
 
+// Programmatic dependent launch.  A kernel launched with the stream-serialisation attribute may become
+// resident while the kernel before it in the stream is still running; dep_wait() returns once that
+// kernel has completed and its writes are visible (a no-op for a launch without the attribute), so
+// everything above it -- barrier set-up, TMEM allocation, descriptor prefetch -- overlaps the tail of
+// the previous kernel.  dep_launch() lets the next kernel in the stream do the same with this one.
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void named_bar_sync(int id, int threads) {
