@@ -112,6 +112,8 @@ size_t ab_static_scratch_elems(void);
  *   Any of dX, dA, dB may be NULL (not wanted: groups that train only A or only B).
  *   T_saved: the T written by ab_layer_forward, or NULL to recompute it from x.
  *   Sums over N are taken in a fixed order: two runs give identical bits.
+ *   No output may overlap an input or another output (the kernels of one call run partly side
+ *   by side: dA is accumulated from dY and T while dX is still being written).
  */
 int ab_layer_backward(const void* x, const void* dY, const void* A, const void* B,
                       const void* T_saved, void* dX, float* dA, float* dB,

@@ -573,6 +573,7 @@ struct GradParams {
   int slices, rows_per_slice;   // rows_per_slice is a multiple of 64
   int N;
   int clear_status;
+  int job0_independent;   // 1: job 0 reads nothing the kernel before this one in the stream writes (see grad_kernel)
   int* status;
 };
 
@@ -613,7 +614,12 @@ grad_kernel(const __grid_constant__ CUtensorMap tmAct0, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
-  dep_wait();            // nothing above touches global memory
+  // In a full backward the kernel before this one is the dT/dX chain, which writes dT and dX: the dB
+  // job reads dT and has to wait for it, the dA job reads only dY and T.  This kernel becomes resident
+  // only after every CTA of the chain kernel has passed its own dep_wait, i.e. after everything
+  // earlier in the stream (T included) is complete, so the dA CTAs start at once on the SMs that the
+  // chain kernel's short CTAs have already left (its last third runs on two thirds of the SMs).
+  if (!(p.job0_independent && jb == 0)) dep_wait();
   dep_launch();
   clear_status_word(p.clear_status, p.status);
 
@@ -1005,6 +1011,7 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
       (dB && !aligned(dB, 16)))
     return AB_ERR_INVALID_ARG;
   bool first = true;     // the first kernel of the call zeroes the status word
+  bool after_chain = false;   // the dT/dX chain kernel is the launch right before the gradient kernel
   const bf16* T = static_cast<const bf16*>(T_saved);
   if (dA && !T) {   // recompute T = x B^T (first product only)
     AB_TRY(launch_row_chain(x, N, n, B, ldB, nullptr, 0, 0, nullptr, w.T, r, w.status, first, st));
@@ -1022,6 +1029,7 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
     }
     // dT = dY A (kept for dB), dX = dT B
     AB_TRY(launch_row_chain(dY, N, m, w.At, m, w.Bt, r, n, dX, dB ? w.dT : nullptr, r, w.status, false, st));
+    after_chain = true;
   }
   if (dA || dB) {
     GradPlan gp = grad_plan(N, m, n, r);
@@ -1044,6 +1052,7 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
     if (nj == 1) { tmAct[1] = tmAct[0]; tmSmall[1] = tmSmall[0]; p.job[1] = p.job[0]; p.job[1].chunks = 0; }
     p.njobs = nj; p.r = rp; p.natoms = gp.natoms; p.ns = gp.ns; p.slot_bytes = gp.slot_bytes;
     p.slices = gp.slices; p.rows_per_slice = gp.rows_per_slice; p.N = (int)N; p.clear_status = first ? 1 : 0; p.status = w.status;
+    p.job0_independent = (after_chain && dA) ? 1 : 0;   // job 0 is the dA job whenever dA is asked for
     AB_CUDA_OK(cudaFuncSetAttribute(grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gp.smem));
     const unsigned grid = (unsigned)((p.job[0].chunks + p.job[1].chunks) * gp.slices);
     AB_LAUNCH_DEP(grad_kernel, dim3(grid), dim3(192), gp.smem, st, tmAct[0], tmSmall[0], tmAct[1], tmSmall[1], p);
