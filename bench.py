@@ -34,9 +34,9 @@ NOMINAL_BF16_TFLOPS = 2250.0
 R = 192
 LAYERS = ((3072, 768), (768, 3072))
 K_GROUPS = 4
-# dram__bytes_read.sum + dram__bytes_write.sum of one row_chain_kernel launch (forward, 50,432 rows),
+# dram__bytes_read.sum + dram__bytes_write.sum of one row_chain_units_kernel launch (forward, 50,432 rows),
 # from the ncu capture summarised under profiles/; None until the kernel of that capture is current.
-ROW_CHAIN_DRAM_BYTES_PER_LAUNCH = 349.2e6   # forward of W1: 79.4 MB read + 269.9 MB written (ncu capture under profiles/)
+ROW_CHAIN_DRAM_BYTES_PER_LAUNCH = 349.8e6   # forward of W1: 79.4 MB read + 270.4 MB written (ncu capture under profiles/)
 
 
 def chain_flops(N, layers=LAYERS, r=R):

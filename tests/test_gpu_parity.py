@@ -121,6 +121,34 @@ def test_backward_optional_outputs_and_determinism(ab):
         assert torch.equal(a, b)       # fixed reduction order: identical bits
 
 
+def test_backward_back_to_back_on_one_workspace(ab):
+    """The kernels of consecutive calls overlap at their boundaries (a kernel's set-up runs during the tail
+    of the one before it, and dA starts while dX is still being written).  Calls queued back to back on
+    one stream and one workspace, with different inputs and T rebuilt inside the call, must give the bits
+    of the same calls run one at a time with a synchronisation in between."""
+    N, m, n, r = 148 * 128 * 2 + 1000, 512, 256, 64        # more 128-row blocks than SMs, ragged tail
+    cases = [synth.chain_case(20 + i, m, n, r, N, bf16=True) for i in range(2)]
+    ins = [tuple(dev(d[k], True) for k in ("x", "dY", "A", "B")) for d in cases]
+    ws = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_BACKWARD, N, m, n, r, 1, ab.AB_BF16), "cuda")
+    alone = []
+    for x, dY, A, B in ins:
+        alone.append(ab.ab_layer_backward(x, dY, A, B, ws=ws))
+        torch.cuda.synchronize()
+    queued = []
+    for rep in range(3):
+        for x, dY, A, B in ins:
+            queued.append(ab.ab_layer_backward(x, dY, A, B, ws=ws))
+    torch.cuda.synchronize()
+    assert ab.workspace_status(ws) == 0
+    for i, got in enumerate(queued):
+        for a, b in zip(alone[i % 2], got):
+            assert torch.equal(a, b)
+    d = cases[0]
+    dA_ref, dB_ref = _oracle_backward_chunked(d["x"], d["dY"], d["A"], d["B"])
+    assert orc.rel_frob(host(alone[0][1]), dA_ref) <= TOL_BF16
+    assert orc.rel_frob(host(alone[0][2]), dB_ref) <= TOL_BF16
+
+
 def test_empty_batch(ab):
     A = torch.randn(8, 2, device="cuda")
     B = torch.randn(2, 6, device="cuda")
