@@ -482,6 +482,16 @@ def run_ours(args):
     if int(plan.status.abs().sum().item()) != 0:
         raise SystemExit("group sync reported a device-side error status")
 
+    # the chain alone, steps queued back to back (as between two synchronisations of a training cycle)
+    barrier()
+    b0, b1 = ev(), ev()
+    b0.record()
+    for _ in range(args.steps):
+        chain()
+    b1.record()
+    barrier()
+    b2b_ms = b0.elapsed_time(b1)
+
     # end to end: inputs start in pinned host memory, results end there
     for _ in range(2):
         e2e_step()
@@ -500,8 +510,8 @@ def run_ours(args):
     barrier()
     e2e_sync_ms = e0.elapsed_time(e1)
 
-    total_ms, chain_ms, sync_ms, e2e_ms, e2e_sync_ms = max_over_ranks(
-        [total_ms, chain_ms, sync_ms, e2e_ms, e2e_sync_ms], "cuda", world)
+    total_ms, chain_ms, sync_ms, e2e_ms, e2e_sync_ms, b2b_ms = max_over_ranks(
+        [total_ms, chain_ms, sync_ms, e2e_ms, e2e_sync_ms, b2b_ms], "cuda", world)
     sampler.join(timeout=2.0)
     if rank == 0:
         pk = measured_peaks()
@@ -535,6 +545,8 @@ def run_ours(args):
                                 l2="inputs larger than L2 (about 0.8 GB of activations read per step)"),
                     chain_ms_per_step=chain_ms / K, chain_ms_median=chain_each[len(chain_each) // 2],
                     chain_ms_min=chain_each[0], group_sync_ms_per_step=sync_ms / K,
+                    chain_back_to_back=dict(ms_per_step=b2b_ms / K, tflops=flops_step * K / (b2b_ms * 1e-3) / 1e12,
+                                            note="chain steps queued one after the other, no group sync between them"),
                     pct_of_nominal_bf16_peak=100.0 * per_gpu / NOMINAL_BF16_TFLOPS,
                     e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                              ms_per_step=e2e_ms / K, ms_per_step_with_group_sync=e2e_sync_ms / K),
