@@ -561,7 +561,7 @@ def run_ours(args):
             line["other_workloads"] = other_workloads(ab, torch)
             line["adamw_update_vit_factors"] = optimizer_step(ab, torch)
         if world == 1 and not args.no_cpu_baseline:
-            cb = cpu_baseline(inputs, min(N, args.ref_rows))
+            cb = cpu_baseline(inputs, min(N, args.baseline_rows), sync_scale=4)    # about 10 s of host work
             line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
         print(json.dumps(line))
     if world > 1:
@@ -575,7 +575,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=256 * 197, help="token rows per layer (default: batch 256 x 197)")
-    ap.add_argument("--ref-rows", type=int, default=8192, help="rows of the CPU checker's bounded sample")
+    ap.add_argument("--ref-rows", type=int, default=8192,
+                    help="rows of the CPU checker's bounded sample per step of --impl reference")
+    ap.add_argument("--baseline-rows", type=int, default=32768,
+                    help="rows of the CPU checker's bounded sample timed once beside the GPU run (cpu_baseline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-model-sync", action="store_true", help="skip the full-ViT group-sync measurement")
     ap.add_argument("--no-other-workloads", action="store_true",
