@@ -394,6 +394,8 @@ int launch_jacobi(const JacobiJob* jobs, int count, int rmax, float tol, cudaStr
   return launch_jacobi_el<8>(jobs, count, rmax, tol, st);
 }
 
+constexpr int kCPanel = 8;       // rows per panel of the Cholesky elimination (kCThreads / 64)
+
 struct CholJob {
   const float* G;   // nparts partial sums of an r x r symmetric positive semi-definite matrix (row stride r,
                     // r * r apart); only the upper triangle is read
@@ -417,10 +419,18 @@ __global__ void __launch_bounds__(kCThreads, 1) chol_inv_kernel(const CholJob* _
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = kCThreads / 32;
 
   if (tid == 0) maxdiag = 0.f;
-  for (int idx = tid; idx < r * r; idx += kCThreads) {
-    float v = job.G[idx];
-    for (int q = 1; q < job.nparts; ++q) v += job.G[(size_t)q * r * r + idx];      // ascending part order
-    S[(idx / r) * ld + idx % r] = v;
+  {
+    const float* __restrict__ G = job.G;
+    const size_t part = (size_t)r * r;
+    for (int i = warp; i < r; i += nwarps) {           // one row per warp; the loads of a row are all in flight
+      const float* g = G + (size_t)i * r;
+#pragma unroll 8
+      for (int k = lane; k < r; k += 32) {
+        float v = g[k];
+        for (int q = 1; q < job.nparts; ++q) v += g[q * part + k];                 // ascending part order
+        S[i * ld + k] = v;
+      }
+    }
   }
   __syncthreads();
   for (int i = tid; i < r; i += kCThreads)
@@ -428,17 +438,40 @@ __global__ void __launch_bounds__(kCThreads, 1) chol_inv_kernel(const CholJob* _
   __syncthreads();
   const float cut = kEigThr * maxdiag;
 
-  for (int j = 0; j < r; ++j) {
-    const float dj = S[j * ld + j];
-    const bool live = dj > cut && dj > 0.f;
-    const float inv = live ? 1.f / sqrtf(dj) : 0.f;
-    for (int k = j + 1 + tid; k < r; k += kCThreads) S[j * ld + k] *= inv;     // a dropped row becomes zero
-    __syncthreads();
-    if (tid == 0) { S[j * ld + j] = dj * inv; dinv[j] = inv; }                  // nobody reads the pivot below
-    for (int i = j + 1 + warp; i < r; i += nwarps) {
-      const float f = S[j * ld + i];
-      if (f != 0.f)
-        for (int k = i + lane; k < r; k += 32) S[i * ld + k] = fmaf(-f, S[j * ld + k], S[i * ld + k]);
+  // Panels of kCPanel rows: inside a panel the rows are finished one after the other (scale row j,
+  // subtract it from the few panel rows below it), then all rows below the panel take the panel's
+  // kCPanel rank-one terms in one pass, in ascending j -- the same sums per entry as a column-by-column
+  // elimination, with one long step per panel instead of one per column.
+  for (int j0 = 0; j0 < r; j0 += kCPanel) {
+    const int jend = (j0 + kCPanel < r) ? j0 + kCPanel : r;
+    for (int j = j0; j < jend; ++j) {
+      const float dj = S[j * ld + j];
+      const bool live = dj > cut && dj > 0.f;
+      const float inv = live ? 1.f / sqrtf(dj) : 0.f;
+      for (int k = j + 1 + tid; k < r; k += kCThreads) S[j * ld + k] *= inv;   // a dropped row becomes zero
+      __syncthreads();
+      if (tid == 0) { S[j * ld + j] = dj * inv; dinv[j] = inv; }                // nobody reads the pivot below
+      {                                              // panel rows still open: 64 threads per row
+        const int i = j + 1 + (tid >> 6);
+        if (i < jend) {
+          const float f = S[j * ld + i];
+          for (int k = i + (tid & 63); k < r; k += 64) S[i * ld + k] = fmaf(-f, S[j * ld + k], S[i * ld + k]);
+        }
+      }
+      __syncthreads();
+    }
+    const int np = jend - j0;
+    for (int i = jend + warp; i < r; i += nwarps) {
+      float f[kCPanel];
+#pragma unroll
+      for (int q = 0; q < kCPanel; ++q) f[q] = (q < np) ? S[(j0 + q) * ld + i] : 0.f;
+      for (int k = i + lane; k < r; k += 32) {
+        float acc = S[i * ld + k];
+#pragma unroll
+        for (int q = 0; q < kCPanel; ++q)
+          if (q < np) acc = fmaf(-f[q], S[(j0 + q) * ld + k], acc);
+        S[i * ld + k] = acc;
+      }
     }
     __syncthreads();
   }
