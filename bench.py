@@ -155,7 +155,10 @@ def run_reference(args):
     line = dict(impl="reference", metric=METRIC, value=v, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=dt * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="f64", data="synthetic",
-                config=dict(workload="vit_b16_mlp_pair_r192 (bounded sample)", rows=rows, K=K_GROUPS, r=R),
+                config=dict(workload="vit_b16_mlp_pair_r192 (bounded sample)", rows=rows, K=K_GROUPS, r=R,
+                            same_config=False,
+                            sample=f"first {rows} of 50432 rows of both layers per step (a rate: FLOP of the sample "
+                                   "over its time); the GPU arm runs all 50432 rows"),
                 cpu_baseline=dict(value=v, unit=UNIT, cores=last["cores"], kind="oracle", sample=last["sample"]),
                 e2e=dict(value=v, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
     print(json.dumps(line))
@@ -281,10 +284,10 @@ def other_workloads(ab, torch, iters=10):
         flop = 6.0 * N * r * (m + n)
         nbytes = (2.0 if bf16 else 4.0) * N * (3 * n + 2 * m)
         tf = flop / (ms * 1e-3) / 1e12
-        ceil_tf = min(pk["tc_sustained"], flop / nbytes * pk["hbm"] / 1e3)
+        ceil_tf = min(pk["tc_burst"], flop / nbytes * pk["hbm"] / 1e3)
         return dict(N=N, m=m, n=n, r=r, ms=ms, tflops=tf, algorithmic_gbs=nbytes / (ms * 1e-3) / 1e9,
                     ceiling_tflops=ceil_tf, frac_of_ceiling=tf / ceil_tf,
-                    bound="hbm" if ceil_tf < pk["tc_sustained"] else "tensor")
+                    bound="hbm" if ceil_tf < pk["tc_burst"] else "tensor")
 
     out = {}
     d = synth.resnet_conv(2)
@@ -303,6 +306,34 @@ def other_workloads(ab, torch, iters=10):
     d["A"], d["B"] = A.cpu().numpy(), B.cpu().numpy()
     one = layer(d, False)
     out["linear_256x512_fp32_r32"] = dict(N=one["N"], us_fwd_bwd=one["ms"] * 1e3, note="launch-latency bound")
+    return out
+
+
+def dense_split_times(ab, torch, iters=3):
+    """The decomposition Algorithm 1 runs after the full-rank rebound phase: W is dense and no longer of rank
+    <= r, so the factored route does not apply.  ab_svd_split (r_max 192, fixed rank) of one matrix of each
+    ViT-B/16 shape, W = 0.02 G + P diag(0.9^i) Q^T, event-timed; LAPACK's float64 time on the host beside it."""
+    from paper_2405_01067_b200 import synth
+    out = {}
+    w = synth.vit_mlp_weights(seed=1)
+    st = synth.streams(11, ["g", "p"])
+    sq = synth.normal(st["g"], (768, 768), 0.02) + synth.planted_matrix(st["p"], 768, 768, 0.9 ** np.arange(768))
+    for name, W in (("768x768", sq), ("3072x768", w["W1"]), ("768x3072", w["W2"])):
+        Wd = torch.from_numpy(W).cuda()
+        m, n = W.shape
+        ws = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_SVD_SPLIT, 0, m, n, 192, 1, ab.AB_F32), "cuda")
+        res = ab.ab_svd_split(Wd, 192, 0.0, ws=ws)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            res = ab.ab_svd_split(Wd, 192, 0.0, ws=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        np.linalg.svd(W.astype(np.float64), full_matrices=False)
+        out[name] = dict(ms=e0.elapsed_time(e1) / iters, device_status=int(res[4].item()),
+                         lapack_f64_host_ms=(time.perf_counter() - t0) * 1e3)
     return out
 
 
@@ -527,16 +558,28 @@ def run_ours(args):
         # it; backward launches it once more).  Algorithmic work of a forward launch: 2 N r (m+n) FLOP
         # (both layers have m+n = 3840), 2 N (m+n) bytes.
         fwd_flops = 2.0 * N * R * 3840
+        fwd_bytes = 2.0 * N * 3840
         fwd_tflops = fwd_flops / (fwd_ms * 1e-3) / 1e12
-        roof = dict(bound="tensor", kernel="row_chain_units_kernel (one launch = ab_layer_forward of one layer at this size)",
-                    achieved=fwd_tflops, peak=pk["tc_sustained"], unit="TFLOP/s", frac=fwd_tflops / pk["tc_sustained"],
-                    traffic=ROW_CHAIN_DRAM_BYTES_PER_LAUNCH, us_per_launch=fwd_ms * 1e3,
-                    peak_source=f"bf16_tflops_sustained of {pk['source']}",
-                    frac_of_nominal_2250=fwd_tflops / NOMINAL_BF16_TFLOPS,
-                    algorithmic_gbs=2.0 * N * 3840 / (fwd_ms * 1e-3) / 1e9, hbm_peak_gbs=pk["hbm"],
-                    whole_chain=dict(tflops=per_gpu, frac_of_measured=per_gpu / pk["tc_sustained"],
-                                     frac_of_nominal_2250=per_gpu / NOMINAL_BF16_TFLOPS,
-                                     algorithmic_gbs=chain_bytes(N) * K / (chain_ms * 1e-3) / 1e9))
+        fwd_gbs = fwd_bytes / (fwd_ms * 1e-3) / 1e9
+        # which roof binds a forward launch: the tensor peak (burst figure: the launch is timed by itself,
+        # 0.1 ms at full clocks) or its intensity times the HBM peak
+        hbm_ceiling_tflops = fwd_flops / fwd_bytes * pk["hbm"] / 1e3
+        hbm_bound = hbm_ceiling_tflops < pk["tc_burst"]
+        kernel = "row_chain_units_kernel (one launch = ab_layer_forward of one layer at this size)"
+        common = dict(kernel=kernel, traffic=ROW_CHAIN_DRAM_BYTES_PER_LAUNCH, us_per_launch=fwd_ms * 1e3,
+                      tflops=fwd_tflops, algorithmic_gbs=fwd_gbs, hbm_peak_gbs=pk["hbm"], tensor_peak_tflops=pk["tc_burst"],
+                      frac_of_tensor_burst=fwd_tflops / pk["tc_burst"], frac_of_hbm=fwd_gbs / pk["hbm"],
+                      frac_of_nominal_2250=fwd_tflops / NOMINAL_BF16_TFLOPS,
+                      whole_chain=dict(tflops=per_gpu, frac_of_measured_burst=per_gpu / pk["tc_burst"],
+                                       frac_of_nominal_2250=per_gpu / NOMINAL_BF16_TFLOPS,
+                                       algorithmic_gbs=chain_bytes(N) * K / (chain_ms * 1e-3) / 1e9,
+                                       frac_of_hbm=chain_bytes(N) * K / (chain_ms * 1e-3) / 1e9 / pk["hbm"]))
+        if hbm_bound:
+            roof = dict(bound="hbm", achieved=fwd_gbs, peak=pk["hbm"], unit="GB/s", frac=fwd_gbs / pk["hbm"],
+                        peak_source=f"hbm_gbs of {pk['source']}", **common)
+        else:
+            roof = dict(bound="tensor", achieved=fwd_tflops, peak=pk["tc_burst"], unit="TFLOP/s",
+                        frac=fwd_tflops / pk["tc_burst"], peak_source=f"bf16_tflops (burst) of {pk['source']}", **common)
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=K, warmup=args.warmup,
                     ms_per_step=total_ms / K, higher_is_better=True, scaling="weak", vs_baseline=None,
                     dtype="bf16", data="synthetic",
@@ -560,12 +603,26 @@ def run_ours(args):
         if world == 1 and not args.no_other_workloads:
             line["other_workloads"] = other_workloads(ab, torch)
             line["adamw_update_vit_factors"] = optimizer_step(ab, torch)
+            line["dense_split_ms"] = dense_split_times(ab, torch)
         if world == 1 and not args.no_cpu_baseline:
             cb = cpu_baseline(inputs, min(N, args.baseline_rows), sync_scale=4)    # about 10 s of host work
             line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def spawn_ranks(n):
+    """`python bench.py --gpus N` outside torchrun: start the N ranks (one process per GPU, rendezvous on
+    127.0.0.1) with the same arguments and hand their exit status back.  Rank 0 prints the JSON line."""
+    import socket
+    import subprocess
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -585,6 +642,8 @@ def main():
                     help="skip the ResNet-50 / VGG16 / small fp32 layer measurements")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -8,8 +8,11 @@
  *
  * Conventions for every call
  *  - Pointers are DEVICE pointers owned by the caller unless a parameter says "host".
- *    The library allocates no device memory and keeps no state between calls; scratch
- *    space is passed in as `ws` (size from ab_workspace_bytes, 256-byte aligned).
+ *    The library allocates no device memory; scratch space is passed in as `ws` (size from
+ *    ab_workspace_bytes, 256-byte aligned).  No result depends on an earlier call.  What the
+ *    library does keep per process: a count of its kernel launches (ab_launch_count), cached
+ *    device properties, the address of the built-in array of ab_layer_forward_static, and one
+ *    low-priority helper stream per device that ab_group_sync creates on first use (see there).
  *  - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
  *    default stream).  Buffers must stay valid until the stream has run the call.
  *  - Arguments that can be checked on the host (NULL, non-positive sizes, r > min(m,n),
@@ -58,6 +61,15 @@ const char* ab_version(void);
 
 /* Number of kernels this library has launched in this process since it was loaded. */
 long long ab_launch_count(void);
+
+/*
+ * Self-test of the failure path (no counterpart in the paper).  Every on-chip wait of the fused kernels
+ * is bounded: when it runs out the kernel writes AB_ERR_TIMEOUT to its status word and exits normally.
+ * This call launches one small kernel whose only thread waits, with the same wait routine, on a barrier
+ * that nothing ever signals, for limit_us microseconds (1 .. 1,000,000); dev_status (device int) then
+ * holds AB_ERR_TIMEOUT.  Nothing hangs, traps or faults; the context stays usable.
+ */
+int ab_selftest_bounded_wait(int* dev_status, unsigned limit_us, void* cuda_stream);
 
 /*
  * Scratch bytes a call needs (0 if none).  Arguments a given op does not use are ignored

@@ -18,8 +18,9 @@ What each function follows:
 
 Pins (tests/test_oracle_*.py): finite differences, the dense restatement,
 Eckart-Young, exact recovery at rank <= r, closed-form singular values,
-LAPACK, planted spectra, bit-level properties of the fixed-order fp32 mean.
-No function here is "parity unpinned".
+LAPACK, planted spectra, bit-level properties of the fixed-order fp32 mean,
+hand-computed values of the two error yardsticks (``rel_frob``,
+``max_tile_rel_frob``).  No function here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -187,12 +188,6 @@ def svd_split(W, r_max, sigma_cutoff=0.0):
     return A, B, s, r
 
 
-def truncate(W, r):
-    """Best rank-r approximation of W in the Frobenius norm (via ``jacobi_svd``)."""
-    U, s, Vt, _ = jacobi_svd(W)
-    return (U[:, :r] * s[None, :r]) @ Vt[:r]
-
-
 # ------------------------------------------------------------------ whole step
 
 def group_sync(A_copies, B_copies, r_max, sigma_cutoff):
@@ -232,3 +227,29 @@ def rel_frob(a, b):
     den = np.linalg.norm(b)
     num = np.linalg.norm(a - b)
     return 0.0 if num == 0.0 else num / den
+
+
+def max_tile_rel_frob(a, b, tile_rows=128, tile_cols=64):
+    """Largest relative Frobenius error over the tiles of a grid laid on the matrices:
+    max over tiles of ||a_tile - b_tile||_F / max(||b_tile||_F, floor), where the floor is the norm a tile
+    of that size would have at 1e-3 of b's root-mean-square value (so that a tile of b that happens to be
+    all zeros does not divide by zero).  A wrong tile cannot hide behind the norm of the whole matrix."""
+    a, b = _f64(a), _f64(b)
+    if b.size == 0:
+        return 0.0
+    rms = np.sqrt(np.mean(b * b))
+    ri = np.arange(0, b.shape[0], tile_rows)
+    ci = np.arange(0, b.shape[1], tile_cols)
+
+    def tile_sums(sq):          # sum of the entries of every tile
+        return np.add.reduceat(np.add.reduceat(sq, ri, axis=0), ci, axis=1)
+
+    num = np.sqrt(tile_sums((a - b) ** 2))
+    den = np.sqrt(tile_sums(b * b))
+    sizes = np.outer(np.diff(np.append(ri, b.shape[0])), np.diff(np.append(ci, b.shape[1])))
+    den = np.maximum(den, 1e-3 * rms * np.sqrt(sizes))
+    with np.errstate(divide="ignore", invalid="ignore"):
+        rel = np.where(num > 0.0, num / den, 0.0)
+    worst = rel.max()
+    return float(worst)
+

@@ -23,7 +23,7 @@ AB_SYNC_AUTO, AB_SYNC_DENSE, AB_SYNC_FACTORED = 0, 1, 2
 
 EXPORTS = ["ab_status_string", "ab_version", "ab_launch_count", "ab_workspace_bytes", "ab_layer_forward", "ab_layer_backward",
            "ab_group_average", "ab_recombine", "ab_svd_split", "ab_group_sync", "ab_sync_workspace_bytes",
-           "ab_layer_forward_static", "ab_static_scratch_elems", "ab_adamw_step", "ab_lr_rebound_factor"]
+           "ab_layer_forward_static", "ab_static_scratch_elems", "ab_adamw_step", "ab_lr_rebound_factor", "ab_selftest_bounded_wait"]
 
 
 class AbError(RuntimeError):
@@ -79,8 +79,18 @@ def lib() -> ctypes.CDLL:
     L.ab_adamw_step.argtypes = [c_void_p] * 5 + [c_int64] + [c_float] * 5 + [c_int, c_void_p]
     L.ab_lr_rebound_factor.restype = c_float
     L.ab_lr_rebound_factor.argtypes = [c_int, c_int, c_float]
+    L.ab_selftest_bounded_wait.restype = c_int
+    L.ab_selftest_bounded_wait.argtypes = [c_void_p, ctypes.c_uint, c_void_p]
     _lib = L
     return L
+
+
+def ab_selftest_bounded_wait(limit_us: int = 1000, stream=None) -> int:
+    """Runs the bounded-wait self-test and returns the device status it left (AB_ERR_TIMEOUT when the wait
+    gave up as designed).  Synchronises."""
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    _check(lib().ab_selftest_bounded_wait(_ptr(status), int(limit_us), _stream(stream)), "ab_selftest_bounded_wait")
+    return int(status.item())
 
 
 def ab_launch_count() -> int:

@@ -10,6 +10,20 @@ namespace ab {
 static std::atomic<long long> g_launches{0};
 void count_launches(long long n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+int sm_count() {
+  static std::atomic<int> cache[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (dev >= 0 && dev < 64) {
+    const int c = cache[dev].load(std::memory_order_relaxed);
+    if (c > 0) return c;
+  }
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  if (dev >= 0 && dev < 64) cache[dev].store(sms, std::memory_order_relaxed);
+  return sms;
+}
+
 namespace {
 
 template <typename TI, typename TO>
@@ -20,7 +34,8 @@ __global__ void cast_kernel(const TI* __restrict__ in, TO* __restrict__ out, int
 
 int cast_f32_to(const float* in, void* out, int dt, int64_t count, cudaStream_t st) {
   if (count == 0) return AB_OK;
-  unsigned grid = (unsigned)((count + 255) / 256 < 148 * 8 ? (count + 255) / 256 : 148 * 8);
+  const int64_t cap = (int64_t)(sm_count() > 0 ? sm_count() : 1) * 8;
+  unsigned grid = (unsigned)((count + 255) / 256 < cap ? (count + 255) / 256 : cap);
   if (dt == AB_F32) cast_kernel<float, float><<<grid, 256, 0, st>>>(in, static_cast<float*>(out), count);
   else cast_kernel<float, bf16><<<grid, 256, 0, st>>>(in, static_cast<bf16*>(out), count);
   AB_LAUNCH_OK();
@@ -130,6 +145,12 @@ size_t ab_workspace_bytes(int op, int64_t N, int m, int n, int r, int K, int dt)
     }
     default: return 0;
   }
+}
+
+int ab_selftest_bounded_wait(int* dev_status, unsigned limit_us, void* cuda_stream) {
+  if (!dev_status || limit_us == 0 || limit_us > 1000000u) return AB_ERR_INVALID_ARG;
+  if (!have_device()) return AB_ERR_CUDA;
+  return bounded_wait_selftest(dev_status, limit_us, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int ab_layer_forward(const void* x, const void* A, const void* B, void* y, void* T_save,

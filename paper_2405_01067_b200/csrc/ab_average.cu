@@ -139,7 +139,7 @@ int run(const void* base_, int64_t stride, int K, int64_t count, void* out_, cud
   const float inv = 1.0f / (float)K;
   const bool vec_ok = aligned(base, 16) && aligned(out, 16) && (stride % V == 0);
   int64_t nvec = vec_ok ? count / V : 0;
-  int sms = 148;
+  const int sms = sm_count() > 0 ? sm_count() : 1;
   if (nvec > 0) {
     int64_t blocks = (nvec + 255) / 256;
     int64_t cap = (int64_t)1 << 30;          // beyond that the kernel's stride loop takes over

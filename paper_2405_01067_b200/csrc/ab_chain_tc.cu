@@ -772,6 +772,20 @@ __global__ void transpose_factors_kernel(const bf16* __restrict__ A, int m, int 
   }
 }
 
+// Self-test of the bounded wait every pipeline stage of the kernels above relies on: one thread waits on
+// an mbarrier that nobody ever arrives at.  The wait gives up after limit_ns and the kernel reports
+// AB_ERR_TIMEOUT through the status word, exactly as the chain kernels do; nothing spins for ever and the
+// context stays usable.
+__global__ void bounded_wait_selftest_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) *status = mbar_wait(&bar, 0, limit_ns) ? (int)AB_OK : (int)AB_ERR_TIMEOUT;
+}
+
 // ---------------------------------------------------------------------------------------------
 // host side
 // Launch with programmatic stream serialisation (see dep_wait): only for kernels that call dep_wait()
@@ -879,14 +893,6 @@ UnitPlan unit_plan(int r) {    // r: padded rank
   return pl;
 }
 
-int sm_count() {
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return 0;
-  return sms;
-}
-
 struct GradPlan { int natoms, ns, slot_bytes, slices, rows_per_slice; size_t smem; };
 GradPlan grad_plan(int64_t N, int m, int n, int r) {
   GradPlan pl;
@@ -897,7 +903,7 @@ GradPlan grad_plan(int64_t N, int m, int n, int r) {
   if (pl.ns > kMaxStages) pl.ns = kMaxStages;
   pl.smem = (size_t)fixed + (size_t)pl.ns * pl.slot_bytes;
   const int tiles = (m + 255) / 256 + (n + 255) / 256;
-  int slices = 148 / tiles;
+  int slices = (sm_count() > 0 ? sm_count() : 1) / tiles;   // one wave of CTAs
   if (slices < 1) slices = 1;
   const int64_t slabs = (N + 63) / 64;
   if (slices > slabs) slices = (int)slabs;
@@ -973,6 +979,12 @@ int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1
 }
 
 }  // namespace
+
+int bounded_wait_selftest(int* dev_status, unsigned limit_us, cudaStream_t st) {
+  bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(dev_status, (unsigned long long)limit_us * 1000ull);
+  AB_LAUNCH_OK();
+  return AB_OK;
+}
 
 bool chain_tc_supported(int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
                         const void* x, const void* A, const void* B, const void* y) {

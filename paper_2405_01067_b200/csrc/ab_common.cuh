@@ -36,6 +36,10 @@ void count_launches(long long n);
     if (_s != AB_OK) return _s;                            \
   } while (0)
 
+// Multiprocessors of the current device (cached per device; 0 if the query fails).  Grid sizes that are
+// meant to fill the GPU are derived from it.
+int sm_count();
+
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static inline size_t dtype_size(int dt) { return dt == AB_BF16 ? 2 : 4; }
 static inline bool dtype_ok(int dt) { return dt == AB_F32 || dt == AB_BF16; }
@@ -101,6 +105,8 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
                       const void* T_saved, void* dX, float* dA, float* dB,
                       int64_t N, int m, int n, int r, int ldA, int ldB,
                       void* ws, size_t ws_bytes, cudaStream_t st);
+
+int bounded_wait_selftest(int* dev_status, unsigned limit_us, cudaStream_t st);
 
 // ---- SVD pipeline (ab_svd.cu) ------------------------------------------------------------------
 struct SvdItem {

@@ -51,7 +51,8 @@ int ab_layer_forward_static(const void* x, const void* A, const void* B, void* y
   if (!dtype_ok(dt)) return AB_ERR_INVALID_ARG;
   if (N < 0 || m <= 0 || n <= 0 || r <= 0 || r > m || r > n || ldA < r || ldB < n) return AB_ERR_INVALID_ARG;
   if (!A || !B || (N > 0 && (!x || !y))) return AB_ERR_INVALID_ARG;
-  if ((uint64_t)N * (uint64_t)r > kStaticScratchElems) return AB_ERR_UNSUPPORTED;   // N*r beyond the built-in scratch
+  // N*r beyond the built-in scratch (by division: the product of two unchecked arguments could wrap)
+  if ((uint64_t)N > kStaticScratchElems / (uint64_t)r) return AB_ERR_UNSUPPORTED;
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev <= 0) return AB_ERR_CUDA;
   if (N == 0) return AB_OK;

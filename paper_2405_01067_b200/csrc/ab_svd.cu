@@ -689,7 +689,7 @@ int svd_batch(const SvdItem* items, int L, float sigma_cutoff, void* ws, size_t 
       int64_t lt = p.tall ? it.r_max : 1, lk = p.tall ? 1 : it.n;
       int64_t sk = p.tall ? it.n : 1, su = p.tall ? 1 : it.r_max;
       int64_t total = (int64_t)(p.L + s) * it.r_max;
-      unsigned grid = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8);
+      unsigned grid = (unsigned)std::min<int64_t>((total + 255) / 256, (int64_t)std::max(sm_count(), 1) * 8);
       if (it.out_dt == AB_F32)
         write_factors_kernel<float><<<grid, 256, 0, stream>>>(w.Y, yt, yk, w.Vr, it.sigma, it.r_out, p.L, s, p.r_cap,
                                                              it.r_max, (float*)Fl, lt, lk, (float*)Fs, sk, su);

@@ -13,7 +13,6 @@
 // for factors truncated by the rank rule (zero columns of A, zero rows of B).  Otherwise the
 // factors need a condition number below about 300 -- all workloads here are far inside.
 #include <algorithm>
-#include <cstdio>
 #include <cstring>
 #include <mutex>
 #include <type_traits>
@@ -295,9 +294,6 @@ jacobi_rows_cluster_kernel(const JacobiJob* __restrict__ jobs, float tol) {
 #pragma unroll
     for (int c = 0; c < kC; ++c) any = max(any, lflag[c]);
     converged = (__int_as_float(any) <= kJEarly2);     // nothing rotated, or only by angles whose square is noise
-#ifdef AB_TRACE_SWEEPS
-    if (crank == 0 && tid == 0) printf("  job %d sweep %d: largest rotated cos^2 %.3e\n", (int)(blockIdx.x / kC), sweeps, __int_as_float(any));
-#endif
   }
 
   // norms, descending order, unit rows: each CTA finishes the rows it holds
@@ -322,9 +318,6 @@ jacobi_rows_cluster_kernel(const JacobiJob* __restrict__ jobs, float tol) {
     if (lane == 0) job.norms[rank[lr]] = nrm;
   }
   if (crank == 0 && tid == 0 && job.status) *job.status = converged ? AB_OK : AB_ERR_NOT_CONVERGED;
-#ifdef AB_TRACE_SWEEPS
-  if (crank == 0 && tid == 0) printf("jacobi job %d: k=%d r=%d sweeps=%d converged=%d\n", (int)(blockIdx.x / kC), k, r, sweeps, (int)converged);
-#endif
   csync();                              // nobody leaves while a peer may still read its rows
 }
 
@@ -359,9 +352,9 @@ int try_launch_jacobi(const JacobiJob* jobs, int count, int rmax, float tol, cud
                                   (int)cfg.dynamicSmemBytes));
   if (C > 1) {
     // one CTA per SM: CTAs that share an SM would only take turns on its issue slots
-    int dev = 0, sms = 0, resident = 0;
-    AB_CUDA_OK(cudaGetDevice(&dev));
-    AB_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    int resident = 0;
+    const int sms = sm_count();
+    if (sms <= 0) return AB_ERR_CUDA;
     if (rmax < 16 * C || (long long)count * C > sms) return 1;
     if (cudaOccupancyMaxActiveClusters(&resident, jacobi_rows_cluster_kernel<EL, C>, &cfg) != cudaSuccess) {
       (void)cudaGetLastError();
@@ -633,11 +626,8 @@ float rows_jacobi_tol(int s) { return 5e-7f * sqrtf((float)s) < 4e-6f ? 4e-6f : 
 bool rows_jacobi_fits(int count, int s) {
   if (s < 1 || s > 256 || count < 1) return false;
   if (jacobi_smem_bytes(s, s, 1) <= 227 * 1024 - 256) return true;
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return false;
-  return (long long)count * 2 <= sms && s >= 32;
+  const int sms = sm_count();
+  return sms > 0 && (long long)count * 2 <= sms && s >= 32;
 }
 
 size_t rows_jacobi_scratch_bytes(int count) { return align_up((size_t)count * sizeof(JacobiJob), 256); }
@@ -765,17 +755,24 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   // a8 (optional): forked off where the Jacobi kernel starts (the kernels before it fill every SM
   // themselves), joined at the end
   cudaStream_t side = any_w ? side_stream() : nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
-  if (side) {
-    if (cudaEventCreateWithFlags(&fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&join, cudaEventDisableTiming) != cudaSuccess) {
+  // the two events live for this call only; every return below destroys them (destroying an event that
+  // has been recorded releases it once the recorded work is done)
+  struct EventPair {
+    cudaEvent_t fork = nullptr, join = nullptr;
+    bool create() {
+      if (cudaEventCreateWithFlags(&fork, cudaEventDisableTiming) == cudaSuccess &&
+          cudaEventCreateWithFlags(&join, cudaEventDisableTiming) == cudaSuccess)
+        return true;
       (void)cudaGetLastError();
+      return false;
+    }
+    ~EventPair() {
       if (fork) cudaEventDestroy(fork);
       if (join) cudaEventDestroy(join);
-      fork = join = nullptr;
-      side = nullptr;
     }
-  }
+  } evs;
+  if (side && !evs.create()) side = nullptr;
+  cudaEvent_t fork = evs.fork, join = evs.join;
   if (any_w && !side) AB_TRY(gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, st));
   AB_TRY(gemm_simt_batched(w.gram_descs, (int)gg.size(), rmax, rmax, st));                  // Gram slices
   const size_t csm = chol_smem_bytes(rmax);
@@ -800,8 +797,6 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   AB_TRY(gemm_simt_batched(w.descs + 7 * L, L, rmax, nmax, st));                            // B'
   if (side) {
     if (side_rc == AB_OK && cudaStreamWaitEvent(st, join, 0) != cudaSuccess) side_rc = AB_ERR_CUDA;
-    cudaEventDestroy(fork);      // released once the recorded work is done
-    cudaEventDestroy(join);
     if (side_rc != AB_OK) { (void)cudaGetLastError(); return side_rc; }
   }
   return AB_OK;

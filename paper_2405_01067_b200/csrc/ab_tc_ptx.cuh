@@ -40,14 +40,16 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-// Waits for the phase with the given parity to complete, for at most about one second.
-// Returns false on expiry (the caller raises the CTA's abort flag and unwinds).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// Waits for the phase with the given parity to complete, for at most limit_ns (about one second
+// unless the caller says otherwise).  Returns false on expiry (the caller raises the CTA's abort
+// flag and unwinds).
+constexpr uint64_t kWaitLimitNs = 1000000000ull;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 255u && globaltimer_ns() - t0 > 1000000000ull) return false;
+    if ((it & 255u) == 255u && globaltimer_ns() - t0 > limit_ns) return false;
   }
 }
 

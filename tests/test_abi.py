@@ -93,3 +93,12 @@ def test_package_never_imports_the_checker():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 src = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in src, f
+
+
+def test_static_forward_rejects_sizes_that_would_wrap(L):
+    """N * r is checked by division: a row count near 2^63 (or 2^58 at r = 64, whose product wraps to a
+    small number) is refused on the host, before any launch, with or without a device."""
+    from paper_2405_01067_b200 import binding as b
+    p = ctypes.c_void_p(256)
+    for N in ((2 ** 63 - 1) // 2, 2 ** 58, 2 ** 58 + 1):
+        assert L.ab_layer_forward_static(p, p, p, p, N, 128, 128, 64, 64, 128, 0, None) == b.AB_ERR_UNSUPPORTED

@@ -1,9 +1,10 @@
 """ab_layer_forward_static: the forward call for users who cannot allocate device memory (a
 plug-in inside an application that owns the whole memory pool, a loop that must not touch
 cudaMalloc).  Its scratch is an array built into the library, so the test checks what such a
-user relies on: the result equals ab_layer_forward's, a second call right after the first is
-not disturbed by what the first left in the shared array, no device memory is allocated by
-the call, and a size beyond the built-in array is refused instead of overrunning it.
+user relies on: the result equals ab_layer_forward's and the CPU checker's, a second call right
+after the first is not disturbed by what the first left in the shared array, the device's free
+memory does not move across the calls, and a size beyond the built-in array is refused instead
+of overrunning it.
 Collected last on purpose: a failure here cannot hide another test's result."""
 import ctypes
 
@@ -11,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import ab_oracle as orc
 from paper_2405_01067_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -40,17 +42,26 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(ab, bf16, tol):
     outs, refs = [], []
     tensors = [[_dev(d[k], bf16) for k in ("x", "A", "B")] for d in cases]
     ys = [torch.empty((d["N"], d["m"]), dtype=t[0].dtype, device="cuda") for d, t in zip(cases, tensors)]
+    # one call first: loading the kernels and the first look-up of the array's address are behind us
+    ab.ab_layer_forward_static(*tensors[1], ys[1])
     torch.cuda.synchronize()
-    before = torch.cuda.memory_allocated()
+    ys[1].zero_()
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]      # the driver's own count of free bytes on the device
+    torch_before = torch.cuda.memory_allocated()
     for (x, A, B), y in zip(tensors, ys):          # back to back on one stream, no sync in between
         outs.append(ab.ab_layer_forward_static(x, A, B, y))
-    assert torch.cuda.memory_allocated() == before   # nothing was allocated through torch either
     torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before     # no cudaMalloc / cudaFree behind the calls
+    assert torch.cuda.memory_allocated() == torch_before   # and nothing through torch's allocator
     for (x, A, B) in tensors:
         refs.append(ab.ab_layer_forward(x, A, B)[0])
     torch.cuda.synchronize()
-    for got, ref in zip(outs, refs):
+    for got, ref, d in zip(outs, refs, cases):
         assert _rel(got, ref) <= tol
+        y_ref = orc.forward(d["x"], d["A"], d["B"])[1]
+        g = got.float().cpu().numpy()
+        assert orc.rel_frob(g, y_ref) <= tol and orc.max_tile_rel_frob(g, y_ref) <= tol
 
 
 def test_size_limit_and_bad_arguments(ab):
@@ -60,6 +71,9 @@ def test_size_limit_and_bad_arguments(ab):
     p = ctypes.c_void_p(256)      # never dereferenced: the calls below are rejected on the host
     N = cap // 64 + 1             # N * r just beyond the array
     assert L.ab_layer_forward_static(p, p, p, p, N, 128, 128, 64, 64, 128, 0, None) == ab.AB_ERR_UNSUPPORTED
+    # a row count whose product with r does not fit 64 bits must not slip under the limit
+    assert L.ab_layer_forward_static(p, p, p, p, (2 ** 63 - 1) // 2, 128, 128, 64, 64, 128, 0, None) == ab.AB_ERR_UNSUPPORTED
+    assert L.ab_layer_forward_static(p, p, p, p, 2 ** 58, 128, 128, 64, 64, 128, 0, None) == ab.AB_ERR_UNSUPPORTED
     assert L.ab_layer_forward_static(None, p, p, p, 8, 128, 128, 64, 64, 128, 0, None) == ab.AB_ERR_INVALID_ARG
     assert L.ab_layer_forward_static(p, p, p, p, 8, 128, 128, 200, 200, 128, 0, None) == ab.AB_ERR_INVALID_ARG
     # exactly at the limit is accepted and correct
@@ -70,3 +84,4 @@ def test_size_limit_and_bad_arguments(ab):
     ref = ab.ab_layer_forward(x, A, B)[0]
     torch.cuda.synchronize()
     assert _rel(y, ref) <= 2e-2
+    assert orc.rel_frob(y.float().cpu().numpy(), orc.forward(d["x"], d["A"], d["B"])[1]) <= 2e-2
