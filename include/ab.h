@@ -40,7 +40,10 @@ typedef enum {
   AB_ERR_WORKSPACE = -3,     /* ws NULL, misaligned or smaller than ab_workspace_bytes says */
   AB_ERR_NOT_CONVERGED = -4, /* device status: Jacobi sweep cap reached */
   AB_ERR_TIMEOUT = -5,       /* device status: a bounded on-chip wait expired */
-  AB_ERR_CUDA = -6           /* a CUDA runtime call failed (no device, launch error) */
+  AB_ERR_CUDA = -6,          /* a CUDA runtime call failed (no device, launch error) */
+  AB_ERR_ACCURACY = -7       /* device status: the split kept singular values below the accuracy domain of
+                                the route that computed them (stated at ab_svd_split / ab_group_sync); the
+                                outputs are written, those values are not accurate to 1e-4 */
 } ab_status;
 
 typedef enum { AB_F32 = 0, AB_BF16 = 1 } ab_dtype;
@@ -70,6 +73,16 @@ long long ab_launch_count(void);
  * holds AB_ERR_TIMEOUT.  Nothing hangs, traps or faults; the context stays usable.
  */
 int ab_selftest_bounded_wait(int* dev_status, unsigned limit_us, void* cuda_stream);
+
+/*
+ * The same for the whole failure path of the fused chain kernel (no counterpart in the paper): the kernel
+ * is launched on scratch operands inside ws with its loader switched off, so the waits of its other roles
+ * run out after limit_us microseconds; each role gives up, the kernel unwinds through its common exit,
+ * releases its tensor memory and leaves AB_ERR_TIMEOUT in the first int of ws.  ws: device memory of
+ * ab_selftest_chain_stall_workspace_bytes() bytes, 256-byte aligned.  Nothing hangs, traps or faults.
+ */
+int ab_selftest_chain_stall(void* ws, size_t ws_bytes, unsigned limit_us, void* cuda_stream);
+size_t ab_selftest_chain_stall_workspace_bytes(void);
 
 /*
  * Scratch bytes a call needs (0 if none).  Arguments a given op does not use are ignored
@@ -179,10 +192,13 @@ int ab_recombine(const void* Abar, const void* Bbar, float* W, int m, int n, int
  *   W [m,n] dense of type w_dt.  A [m,r_max] (row stride r_max) and B [r_max,n] of type
  *   out_dt; columns of A and rows of B with index >= r' are zero.  sigma [r_cap] fp32,
  *   descending up to rounding; r_out: device int that receives r'; dev_status: device
- *   int that receives AB_OK or AB_ERR_NOT_CONVERGED.  sigma_cutoff = 0 keeps r_cap.
- *   The decomposition works on the Gram matrix of the shorter side in fp32; singular
- *   values below about 2% of the largest lose relative accuracy (they keep absolute
- *   accuracy 1e-6 * s_0).  min(m,n) <= 3072.
+ *   int that receives AB_OK, AB_ERR_NOT_CONVERGED or AB_ERR_ACCURACY.  sigma_cutoff = 0 keeps r_cap.
+ *   Accuracy domain: the decomposition works on the Gram matrix of the shorter side in fp32, so
+ *   singular values below 1% of the largest lose relative accuracy (they keep absolute accuracy
+ *   1e-6 * s_0).  If a value between 1e-5 and 1e-2 of the largest is among the kept ones,
+ *   dev_status says AB_ERR_ACCURACY (outputs are still written); with sigma_cutoff >= 0.01 every
+ *   kept value is inside the domain.  Values below 1e-5 * s_0 count as zero (a W of lower rank
+ *   than r_max).  min(m,n) <= 3072.
  */
 int ab_svd_split(const void* W, int m, int n, int r_max, float sigma_cutoff,
                  void* A, void* B, float* sigma, int* r_out, int* dev_status,
@@ -215,11 +231,15 @@ typedef enum {
  * path: an ab_sync_path.  The factored path uses that W = Abar Bbar has rank <= r: the
  * decomposition reduces to Cholesky factors of Abar^T Abar and Bbar Bbar^T and the SVD of an
  * r x r core, each solved inside shared memory (one CTA, or a cluster of CTAs, per matrix); W
- * itself is only written if W_out asks for it.  It needs r <= 236 (shared-memory capacity) and
- * factors whose condition number is below about 300 (Cholesky pivots under 1e-6 of the largest
- * diagonal entry of a Gram matrix are taken as zero, which is exact for factors already
- * truncated by the rank rule); AB_SYNC_FACTORED returns
- * AB_ERR_UNSUPPORTED when r is too large, AB_SYNC_AUTO falls back to the dense path.
+ * itself is only written if W_out asks for it.  It needs r <= 236 (shared-memory capacity);
+ * AB_SYNC_FACTORED returns AB_ERR_UNSUPPORTED when r is too large, AB_SYNC_AUTO falls back to the
+ * dense path.  Accuracy domain of the factored path: singular values down to 1e-3 of the largest
+ * come out to 1e-4 relative.  dev_status[i] says AB_ERR_ACCURACY (outputs still written) when a
+ * kept value lies between 1e-6 and 1e-3 of the largest, or when a Cholesky pivot of a Gram matrix
+ * fell under 1e-6 of its largest diagonal entry without being exactly zero (exactly zero pivots
+ * are the columns of A / rows of B that an earlier rank rule removed: dropping them is exact).
+ * A caller that gets this status can rerun that matrix with AB_SYNC_DENSE, whose domain is
+ * stated at ab_svd_split; with sigma_cutoff >= 0.01 neither path keeps a value outside its domain.
  * Workspace: ab_sync_workspace_bytes (covers either path).  When a W_out is given, the factored
  * path runs that product on a helper stream of the library (one per device, lowest priority,
  * created on first use) beside its Jacobi kernel and joins it before the call's last kernel, so

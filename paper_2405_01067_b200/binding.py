@@ -18,12 +18,13 @@ AB_F32, AB_BF16 = 0, 1
 AB_OP_LAYER_FORWARD, AB_OP_LAYER_BACKWARD, AB_OP_GROUP_AVERAGE, AB_OP_RECOMBINE, AB_OP_SVD_SPLIT = range(5)
 AB_OK = 0
 AB_ERR_INVALID_ARG, AB_ERR_UNSUPPORTED, AB_ERR_WORKSPACE = -1, -2, -3
-AB_ERR_NOT_CONVERGED, AB_ERR_TIMEOUT, AB_ERR_CUDA = -4, -5, -6
+AB_ERR_NOT_CONVERGED, AB_ERR_TIMEOUT, AB_ERR_CUDA, AB_ERR_ACCURACY = -4, -5, -6, -7
 AB_SYNC_AUTO, AB_SYNC_DENSE, AB_SYNC_FACTORED = 0, 1, 2
 
 EXPORTS = ["ab_status_string", "ab_version", "ab_launch_count", "ab_workspace_bytes", "ab_layer_forward", "ab_layer_backward",
            "ab_group_average", "ab_recombine", "ab_svd_split", "ab_group_sync", "ab_sync_workspace_bytes",
-           "ab_layer_forward_static", "ab_static_scratch_elems", "ab_adamw_step", "ab_lr_rebound_factor", "ab_selftest_bounded_wait"]
+           "ab_layer_forward_static", "ab_static_scratch_elems", "ab_adamw_step", "ab_lr_rebound_factor", "ab_selftest_bounded_wait",
+           "ab_selftest_chain_stall", "ab_selftest_chain_stall_workspace_bytes"]
 
 
 class AbError(RuntimeError):
@@ -81,6 +82,9 @@ def lib() -> ctypes.CDLL:
     L.ab_lr_rebound_factor.argtypes = [c_int, c_int, c_float]
     L.ab_selftest_bounded_wait.restype = c_int
     L.ab_selftest_bounded_wait.argtypes = [c_void_p, ctypes.c_uint, c_void_p]
+    L.ab_selftest_chain_stall.restype = c_int
+    L.ab_selftest_chain_stall.argtypes = [c_void_p, c_size_t, ctypes.c_uint, c_void_p]
+    L.ab_selftest_chain_stall_workspace_bytes.restype = c_size_t
     _lib = L
     return L
 
@@ -91,6 +95,14 @@ def ab_selftest_bounded_wait(limit_us: int = 1000, stream=None) -> int:
     status = torch.zeros((1,), dtype=torch.int32, device="cuda")
     _check(lib().ab_selftest_bounded_wait(_ptr(status), int(limit_us), _stream(stream)), "ab_selftest_bounded_wait")
     return int(status.item())
+
+
+def ab_selftest_chain_stall(limit_us: int = 1000, stream=None) -> int:
+    """Runs the fused chain kernel with its loader switched off and returns the device status its unwinding
+    left (AB_ERR_TIMEOUT).  Synchronises."""
+    ws = workspace(int(lib().ab_selftest_chain_stall_workspace_bytes()), "cuda")
+    _check(lib().ab_selftest_chain_stall(_ptr(ws), ws.numel(), int(limit_us), _stream(stream)), "ab_selftest_chain_stall")
+    return workspace_status(ws)
 
 
 def ab_launch_count() -> int:

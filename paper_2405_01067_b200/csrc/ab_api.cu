@@ -117,6 +117,7 @@ const char* ab_status_string(int s) {
     case AB_ERR_NOT_CONVERGED: return "iteration did not converge";
     case AB_ERR_TIMEOUT: return "bounded device wait expired";
     case AB_ERR_CUDA: return "CUDA runtime error";
+    case AB_ERR_ACCURACY: return "kept singular values below the accuracy domain";
     default: return "unknown status";
   }
 }
@@ -151,6 +152,14 @@ int ab_selftest_bounded_wait(int* dev_status, unsigned limit_us, void* cuda_stre
   if (!dev_status || limit_us == 0 || limit_us > 1000000u) return AB_ERR_INVALID_ARG;
   if (!have_device()) return AB_ERR_CUDA;
   return bounded_wait_selftest(dev_status, limit_us, static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t ab_selftest_chain_stall_workspace_bytes(void) { return chain_stall_selftest_ws(); }
+
+int ab_selftest_chain_stall(void* ws, size_t ws_bytes, unsigned limit_us, void* cuda_stream) {
+  if (limit_us == 0 || limit_us > 1000000u) return AB_ERR_INVALID_ARG;
+  if (!have_device()) return AB_ERR_CUDA;
+  return chain_stall_selftest(ws, ws_bytes, limit_us, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int ab_layer_forward(const void* x, const void* A, const void* B, void* y, void* T_save,

@@ -1,21 +1,17 @@
 // Fused tensor-core chain for bf16 storage (fp32 accumulation) on sm_100a.
 //
-// row_chain_kernel: one CTA per block of 128 rows computes  S = In F1^T  (128 x r, K-loop over
-// the input width, accumulator in TMEM), rounds S to bf16 into shared memory, and multiplies
-// on:  Out = S F2^T  in 128-column chunks (two TMEM accumulators so the epilogue of one chunk
-// overlaps the MMAs of the next).  The rank-r intermediate never goes to HBM unless the
-// caller asks for a copy.
-//   forward : In = x,  F1 = B  (r x n), F2 = A   (m x r), Out = y,  S = T
-//   backward: In = dY, F1 = A^T (r x m), F2 = B^T (n x r), Out = dX, S = dT
-// grad_kernel: dA = dY^T T and dB^T = x^T dT are reductions over the rows; a CTA owns 128
-// output rows (a slice of m or of n) and one slice of the N rows, streams 64-row slabs of
-// both operands (both "MN-major": the reduction index is the slow one in memory) and leaves
-// an fp32 partial; reduce_kernel adds the partials in ascending slice order.
+// chain_kernel: persistent CTAs; for a block of 128 rows  S = In F1^T  (128 x r, K-loop over the input
+// width, accumulator in TMEM), S rounded to bf16 into shared memory, multiplied on:  Out = S F2^T  in
+// 256-column chunks.  The rank-r intermediate never goes to HBM unless the caller asks for a copy.
+//   forward : In = x,  F1 = B   (r x n), F2 = A   (m x r), Out = y,  S = T
+//   backward: In = dY, F1 = A^T (r x m), F2 = B^T (n x r), Out = dX, S = dT   (A and B read as they lie)
+// grad_kernel: dA = dY^T T and dB^T = x^T dT are reductions over the rows; a CTA owns 256 output rows (a
+// slice of m or of n) and one slice of the N rows, streams 64-row slabs of both operands (both
+// "MN-major": the reduction index is the slow one in memory) and leaves an fp32 partial;
+// reduce_partials_kernel adds the partials in ascending slice order.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner),
-// warps 2-5 = epilogue (TMEM -> registers -> shared/global).  All operand tiles are TMA
-// boxes of 64 bf16 (128 bytes) x rows with 128-byte swizzle.  Every mbarrier wait gives up
-// after about a second, raises AB_ERR_TIMEOUT in the status word and unwinds to the common
+// All operand tiles are TMA boxes of 64 bf16 (128 bytes) x rows with 128-byte swizzle.  Every mbarrier
+// wait gives up after about a second, raises AB_ERR_TIMEOUT in the status word and unwinds to the common
 // exit, where TMEM is released.
 #include <mutex>
 
@@ -28,7 +24,7 @@ namespace {
 using namespace tc;
 
 constexpr int kAtomBytes = 16384;      // 128 rows x 128 bytes
-constexpr int kMaxStages = 6;
+constexpr int kMaxStages = 10;
 constexpr int kMaxStages2 = 6;         // 32 KB slots of the second product, carved from the same ring memory
 constexpr int kChunk = 256;            // output columns per accumulator of the second product
 constexpr int kAtom2Bytes = kChunk * 128;   // one 256 x 64 tile of F2
@@ -36,18 +32,32 @@ constexpr int kSmemLimit = 227 * 1024;
 constexpr int kTmemCols = 512;
 constexpr int kEpiThreads = 128;
 
-struct RowChainParams {
+constexpr int kEpiWarps = 4;                         // 4 or 8: one or two warps per quarter of the TMEM lanes
+constexpr int kWarpsPerQuarter = kEpiWarps / 4;
+constexpr int kPiecesPerWarp = 4 / kWarpsPerQuarter;  // 64-column pieces of a 256-column chunk per warp
+constexpr int kStgTiles = 2;                         // staging tiles per epilogue warp
+constexpr int kChainThreads = 32 * (2 + kEpiWarps);
+constexpr int kGroupRows = 32;                   // rows are dealt to CTAs, loaded and stored in groups of 32
+constexpr int kGroupBytes = kGroupRows * 128;    // one group of one 64-column tile
+constexpr int kF1AtomBytes = 8192;               // 64 x 64 box of an MN-major factor
+
+struct ChainParams {
   int K1;        // width of In (reduction length of the first product)
   int P;         // width of Out (0: first product only)
-  int r;
+  int r;         // rank, padded to a multiple of 16
   int nk1;       // ceil(K1 / 64)
   int nchunks;   // ceil(P / 256)
   int natoms;    // ceil(r / 64)
-  int ns;        // ring stages
-  int slot_bytes;
-  int ns2;       // stages of the second product's ring (one 128 x 64 atom of F2 each)
-  int save_s;    // 1: copy S to global through tmS
-  int clear_status;   // 1: this is the first kernel of a call and zeroes the status word (see clear_status_word)
+  int max_blocks;          // 128-row blocks per unit: 1 or 2
+  int ns, slot_bytes;      // first product: slots of max_blocks In tiles + one slab of F1
+  int ns2;                 // second product: 32 KB slots at the start of shared memory
+  int f1_bytes;            // bytes of one F1 slab as the loads deliver it
+  int f1_mn, f2_mn;        // 1: the factor is held with the reduction index as the slow one (MN-major operand)
+  int save_s;              // 1: copy S to global through tmS
+  int groups;              // 32-row groups in all
+  int clear_status;        // 1: this is the first kernel of a call and zeroes the status word (see clear_status_word)
+  int stall_selftest;      // 1: the producer loads nothing, so every wait of the kernel runs out (failure-path self-test)
+  unsigned long long wait_ns;   // limit of every on-chip wait
   int* status;
 };
 
@@ -58,7 +68,7 @@ struct Bars {
   uint64_t acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   int abort_any;   // set by any role that gave up
-  int epi_abort;   // written and read by the epilogue warps only, around their own barrier
+  int epi_abort;   // used by the gradient kernel's epilogue warps around their own barrier
 };
 
 __device__ __forceinline__ void raise_timeout(Bars* b, int* status) {
@@ -75,7 +85,7 @@ __device__ __forceinline__ void clear_status_word(int enabled, int* status) {
   if (enabled && blockIdx.x == 0 && threadIdx.x == 0) atomicExch(status, 0);
 }
 
-// epilogue-wide wait: every epilogue thread calls it; the verdict is uniform
+// epilogue-wide wait of the gradient kernel: every epilogue thread calls it; the verdict is uniform
 __device__ __forceinline__ bool epi_wait(Bars* b, uint64_t* bar, uint32_t parity, int* status) {
   if (!mbar_wait(bar, parity)) {
     *reinterpret_cast<volatile int*>(&b->epi_abort) = 1;
@@ -85,7 +95,17 @@ __device__ __forceinline__ bool epi_wait(Bars* b, uint64_t* bar, uint32_t parity
   return *reinterpret_cast<volatile int*>(&b->epi_abort) == 0;
 }
 
-__device__ __forceinline__ void store_bf16x16_swizzled(uint8_t* row_base, int row, int c0, const uint32_t (&v)[16]) {
+// one warp waits; the verdict is uniform over the warp
+__device__ __forceinline__ bool warp_wait(Bars* b, uint64_t* bar, uint32_t parity, unsigned long long limit, int* status) {
+  int ok = 1;
+  if ((threadIdx.x & 31) == 0) {          // one lane polls; the others rest at the shuffle
+    ok = mbar_wait(bar, parity, limit) ? 1 : 0;
+    if (!ok) raise_timeout(b, status);
+  }
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+__device__ __forceinline__ void store_bf16x16_swizzled(uint8_t* row_base, int row, int c0, const uint32_t* v) {
   // 16 consecutive columns c0..c0+15 (c0 % 16 == 0) of a 128-byte row inside a swizzled atom
   uint32_t w[8];
 #pragma unroll
@@ -100,22 +120,51 @@ __device__ __forceinline__ void store_bf16x16_swizzled(uint8_t* row_base, int ro
   *p1 = make_uint4(w[4], w[5], w[6], w[7]);
 }
 
-__global__ void __launch_bounds__(192, 1)
-row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ CUtensorMap tmF1,
-                 const __grid_constant__ CUtensorMap tmF2, const __grid_constant__ CUtensorMap tmOut,
-                 const __grid_constant__ CUtensorMap tmS, const RowChainParams p) {
+// ---------------------------------------------------------------------------------------------
+// chain_kernel:  S = In F1^T (rows x r, accumulated in TMEM over the width of In), S rounded to bf16 into
+// shared memory, Out = S F2^T in 256-column chunks, stored as bf16.  One persistent CTA per SM.
+//
+// Rows.  The rows are cut into groups of 32 and every CTA owns a contiguous run of groups, as equal as the
+// group count allows, so the CTAs finish together whatever the row count is.  A CTA works through its run
+// in units of up to two blocks of 128 rows (one block when max_blocks == 1).  Both blocks of a unit share
+// every factor tile that is loaded -- each slab of F1 feeds two first-product MMAs, each tile of F2 two
+// second-product MMAs -- so a row costs half the factor bytes from L2.  A block at the end of a run may
+// hold fewer than four groups: only its groups are stored; the block is loaded and multiplied whole (rows are
+// independent in every product, and the rows past the run are never stored).
+//
+// Warps (192 threads): 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..5 = epilogue.  An epilogue
+// warp may read the quarter of the TMEM lanes given by its index modulo 4, i.e. the 32 rows of one group.
+// Each warp converts its 32 x 64 pieces into staging tiles of its own (two, used in turn) and stores them
+// with TMA stores of its own: no barrier spans the epilogue warps.  (Measured: two warps per quarter with
+// one staging tile each are slower, 129 against 110 us for a ViT forward; more pollers, no more overlap.)
+//
+// TMEM: block b of a unit keeps its S accumulator at column 256 b while the first product runs; the
+// accumulators of the second product take the same columns afterwards (in a two-block unit accumulator b
+// belongs to block b; in a one-block unit the two alternate between chunks).
+//
+// Factors.  F1 is r x K1 and F2 is P x r as operands.  Either may be given as it lies in memory (K-major:
+// the reduction index is the fast one -- B and A in the forward pass) or transposed (MN-major: the
+// reduction index is the slow one -- A and B in the backward pass, where F1 = A^T and F2 = B^T), which the
+// shared-memory descriptors of the MMAs express directly; nothing is transposed in memory.
+__global__ void __launch_bounds__(kChainThreads, 1)
+chain_kernel(const __grid_constant__ CUtensorMap tmIn,
+             const __grid_constant__ CUtensorMap tmF1, const __grid_constant__ CUtensorMap tmF2,
+             const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmS, const ChainParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* S = smem;
-  uint8_t* stg = S + p.natoms * kAtomBytes;
-  uint8_t* ring = stg + 2 * kAtomBytes;
-  Bars* bars = reinterpret_cast<Bars*>(ring + (size_t)p.ns * p.slot_bytes);
+  // [ second-product ring | S of block 0 | S of block 1 | one staging tile per epilogue warp | barriers ]; the
+  // first product's ring lies over the first three regions, which it has to itself while it runs
+  uint8_t* ring = smem;
+  uint8_t* S0 = smem + (size_t)p.ns2 * kAtom2Bytes;
+  uint8_t* stg = S0 + (size_t)p.max_blocks * p.natoms * kAtomBytes;
+  Bars* bars = reinterpret_cast<Bars*>(stg + kEpiWarps * kStgTiles * kGroupBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row0 = blockIdx.x * 128;
-  // All CTAs walk the same factor tiles.  Started together they would all ask L2 for the same
-  // few lines at the same moment (measured: 29 GB/s per SM); each CTA therefore starts its walk
-  // at a different slab / chunk and wraps round.  The order is a function of blockIdx only.
+  const int g_begin = (int)((int64_t)blockIdx.x * p.groups / gridDim.x);
+  const int g_end = (int)((int64_t)(blockIdx.x + 1) * p.groups / gridDim.x);
+  const int unit_groups = 4 * p.max_blocks;
+  // All CTAs walk the same factor tiles.  Started together they would all ask L2 for the same few lines at
+  // the same moment; each CTA therefore starts its walk at a different slab / chunk and wraps round.
   const int rot1 = blockIdx.x % p.nk1;
   const int rot2 = p.nchunks > 0 ? (blockIdx.x * 5) % p.nchunks : 0;
 
@@ -123,8 +172,9 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
     for (int i = 0; i < p.ns; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
     for (int i = 0; i < p.ns2; ++i) { mbar_init(&bars->full2[i], 1); mbar_init(&bars->empty2[i], 1); }
     mbar_init(&bars->t_full, 1);
-    mbar_init(&bars->s_ready, kEpiThreads);
-    for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 4); }
+    mbar_init(&bars->s_ready, kEpiWarps);
+    mbar_init(&bars->unit_done, 1 + kEpiWarps);   // the MMA issuer's commit and every epilogue warp
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], kEpiWarps); }
     bars->abort_any = 0;
     bars->epi_abort = 0;
     fence_barrier_init();
@@ -139,153 +189,227 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
   dep_wait();            // nothing above touches global memory
   dep_launch();
   clear_status_word(p.clear_status, p.status);
-  // T (r <= 256 columns) is read out into S before the second product starts, so the two
-  // 256-column accumulators of the second product reuse its columns.
-  const uint32_t tT = tmem_base;
-  const uint32_t tAcc0 = tmem_base;
+  const unsigned long long lim = p.wait_ns;
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      int i = 0;
+    if (lane == 0 && !p.stall_selftest) {
+      int i1 = 0, i2 = 0, u = 0;
       bool ok = true;
-      for (int ks = 0; ks < p.nk1 && ok; ++ks, ++i) {
-        const int slot = i % p.ns, ph = (i / p.ns) & 1;
-        if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
-        uint8_t* dst = ring + (size_t)slot * p.slot_bytes;
-        mbar_arrive_expect_tx(&bars->full[slot], kAtomBytes + p.r * 128);
-        const int kr = (ks + rot1) % p.nk1;   // every CTA starts on a different slab: see rot1
-        tma_load_2d(dst, &tmIn, &bars->full[slot], kr * 64, row0);
-        tma_load_2d(dst + kAtomBytes, &tmF1, &bars->full[slot], kr * 64, 0);
-      }
-      // The second product re-cuts the ring memory into 16 KB slots, so that many atoms of F2
-      // are in flight at once (L2 latency x the rate the MMAs need is > 100 KB); it may only be
-      // refilled once every MMA of the first product has read its slabs.
-      if (ok && p.nchunks > 0 && !mbar_wait(&bars->t_full, 0)) { raise_timeout(bars, p.status); ok = false; }
-      i = 0;
-      for (int c = 0; c < p.nchunks && ok; ++c) {
-        for (int j = 0; j < p.natoms; ++j, ++i) {
-          const int slot = i % p.ns2, ph = (i / p.ns2) & 1;
-          if (!mbar_wait(&bars->empty2[slot], ph ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
-          mbar_arrive_expect_tx(&bars->full2[slot], kAtom2Bytes);
-          tma_load_2d(ring + (size_t)slot * kAtom2Bytes, &tmF2, &bars->full2[slot], j * 64, ((c + rot2) % p.nchunks) * kChunk);
+      for (int g = g_begin; g < g_end && ok; ++u) {
+        const int ng = (g_end - g < unit_groups) ? g_end - g : unit_groups;
+        const int nt = ng > 4 ? 2 : 1;
+        const int row0 = g * kGroupRows;
+        // the shared memory of the last unit is free once its MMAs are done and its stores have been read
+        if (u > 0 && !mbar_wait(&bars->unit_done, (u - 1) & 1, lim)) { raise_timeout(bars, p.status); ok = false; break; }
+        for (int ks = 0; ks < p.nk1 && ok; ++ks, ++i1) {
+          const int slot = i1 % p.ns, ph = (i1 / p.ns) & 1;
+          if (!mbar_wait(&bars->empty[slot], ph ^ 1, lim)) { raise_timeout(bars, p.status); ok = false; break; }
+          uint8_t* dst = smem + (size_t)slot * p.slot_bytes;
+          mbar_arrive_expect_tx(&bars->full[slot], nt * kAtomBytes + p.f1_bytes);
+          const int kr = (ks + rot1) % p.nk1;
+          // a block at the end of the run is loaded whole as well: the rows past the run are a neighbour's
+          // (or zeros past the last row) and cost less than four separate 32-row loads
+          for (int tt = 0; tt < nt; ++tt) tma_load_2d(dst + tt * kAtomBytes, &tmIn, &bars->full[slot], kr * 64, row0 + tt * 128);
+          uint8_t* f1 = dst + p.max_blocks * kAtomBytes;
+          if (p.f1_mn)
+            for (int a = 0; a < p.natoms; ++a) tma_load_2d(f1 + a * kF1AtomBytes, &tmF1, &bars->full[slot], a * 64, kr * 64);
+          else
+            tma_load_2d(f1, &tmF1, &bars->full[slot], kr * 64, 0);
         }
+        // the second product's slots lie over the first product's: wait until its MMAs have read them
+        if (ok && !mbar_wait(&bars->t_full, u & 1, lim)) { raise_timeout(bars, p.status); ok = false; }
+        for (int c = 0; c < p.nchunks && ok; ++c) {
+          const int col0 = ((c + rot2) % p.nchunks) * kChunk;
+          for (int j = 0; j < p.natoms; ++j, ++i2) {
+            const int slot = i2 % p.ns2, ph = (i2 / p.ns2) & 1;
+            if (!mbar_wait(&bars->empty2[slot], ph ^ 1, lim)) { raise_timeout(bars, p.status); ok = false; break; }
+            uint8_t* d = ring + (size_t)slot * kAtom2Bytes;
+            mbar_arrive_expect_tx(&bars->full2[slot], kAtom2Bytes);
+            if (p.f2_mn)
+              for (int b = 0; b < 4; ++b) tma_load_2d(d + b * kF1AtomBytes, &tmF2, &bars->full2[slot], col0 + 64 * b, j * 64);
+            else
+              tma_load_2d(d, &tmF2, &bars->full2[slot], j * 64, col0);
+          }
+        }
+        g += ng;
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc1 = instr_desc_bf16(128, p.r, 0, 0);
-      const uint32_t idesc2 = instr_desc_bf16(128, kChunk, 0, 0);
-      int i = 0;
+      const uint32_t idesc1 = instr_desc_bf16(128, p.r, 0, p.f1_mn);
+      const uint32_t idesc2 = instr_desc_bf16(128, kChunk, 0, p.f2_mn);
+      int i1 = 0, i2 = 0, u = 0;
+      int q0 = 0, q1 = 0;                      // uses of each accumulator so far
       bool ok = true;
-      for (int ks = 0; ks < p.nk1; ++ks, ++i) {
-        const int slot = i % p.ns, ph = (i / p.ns) & 1;
-        if (!mbar_wait(&bars->full[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
-        tc_fence_after();
-        const uint32_t sa = smem_u32(ring + (size_t)slot * p.slot_bytes);
-        const uint64_t da = smem_desc_sw128(sa, 16), db = smem_desc_sw128(sa + kAtomBytes, 16);
-        int ksteps = (p.K1 - ((ks + rot1) % p.nk1) * 64 + 15) >> 4;
-        if (ksteps > 4) ksteps = 4;
-        for (int kk = 0; kk < ksteps; ++kk) tc_mma_bf16(tT, da + 2 * kk, db + 2 * kk, idesc1, (ks | kk) != 0);
-        tc_commit(&bars->empty[slot]);
-      }
-      if (ok) {
+      for (int g = g_begin; g < g_end && ok; ++u) {
+        const int ng = (g_end - g < unit_groups) ? g_end - g : unit_groups;
+        const int nt = ng > 4 ? 2 : 1;
+        for (int ks = 0; ks < p.nk1; ++ks, ++i1) {
+          const int slot = i1 % p.ns, ph = (i1 / p.ns) & 1;
+          if (!mbar_wait(&bars->full[slot], ph, lim)) { raise_timeout(bars, p.status); ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + (size_t)slot * p.slot_bytes);
+          const uint32_t sf = sa + p.max_blocks * kAtomBytes;
+          const uint64_t da0 = smem_desc_sw128(sa, 16), da1 = smem_desc_sw128(sa + kAtomBytes, 16);
+          int ksteps = (p.K1 - ((ks + rot1) % p.nk1) * 64 + 15) >> 4;
+          if (ksteps > 4) ksteps = 4;
+          for (int kk = 0; kk < ksteps; ++kk) {
+            const uint64_t db = p.f1_mn ? smem_desc_sw128(sf + kk * 2048, kF1AtomBytes) : smem_desc_sw128(sf, 16) + 2 * kk;
+            tc_mma_bf16(tmem_base, da0 + 2 * kk, db, idesc1, (ks | kk) != 0);
+            if (nt == 2) tc_mma_bf16(tmem_base + 256, da1 + 2 * kk, db, idesc1, (ks | kk) != 0);
+          }
+          tc_commit(&bars->empty[slot]);
+        }
+        if (!ok) break;
         tc_commit(&bars->t_full);
         if (p.nchunks > 0) {
-          if (!mbar_wait(&bars->s_ready, 0)) { raise_timeout(bars, p.status); ok = false; }
+          if (!mbar_wait(&bars->s_ready, u & 1, lim)) { raise_timeout(bars, p.status); ok = false; break; }
           tc_fence_after();
         }
-      }
-      i = 0;
-      for (int c = 0; c < p.nchunks && ok; ++c) {
-        const int b = c & 1;
-        if (!mbar_wait(&bars->acc_empty[b], ((c >> 1) & 1) ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
-        tc_fence_after();
-        const uint32_t tacc = tAcc0 + kChunk * b;
-        for (int j = 0; j < p.natoms; ++j, ++i) {
-          const int slot = i % p.ns2, ph = (i / p.ns2) & 1;
-          if (!mbar_wait(&bars->full2[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
-          tc_fence_after();
-          const uint64_t da = smem_desc_sw128(smem_u32(S + j * kAtomBytes), 16);
-          const uint64_t db = smem_desc_sw128(smem_u32(ring + (size_t)slot * kAtom2Bytes), 16);
-          int ksteps = (p.r - j * 64) >> 4;
-          if (ksteps > 4) ksteps = 4;
-          for (int kk = 0; kk < ksteps; ++kk) tc_mma_bf16(tacc, da + 2 * kk, db + 2 * kk, idesc2, (j | kk) != 0);
-          tc_commit(&bars->empty2[slot]);
+        for (int c = 0; c < p.nchunks && ok; ++c) {
+          for (int tt = 0; tt < nt && ok; ++tt) {
+            const int b = (nt == 2) ? tt : (c & 1);
+            if (!mbar_wait(&bars->acc_empty[b], ((b ? q1 : q0) & 1) ^ 1, lim)) { raise_timeout(bars, p.status); ok = false; break; }
+            tc_fence_after();
+            const uint32_t tacc = tmem_base + kChunk * b;
+            const uint8_t* Sb = S0 + (size_t)tt * p.natoms * kAtomBytes;
+            for (int j = 0; j < p.natoms; ++j) {
+              const int idx = i2 + j, slot = idx % p.ns2, ph = (idx / p.ns2) & 1;
+              if (!mbar_wait(&bars->full2[slot], ph, lim)) { raise_timeout(bars, p.status); ok = false; break; }
+              tc_fence_after();
+              const uint64_t da = smem_desc_sw128(smem_u32(Sb + j * kAtomBytes), 16);
+              const uint32_t sb = smem_u32(ring + (size_t)slot * kAtom2Bytes);
+              int ksteps = (p.r - j * 64) >> 4;
+              if (ksteps > 4) ksteps = 4;
+              for (int kk = 0; kk < ksteps; ++kk) {
+                const uint64_t db = p.f2_mn ? smem_desc_sw128(sb + kk * 2048, kF1AtomBytes) : smem_desc_sw128(sb, 16) + 2 * kk;
+                tc_mma_bf16(tacc, da + 2 * kk, db, idesc2, (j | kk) != 0);
+              }
+              if (tt == nt - 1) tc_commit(&bars->empty2[slot]);     // the last block of the unit is done with this tile
+            }
+            if (ok) { tc_commit(&bars->acc_full[b]); if (b) ++q1; else ++q0; }
+          }
+          i2 += p.natoms;
         }
-        if (ok) tc_commit(&bars->acc_full[b]);
+        if (ok) tc_commit(&bars->unit_done);
+        g += ng;
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
-    const int q = warp & 3;                 // TMEM lane quarter this warp may read
-    const int row = q * 32 + lane;          // row of the 128-row block
-    const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-    const bool issuer = (threadIdx.x == 64);
-    bool ok = epi_wait(bars, &bars->t_full, 0, p.status);
-    if (ok) {
+    // ------------------------------------------------------------ epilogue (warps 2..9)
+    const int qw = warp & 3;                // TMEM lane quarter this warp may read = the 32-row group it serves
+    const int hw = (warp - 2) >> 2;         // which of the warps of that quarter
+    const int row = qw * 32 + lane;         // row of the 128-row block
+    const uint32_t lane_base = (uint32_t)(qw * 32) << 16;
+    uint8_t* mystg = stg + (size_t)(warp - 2) * kStgTiles * kGroupBytes;
+    int nst = 0;                            // stores issued from this warp's staging tiles
+    int q0 = 0, q1 = 0;
+    int u = 0;
+    bool ok = true;
+    for (int g = g_begin; g < g_end && ok; ++u) {
+      const int ng = (g_end - g < unit_groups) ? g_end - g : unit_groups;
+      const int nt = ng > 4 ? 2 : 1;
+      const int row0 = g * kGroupRows;
+      ok = warp_wait(bars, &bars->t_full, u & 1, lim, p.status);
+      if (!ok) break;
       tc_fence_after();
-      for (int c0 = 0; c0 < p.r; c0 += 64) {       // up to four 16-column loads in flight per wait
-        uint32_t v[4][16];
+      // S of every block of the unit: the two warps of a quarter take alternate 64-column tiles
+      for (int tt = 0; tt < nt; ++tt) {
+        uint8_t* Sb = S0 + (size_t)tt * p.natoms * kAtomBytes;
+        for (int j = 0; j < p.natoms; ++j) {
+          if (((tt * p.natoms + j) % kWarpsPerQuarter) != hw) continue;
+          const int c0 = j * 64;
+          uint32_t v[4][16];
 #pragma unroll
-        for (int g = 0; g < 4; ++g)
-          if (c0 + g * 16 < p.r) tmem_ld16_nowait(tT + lane_base + c0 + g * 16, v[g]);
-        tmem_wait_ld();
+          for (int gq = 0; gq < 4; ++gq)
+            if (c0 + gq * 16 < p.r) tmem_ld16_nowait(tmem_base + 256 * tt + lane_base + c0 + gq * 16, v[gq]);
+          tmem_wait_ld();
 #pragma unroll
-        for (int g = 0; g < 4; ++g)
-          if (c0 + g * 16 < p.r) store_bf16x16_swizzled(S + (c0 >> 6) * kAtomBytes + row * 128, row, c0 + g * 16, v[g]);
+          for (int gq = 0; gq < 4; ++gq)
+            if (c0 + gq * 16 < p.r) store_bf16x16_swizzled(Sb + j * kAtomBytes + row * 128, row, c0 + gq * 16, v[gq]);
+        }
       }
       tc_fence_before();
       fence_proxy_async_smem();
-      mbar_arrive(&bars->s_ready);
-      if (p.save_s) {
-        named_bar_sync(1, kEpiThreads);
-        if (issuer) {
-          for (int j = 0; j < p.natoms; ++j) tma_store_2d(&tmS, S + j * kAtomBytes, j * 64, row0);
-          tma_store_commit();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->s_ready);
+      if (p.save_s && lane == 0) {           // this warp's tiles, this warp's 32 rows, if the block has them
+        for (int tt = 0; tt < nt; ++tt) {
+          const int gb = tt == 0 ? (ng < 4 ? ng : 4) : ng - 4;
+          if (qw >= gb) continue;
+          for (int j = 0; j < p.natoms; ++j) {
+            if (((tt * p.natoms + j) % kWarpsPerQuarter) != hw) continue;
+            tma_store_2d(&tmS, S0 + ((size_t)tt * p.natoms + j) * kAtomBytes + qw * kGroupBytes, j * 64,
+                         row0 + tt * 128 + qw * kGroupRows);
+          }
         }
+        tma_store_commit();
       }
-    }
-    int nstores = 0;
-    for (int c = 0; c < p.nchunks && ok; ++c) {
-      const int b = c & 1;
-      ok = epi_wait(bars, &bars->acc_full[b], (c >> 1) & 1, p.status);
-      if (!ok) break;
-      tc_fence_after();
-      const uint32_t tacc = tAcc0 + kChunk * b + lane_base;
-      for (int h = 0; h < kChunk / 64; ++h) {
-        const int col = ((c + rot2) % p.nchunks) * kChunk + h * 64;
-        const bool live = col < p.P;                 // columns beyond the output are not staged at all
-        uint32_t v[4][16];
-        if (live) {
+      for (int c = 0; c < p.nchunks && ok; ++c) {
+        const int col0 = ((c + rot2) % p.nchunks) * kChunk + hw * (64 * kPiecesPerWarp);
+        for (int tt = 0; tt < nt && ok; ++tt) {
+          const int b = (nt == 2) ? tt : (c & 1);
+          ok = warp_wait(bars, &bars->acc_full[b], (b ? q1 : q0) & 1, lim, p.status);
+          if (!ok) break;
+          if (b) ++q1; else ++q0;
+          tc_fence_after();
+          const int gb = tt == 0 ? (ng < 4 ? ng : 4) : ng - 4;
+          const bool rows_live = qw < gb;                 // does this block hold this warp's group?
+          const uint32_t tacc = tmem_base + kChunk * b + lane_base + hw * (64 * kPiecesPerWarp);
+          // the warp's 64-column pieces: each is read from TMEM and rounded to bf16 pairs at once (32
+          // registers a piece); they are staged and stored after the accumulator has been handed back
+          uint32_t w[kPiecesPerWarp][32];
 #pragma unroll
-          for (int g = 0; g < 4; ++g) tmem_ld16_nowait(tacc + h * 64 + g * 16, v[g]);
-          tmem_wait_ld();
-        }
-        if (h == kChunk / 64 - 1) {                  // the last columns are in registers: release the accumulator
+          for (int pc = 0; pc < kPiecesPerWarp; ++pc) {
+            if (rows_live && col0 + pc * 64 < p.P) {
+              uint32_t v[4][16];
+#pragma unroll
+              for (int gq = 0; gq < 4; ++gq) tmem_ld16_nowait(tacc + pc * 64 + gq * 16, v[gq]);
+              tmem_wait_ld();
+#pragma unroll
+              for (int gq = 0; gq < 4; ++gq)
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[gq][2 * i]), __uint_as_float(v[gq][2 * i + 1]));
+                  w[pc][gq * 8 + i] = *reinterpret_cast<uint32_t*>(&h2);
+                }
+            }
+          }
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars->acc_empty[b]);
-        }
-        if (!live) continue;
-        // staging tiles alternate with every store issued, so "at most one store still reading"
-        // always means the other tile
-        uint8_t* buf = stg + (nstores & 1) * kAtomBytes;
-        ++nstores;
-        if (issuer) tma_store_wait_read<1>();
-        named_bar_sync(1, kEpiThreads);
 #pragma unroll
-        for (int g = 0; g < 4; ++g) store_bf16x16_swizzled(buf + row * 128, row, g * 16, v[g]);
-        fence_proxy_async_smem();
-        named_bar_sync(1, kEpiThreads);
-        if (issuer) {
-          tma_store_2d(&tmOut, buf, col, row0);
-          tma_store_commit();
+          for (int pc = 0; pc < kPiecesPerWarp; ++pc) {
+            if (!(rows_live && col0 + pc * 64 < p.P)) continue;
+            uint8_t* buf = mystg + (nst % kStgTiles) * kGroupBytes;
+            ++nst;
+            if (lane == 0) tma_store_wait_read<kStgTiles - 1>();   // the store that last read this staging tile
+            __syncwarp();
+            uint8_t* rowp = buf + lane * 128;
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch)                 // 16-byte chunk ch of the row goes to slot ch ^ (row & 7)
+              *reinterpret_cast<uint4*>(rowp + ((ch ^ (lane & 7)) << 4)) =
+                  make_uint4(w[pc][4 * ch], w[pc][4 * ch + 1], w[pc][4 * ch + 2], w[pc][4 * ch + 3]);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&tmOut, buf, col0 + pc * 64, row0 + tt * 128 + qw * kGroupRows);
+              tma_store_commit();
+            }
+          }
         }
       }
+      // this warp has read all it will of the unit's accumulators; once its stores have read their
+      // shared memory (S tiles and staging) the next unit may overwrite both
+      if (ok) {
+        if (lane == 0) { tma_store_wait_read<0>(); mbar_arrive(&bars->unit_done); }
+        __syncwarp();
+      }
+      g += ng;
     }
-    if (issuer) tma_store_wait_all();
+    if (lane == 0) tma_store_wait_all();
   }
 
   // ------------------------------------------------------------ common exit
@@ -293,262 +417,6 @@ row_chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
   __syncthreads();
   if (*reinterpret_cast<volatile int*>(&bars->abort_any)) {
     // give loads that are still in flight time to land before the shared memory is released
-    const uint64_t t0 = globaltimer_ns();
-    while (globaltimer_ns() - t0 < 200000ull) { }
-    __syncthreads();
-  }
-  if (warp == 1) {
-    tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// row_chain_units_kernel: the same chain for many row blocks per CTA.  A persistent CTA owns a
-// contiguous range of 128-row blocks and works through it in units of two blocks (one block when
-// the range is odd).  Both blocks of a unit share every factor tile that is loaded -- each slab of
-// F1 feeds two first-product MMAs, each tile of F2 two second-product MMAs -- so a row costs half
-// the factor bytes; what paces the single-block kernel is exactly those bytes (1.5 MB of factors
-// against 0.2 MB of activations per block at the ViT shapes).  In a two-block unit the two
-// accumulators belong to the two blocks (the epilogue of one overlaps the MMAs of the other); in a
-// one-block unit they alternate between chunks as in row_chain_kernel.
-struct UnitParams {
-  int K1, P, r, nk1, nchunks, natoms;
-  int ns, slot_bytes;      // first product: slots of two 128-row In tiles + one F1 slab
-  int ns2, ring2_bytes;    // second product: 32 KB slots at the start of shared memory
-  int save_s;
-  int tiles;               // 128-row blocks in all
-  int clear_status;
-  int* status;
-};
-
-__global__ void __launch_bounds__(192, 1)
-row_chain_units_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ CUtensorMap tmF1,
-                       const __grid_constant__ CUtensorMap tmF2, const __grid_constant__ CUtensorMap tmOut,
-                       const __grid_constant__ CUtensorMap tmS, const UnitParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  // [ second-product ring | S of block 0 | S of block 1 | two staging tiles | barriers ]; the first
-  // product's ring lies over the first three regions, which it has to itself while it runs
-  uint8_t* ring = smem;
-  uint8_t* S0 = smem + p.ring2_bytes;
-  uint8_t* stg = S0 + 2 * p.natoms * kAtomBytes;
-  Bars* bars = reinterpret_cast<Bars*>(stg + 2 * kAtomBytes);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t_begin = (int)((int64_t)blockIdx.x * p.tiles / gridDim.x);
-  const int t_end = (int)((int64_t)(blockIdx.x + 1) * p.tiles / gridDim.x);
-  const int rot1 = blockIdx.x % p.nk1;
-  const int rot2 = p.nchunks > 0 ? (blockIdx.x * 5) % p.nchunks : 0;
-
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < p.ns; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
-    for (int i = 0; i < p.ns2; ++i) { mbar_init(&bars->full2[i], 1); mbar_init(&bars->empty2[i], 1); }
-    mbar_init(&bars->t_full, 1);
-    mbar_init(&bars->s_ready, kEpiThreads);
-    mbar_init(&bars->unit_done, 2);             // the MMA issuer's commit and the epilogue's store issuer
-    for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 4); }
-    bars->abort_any = 0;
-    bars->epi_abort = 0;
-    fence_barrier_init();
-    tma_prefetch_desc(&tmIn); tma_prefetch_desc(&tmF1); tma_prefetch_desc(&tmF2);
-    tma_prefetch_desc(&tmOut); tma_prefetch_desc(&tmS);
-  }
-  if (warp == 1) tmem_alloc(&bars->tmem_base, kTmemCols);
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
-  dep_wait();            // nothing above touches global memory
-  dep_launch();
-  clear_status_word(p.clear_status, p.status);
-  // TMEM: block b of a unit keeps its S accumulator at column 256 b while the first product runs;
-  // accumulator b of the second product takes the same 256 columns afterwards.
-
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      int i1 = 0, i2 = 0, u = 0;
-      bool ok = true;
-      for (int t = t_begin; t < t_end && ok; ++u) {
-        const int nt = (t_end - t >= 2) ? 2 : 1;
-        const int row0 = t * 128;
-        // the shared memory of the last unit is free once its MMAs are done and its stores have been read
-        if (u > 0 && !mbar_wait(&bars->unit_done, (u - 1) & 1)) { raise_timeout(bars, p.status); ok = false; break; }
-        for (int ks = 0; ks < p.nk1 && ok; ++ks, ++i1) {
-          const int slot = i1 % p.ns, ph = (i1 / p.ns) & 1;
-          if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
-          uint8_t* dst = smem + (size_t)slot * p.slot_bytes;
-          mbar_arrive_expect_tx(&bars->full[slot], nt * kAtomBytes + p.r * 128);
-          const int kr = (ks + rot1) % p.nk1;
-          tma_load_2d(dst, &tmIn, &bars->full[slot], kr * 64, row0);
-          if (nt == 2) tma_load_2d(dst + kAtomBytes, &tmIn, &bars->full[slot], kr * 64, row0 + 128);
-          tma_load_2d(dst + 2 * kAtomBytes, &tmF1, &bars->full[slot], kr * 64, 0);
-        }
-        // the second product's slots lie over the first product's: wait until its MMAs have read them
-        if (ok && !mbar_wait(&bars->t_full, u & 1)) { raise_timeout(bars, p.status); ok = false; }
-        for (int c = 0; c < p.nchunks && ok; ++c) {
-          for (int j = 0; j < p.natoms; ++j, ++i2) {
-            const int slot = i2 % p.ns2, ph = (i2 / p.ns2) & 1;
-            if (!mbar_wait(&bars->empty2[slot], ph ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
-            mbar_arrive_expect_tx(&bars->full2[slot], kAtom2Bytes);
-            tma_load_2d(ring + (size_t)slot * kAtom2Bytes, &tmF2, &bars->full2[slot], j * 64,
-                        ((c + rot2) % p.nchunks) * kChunk);
-          }
-        }
-        t += nt;
-      }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc1 = instr_desc_bf16(128, p.r, 0, 0);
-      const uint32_t idesc2 = instr_desc_bf16(128, kChunk, 0, 0);
-      int i1 = 0, i2 = 0, u = 0;
-      int q[2] = {0, 0};                       // uses of each accumulator so far
-      bool ok = true;
-      for (int t = t_begin; t < t_end && ok; ++u) {
-        const int nt = (t_end - t >= 2) ? 2 : 1;
-        for (int ks = 0; ks < p.nk1; ++ks, ++i1) {
-          const int slot = i1 % p.ns, ph = (i1 / p.ns) & 1;
-          if (!mbar_wait(&bars->full[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
-          tc_fence_after();
-          const uint32_t sa = smem_u32(smem + (size_t)slot * p.slot_bytes);
-          const uint64_t da0 = smem_desc_sw128(sa, 16), da1 = smem_desc_sw128(sa + kAtomBytes, 16);
-          const uint64_t db = smem_desc_sw128(sa + 2 * kAtomBytes, 16);
-          int ksteps = (p.K1 - ((ks + rot1) % p.nk1) * 64 + 15) >> 4;
-          if (ksteps > 4) ksteps = 4;
-          for (int kk = 0; kk < ksteps; ++kk) {
-            tc_mma_bf16(tmem_base, da0 + 2 * kk, db + 2 * kk, idesc1, (ks | kk) != 0);
-            if (nt == 2) tc_mma_bf16(tmem_base + 256, da1 + 2 * kk, db + 2 * kk, idesc1, (ks | kk) != 0);
-          }
-          tc_commit(&bars->empty[slot]);
-        }
-        if (!ok) break;
-        tc_commit(&bars->t_full);
-        if (p.nchunks > 0) {
-          if (!mbar_wait(&bars->s_ready, u & 1)) { raise_timeout(bars, p.status); ok = false; break; }
-          tc_fence_after();
-        }
-        for (int c = 0; c < p.nchunks && ok; ++c) {
-          for (int tt = 0; tt < nt && ok; ++tt) {
-            const int b = (nt == 2) ? tt : (c & 1);
-            if (!mbar_wait(&bars->acc_empty[b], (q[b] & 1) ^ 1)) { raise_timeout(bars, p.status); ok = false; break; }
-            tc_fence_after();
-            const uint32_t tacc = tmem_base + kChunk * b;
-            const uint8_t* Sb = S0 + (size_t)tt * p.natoms * kAtomBytes;
-            for (int j = 0; j < p.natoms; ++j) {
-              const int idx = i2 + j, slot = idx % p.ns2, ph = (idx / p.ns2) & 1;
-              if (!mbar_wait(&bars->full2[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
-              tc_fence_after();
-              const uint64_t da = smem_desc_sw128(smem_u32(Sb + j * kAtomBytes), 16);
-              const uint64_t db = smem_desc_sw128(smem_u32(ring + (size_t)slot * kAtom2Bytes), 16);
-              int ksteps = (p.r - j * 64) >> 4;
-              if (ksteps > 4) ksteps = 4;
-              for (int kk = 0; kk < ksteps; ++kk) tc_mma_bf16(tacc, da + 2 * kk, db + 2 * kk, idesc2, (j | kk) != 0);
-              if (tt == nt - 1) tc_commit(&bars->empty2[slot]);     // the last block of the unit is done with this tile
-            }
-            if (ok) { tc_commit(&bars->acc_full[b]); ++q[b]; }
-          }
-          i2 += p.natoms;
-        }
-        if (ok) tc_commit(&bars->unit_done);
-        t += nt;
-      }
-    }
-  } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
-    const int qw = warp & 3;                // TMEM lane quarter this warp may read
-    const int row = qw * 32 + lane;
-    const uint32_t lane_base = (uint32_t)(qw * 32) << 16;
-    const bool issuer = (threadIdx.x == 64);
-    int q[2] = {0, 0};
-    int nstores = 0, u = 0;
-    bool ok = true;
-    for (int t = t_begin; t < t_end && ok; ++u) {
-      const int nt = (t_end - t >= 2) ? 2 : 1;
-      const int row0 = t * 128;
-      ok = epi_wait(bars, &bars->t_full, u & 1, p.status);
-      if (!ok) break;
-      tc_fence_after();
-      for (int tt = 0; tt < nt; ++tt) {
-        uint8_t* Sb = S0 + (size_t)tt * p.natoms * kAtomBytes;
-        for (int c0 = 0; c0 < p.r; c0 += 64) {
-          uint32_t v[4][16];
-#pragma unroll
-          for (int g = 0; g < 4; ++g)
-            if (c0 + g * 16 < p.r) tmem_ld16_nowait(tmem_base + 256 * tt + lane_base + c0 + g * 16, v[g]);
-          tmem_wait_ld();
-#pragma unroll
-          for (int g = 0; g < 4; ++g)
-            if (c0 + g * 16 < p.r) store_bf16x16_swizzled(Sb + (c0 >> 6) * kAtomBytes + row * 128, row, c0 + g * 16, v[g]);
-        }
-      }
-      tc_fence_before();
-      fence_proxy_async_smem();
-      mbar_arrive(&bars->s_ready);
-      if (p.save_s) {
-        named_bar_sync(1, kEpiThreads);
-        if (issuer) {
-          for (int tt = 0; tt < nt; ++tt)
-            for (int j = 0; j < p.natoms; ++j)
-              tma_store_2d(&tmS, S0 + ((size_t)tt * p.natoms + j) * kAtomBytes, j * 64, row0 + tt * 128);
-          tma_store_commit();
-        }
-      }
-      for (int c = 0; c < p.nchunks && ok; ++c) {
-        for (int tt = 0; tt < nt && ok; ++tt) {
-          const int b = (nt == 2) ? tt : (c & 1);
-          ok = epi_wait(bars, &bars->acc_full[b], q[b] & 1, p.status);
-          if (!ok) break;
-          ++q[b];
-          tc_fence_after();
-          const uint32_t tacc = tmem_base + kChunk * b + lane_base;
-          for (int h = 0; h < kChunk / 64; ++h) {
-            const int col = ((c + rot2) % p.nchunks) * kChunk + h * 64;
-            const bool live = col < p.P;
-            uint32_t v[4][16];
-            if (live) {
-#pragma unroll
-              for (int g = 0; g < 4; ++g) tmem_ld16_nowait(tacc + h * 64 + g * 16, v[g]);
-              tmem_wait_ld();
-            }
-            if (h == kChunk / 64 - 1) {
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(&bars->acc_empty[b]);
-            }
-            if (!live) continue;
-            uint8_t* buf = stg + (nstores & 1) * kAtomBytes;
-            ++nstores;
-            if (issuer) tma_store_wait_read<1>();
-            named_bar_sync(1, kEpiThreads);
-#pragma unroll
-            for (int g = 0; g < 4; ++g) store_bf16x16_swizzled(buf + row * 128, row, g * 16, v[g]);
-            fence_proxy_async_smem();
-            named_bar_sync(1, kEpiThreads);
-            if (issuer) {
-              tma_store_2d(&tmOut, buf, col, row0 + tt * 128);
-              tma_store_commit();
-            }
-          }
-        }
-      }
-      // every epilogue thread has passed the last barrier, so all TMEM reads of the unit are done; once
-      // the stores issued so far have read their shared memory the next unit may overwrite S
-      if (issuer && ok) {
-        tma_store_wait_read<0>();
-        mbar_arrive(&bars->unit_done);
-      }
-      t += nt;
-    }
-    if (issuer) tma_store_wait_all();
-  }
-
-  // ------------------------------------------------------------ common exit
-  tc_fence_before();
-  __syncthreads();
-  if (*reinterpret_cast<volatile int*>(&bars->abort_any)) {
     const uint64_t t0 = globaltimer_ns();
     while (globaltimer_ns() - t0 < 200000ull) { }
     __syncthreads();
@@ -744,34 +612,6 @@ reduce_partials_kernel(const float* __restrict__ pA, float* __restrict__ dA, int
   }
 }
 
-// Both factor transposes of a backward call in one launch: At[j][i] = A[i][j] (A is m x r, row stride
-// ldA) for blocks [0, nA), Bt[j][i] = B[i][j] (B is r x n, row stride ldB) after that.
-__global__ void transpose_factors_kernel(const bf16* __restrict__ A, int m, int r, int ldA, bf16* __restrict__ At, int nA,
-                                         const bf16* __restrict__ B, int n, int ldB, bf16* __restrict__ Bt,
-                                         int* status_to_clear) {
-  __shared__ bf16 tile[32][33];
-  dep_wait();
-  dep_launch();
-  clear_status_word(status_to_clear != nullptr, status_to_clear);
-  const bool first = (int)blockIdx.x < nA;
-  const bf16* src = first ? A : B;
-  bf16* dst = first ? At : Bt;
-  const int rows = first ? m : r, cols = first ? r : n, ld = first ? ldA : ldB;
-  const int t = first ? blockIdx.x : blockIdx.x - nA;
-  const int tiles_c = (cols + 31) / 32;
-  const int by = (t / tiles_c) * 32, bx = (t % tiles_c) * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  for (int i = ty; i < 32; i += 8) {
-    const int rr = by + i, cc = bx + tx;
-    tile[i][tx] = (rr < rows && cc < cols) ? src[(size_t)rr * ld + cc] : __float2bfloat16(0.f);
-  }
-  __syncthreads();
-  for (int i = ty; i < 32; i += 8) {
-    const int cc = bx + i, rr = by + tx;
-    if (cc < cols && rr < rows) dst[(size_t)cc * rows + rr] = tile[tx][i];
-  }
-}
-
 // Self-test of the bounded wait every pipeline stage of the kernels above relies on: one thread waits on
 // an mbarrier that nobody ever arrives at.  The wait gives up after limit_ns and the kernel reports
 // AB_ERR_TIMEOUT through the status word, exactly as the chain kernels do; nothing spins for ever and the
@@ -859,37 +699,28 @@ int make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint
   return rc == CUDA_SUCCESS ? AB_OK : AB_ERR_CUDA;
 }
 
-struct RowPlan { int natoms, ns, slot_bytes, ns2; size_t smem; };
 // Ranks that are multiples of 8 but not of 16 run as the next multiple of 16: the tensor maps keep the
 // true extents, so the extra rows / columns of every factor tile arrive as zeros.
 int pad16(int r) { return (r + 15) & ~15; }
 
-RowPlan row_plan(int r) {      // r: padded rank
-  RowPlan pl;
-  pl.natoms = (r + 63) / 64;
-  pl.slot_bytes = kAtomBytes + r * 128;
-  const int fixed = pl.natoms * kAtomBytes + 2 * kAtomBytes + (int)sizeof(Bars) + 1024;
-  pl.ns = (kSmemLimit - fixed) / pl.slot_bytes;
-  if (pl.ns > kMaxStages) pl.ns = kMaxStages;
-  pl.smem = (size_t)fixed + (size_t)pl.ns * pl.slot_bytes;
-  pl.ns2 = pl.ns * pl.slot_bytes / kAtom2Bytes;
-  if (pl.ns2 > kMaxStages2) pl.ns2 = kMaxStages2;
-  return pl;
-}
-
-struct UnitPlan { int natoms, ns, slot_bytes, ns2, ring2_bytes; size_t smem; bool ok; };
-UnitPlan unit_plan(int r) {    // r: padded rank
-  UnitPlan pl;
-  pl.natoms = (r + 63) / 64;
-  pl.slot_bytes = 2 * kAtomBytes + r * 128;
-  const int fixed = 2 * pl.natoms * kAtomBytes + 2 * kAtomBytes + (int)sizeof(Bars) + 1024;
+// Shared-memory plan of chain_kernel for a (padded) rank and a number of blocks per unit.
+struct ChainPlan { int natoms, max_blocks, ns, slot_bytes, ns2, f1_bytes; size_t smem; bool ok; };
+ChainPlan chain_plan(int rp, int max_blocks, bool f1_mn) {
+  ChainPlan pl;
+  pl.natoms = (rp + 63) / 64;
+  pl.max_blocks = max_blocks;
+  pl.f1_bytes = f1_mn ? pl.natoms * kF1AtomBytes : rp * 128;
+  pl.slot_bytes = max_blocks * kAtomBytes + pl.f1_bytes;
+  const int s_bytes = max_blocks * pl.natoms * kAtomBytes;
+  const int fixed = s_bytes + kEpiWarps * kStgTiles * kGroupBytes + (int)sizeof(Bars) + 1024;
   pl.ns2 = (kSmemLimit - fixed) / kAtom2Bytes;
   if (pl.ns2 > kMaxStages2) pl.ns2 = kMaxStages2;
-  pl.ring2_bytes = pl.ns2 > 0 ? pl.ns2 * kAtom2Bytes : 0;
-  pl.ns = (pl.ring2_bytes + 2 * pl.natoms * kAtomBytes) / pl.slot_bytes;
+  if (pl.ns2 < 0) pl.ns2 = 0;
+  pl.ns = (pl.ns2 * kAtom2Bytes + s_bytes) / pl.slot_bytes;
   if (pl.ns > kMaxStages) pl.ns = kMaxStages;
-  pl.smem = (size_t)fixed + (size_t)pl.ring2_bytes;
-  pl.ok = pl.ns2 >= pl.natoms && pl.ns2 >= 2 && pl.ns >= 2;
+  pl.smem = (size_t)fixed + (size_t)pl.ns2 * kAtom2Bytes;
+  // a two-block unit keeps every tile of a chunk of F2 until its second block has used it
+  pl.ok = pl.ns >= 2 && pl.ns2 >= 2 && (max_blocks == 1 || pl.ns2 >= pl.natoms);
   return pl;
 }
 
@@ -913,14 +744,12 @@ GradPlan grad_plan(int64_t N, int m, int n, int r) {
   return pl;
 }
 
-struct BwdWs { int* status; bf16 *At, *Bt, *T, *dT; float *pA, *pB; size_t bytes; };
+struct BwdWs { int* status; bf16 *T, *dT; float *pA, *pB; size_t bytes; };
 BwdWs bwd_ws(void* ws, int64_t N, int m, int n, int r) {
   GradPlan gp = grad_plan(N, m, n, r);
   Arena ar(ws, 0);
   BwdWs w;
   w.status = ar.take_n<int>(64);
-  w.At = ar.take_n<bf16>((size_t)r * m);
-  w.Bt = ar.take_n<bf16>((size_t)n * r);
   w.T = ar.take_n<bf16>((size_t)N * r);
   w.dT = ar.take_n<bf16>((size_t)N * r);
   w.pA = ar.take_n<float>((size_t)gp.slices * m * pad16(r));
@@ -929,51 +758,47 @@ BwdWs bwd_ws(void* ws, int64_t N, int m, int n, int r) {
   return w;
 }
 
-// S = In F1^T (saved to Sg if not null), Out = S F2^T (skipped if Out is null)
-int launch_row_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1, const void* F2, int ldF2, int P,
-                     void* Out, void* Sg, int r, int* status, bool clear_status, cudaStream_t st) {
+// S = In F1^T (saved to Sg if not null), Out = S F2^T (skipped if Out is null).
+// f_mn = false: F1 is given as r x K1 (row stride ldF1) and F2 as P x r (row stride ldF2);
+// f_mn = true : F1 is given transposed, K1 x r, and F2 transposed, r x P (the factors A and B as they lie in
+//               memory when the chain runs backwards).
+int launch_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1, const void* F2, int ldF2, int P,
+                 bool f_mn, void* Out, void* Sg, int r, int* status, bool clear_status, cudaStream_t st,
+                 bool stall_selftest = false, unsigned long long wait_ns = kWaitLimitNs) {
   const int rp = pad16(r);
-  RowPlan pl = row_plan(rp);
-  if (pl.ns < 2 || pl.ns2 < 2) return AB_ERR_UNSUPPORTED;
+  const bool second = Out != nullptr && P > 0;
+  const int sms = sm_count();
+  if (sms <= 0) return AB_ERR_CUDA;
+  const int64_t groups = (N + kGroupRows - 1) / kGroupRows;
+  const int grid = (int)(groups < sms ? groups : sms);
+  const int64_t per_cta = (groups + grid - 1) / grid;
+  ChainPlan pl = chain_plan(rp, per_cta > 4 ? 2 : 1, f_mn);
+  if (!pl.ok && pl.max_blocks == 2) pl = chain_plan(rp, 1, f_mn);
+  if (!pl.ok) return AB_ERR_UNSUPPORTED;
   CUtensorMap tmIn, tmF1, tmF2, tmOut, tmS;
   AB_TRY(make_map(&tmIn, In, (uint64_t)N, K1, K1, 64, 128));
-  AB_TRY(make_map(&tmF1, F1, r, K1, ldF1, 64, rp));
-  const bool second = Out != nullptr && P > 0;
+  if (f_mn) AB_TRY(make_map(&tmF1, F1, K1, r, ldF1, 64, 64));
+  else AB_TRY(make_map(&tmF1, F1, r, K1, ldF1, 64, rp));
   // unused maps still have to be valid objects: alias them to the first operand
   if (second) {
-    AB_TRY(make_map(&tmF2, F2, P, r, ldF2, 64, kChunk));
-    AB_TRY(make_map(&tmOut, Out, (uint64_t)N, P, P, 64, 128));
+    if (f_mn) AB_TRY(make_map(&tmF2, F2, r, P, ldF2, 64, 64));
+    else AB_TRY(make_map(&tmF2, F2, P, r, ldF2, 64, kChunk));
+    AB_TRY(make_map(&tmOut, Out, (uint64_t)N, P, P, 64, kGroupRows));
   } else {
     tmF2 = tmIn;
     tmOut = tmIn;
   }
-  if (Sg) AB_TRY(make_map(&tmS, Sg, (uint64_t)N, r, r, 64, 128));
+  if (Sg) AB_TRY(make_map(&tmS, Sg, (uint64_t)N, r, r, 64, kGroupRows));
   else tmS = tmIn;
-  // More row blocks than SMs: persistent CTAs that take two blocks at a time and load each factor
-  // tile once for both.
-  {
-    const int64_t tiles = (N + 127) / 128;
-    const int sms = sm_count();
-    const UnitPlan up = unit_plan(rp);
-    if (second && sms > 0 && tiles > sms && up.ok) {
-      UnitParams q;
-      q.K1 = K1; q.P = P; q.r = rp; q.nk1 = (K1 + 63) / 64; q.nchunks = (P + kChunk - 1) / kChunk; q.natoms = up.natoms;
-      q.ns = up.ns; q.slot_bytes = up.slot_bytes; q.ns2 = up.ns2; q.ring2_bytes = up.ring2_bytes;
-      q.save_s = Sg ? 1 : 0; q.tiles = (int)tiles; q.clear_status = clear_status ? 1 : 0; q.status = status;
-      AB_CUDA_OK(cudaFuncSetAttribute(row_chain_units_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)up.smem));
-      AB_LAUNCH_DEP(row_chain_units_kernel, dim3((unsigned)sms), dim3(192), up.smem, st, tmIn, tmF1, tmF2, tmOut, tmS, q);
-      AB_LAUNCH_OK();
-      return AB_OK;
-    }
-  }
-  RowChainParams p;
-  p.K1 = K1; p.P = second ? P : 0; p.r = rp; p.nk1 = (K1 + 63) / 64; p.nchunks = second ? (P + kChunk - 1) / kChunk : 0;
-  p.natoms = pl.natoms; p.ns = pl.ns; p.slot_bytes = pl.slot_bytes; p.ns2 = pl.ns2; p.save_s = Sg ? 1 : 0;
-  p.clear_status = clear_status ? 1 : 0;
-  p.status = status;
-  AB_CUDA_OK(cudaFuncSetAttribute(row_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
-  const unsigned grid = (unsigned)((N + 127) / 128);
-  AB_LAUNCH_DEP(row_chain_kernel, dim3(grid), dim3(192), pl.smem, st, tmIn, tmF1, tmF2, tmOut, tmS, p);
+  ChainParams q;
+  q.K1 = K1; q.P = second ? P : 0; q.r = rp; q.nk1 = (K1 + 63) / 64; q.nchunks = second ? (P + kChunk - 1) / kChunk : 0;
+  q.natoms = pl.natoms; q.max_blocks = pl.max_blocks; q.ns = pl.ns; q.slot_bytes = pl.slot_bytes; q.ns2 = pl.ns2;
+  q.f1_bytes = pl.f1_bytes; q.f1_mn = f_mn ? 1 : 0; q.f2_mn = f_mn ? 1 : 0; q.save_s = Sg ? 1 : 0;
+  q.groups = (int)groups; q.clear_status = clear_status ? 1 : 0; q.stall_selftest = stall_selftest ? 1 : 0;
+  q.wait_ns = wait_ns; q.status = status;
+  AB_CUDA_OK(cudaFuncSetAttribute(chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
+  AB_LAUNCH_DEP(chain_kernel, dim3((unsigned)grid), dim3(kChainThreads), pl.smem, st, tmIn, tmF1, tmF2, tmOut,
+                tmS, q);
   AB_LAUNCH_OK();
   return AB_OK;
 }
@@ -986,6 +811,40 @@ int bounded_wait_selftest(int* dev_status, unsigned limit_us, cudaStream_t st) {
   return AB_OK;
 }
 
+// The chain kernel itself with a producer that loads nothing: the MMA issuer's and the epilogue warps'
+// waits run out after limit_us, every role unwinds to the common exit, TMEM is released and the status
+// word (first int of ws) holds AB_ERR_TIMEOUT.  The operands are carved from ws; their contents do not
+// matter, since nothing is ever loaded.
+size_t chain_stall_selftest_ws() { return 256 + 4 * 65536; }
+int chain_stall_selftest(void* ws, size_t ws_bytes, unsigned limit_us, cudaStream_t st) {
+  if (!ws || !aligned(ws, 256) || ws_bytes < chain_stall_selftest_ws()) return AB_ERR_WORKSPACE;
+  if (!device_is_sm100() || !encode_fn()) return AB_ERR_UNSUPPORTED;
+  char* base = static_cast<char*>(ws);
+  int* status = reinterpret_cast<int*>(base);
+  void* In = base + 256;                 // 256 x 64 bf16
+  void* F1 = base + 256 + 65536;         // 16 x 64
+  void* F2 = base + 256 + 2 * 65536;     // 64 x 16
+  void* Out = base + 256 + 3 * 65536;    // 256 x 64
+  return launch_chain(In, 256, 64, F1, 64, F2, 16, 64, false, Out, nullptr, 16, status, true, st, true,
+                      (unsigned long long)limit_us * 1000ull);
+}
+
+int make_tensor_map_2d(CUtensorMap* m, const void* ptr, bool f32, uint64_t rows, uint64_t cols, uint64_t ld,
+                       uint32_t box_cols, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return AB_ERR_CUDA;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld * (f32 ? 4 : 2)};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult rc = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr),
+                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? AB_OK : AB_ERR_CUDA;
+}
+
+bool tc_device_ok() { return device_is_sm100() && encode_fn() != nullptr; }
+
 bool chain_tc_supported(int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
                         const void* x, const void* A, const void* B, const void* y) {
   if (dt != AB_BF16) return false;
@@ -994,7 +853,7 @@ bool chain_tc_supported(int64_t N, int m, int n, int r, int ldA, int ldB, int dt
   if (N > (int64_t)1 << 30) return false;
   if (!aligned(x, 16) || !aligned(A, 16) || !aligned(B, 16) || !aligned(y, 16)) return false;
   if (!device_is_sm100() || !encode_fn()) return false;
-  return row_plan(pad16(r)).ns >= 2 && row_plan(pad16(r)).ns2 >= 2;
+  return chain_plan(pad16(r), 1, false).ok && chain_plan(pad16(r), 1, true).ok;
 }
 
 size_t chain_tc_forward_ws(int64_t, int, int, int) { return 256; }
@@ -1009,7 +868,7 @@ int chain_tc_forward(const void* x, const void* A, const void* B, void* y, void*
   if (!ws || ws_bytes < 256) return AB_ERR_WORKSPACE;
   if (T_save && !aligned(T_save, 16)) return AB_ERR_INVALID_ARG;
   int* status = static_cast<int*>(ws);
-  return launch_row_chain(x, N, n, B, ldB, A, ldA, m, y, T_save, r, status, true, st);
+  return launch_chain(x, N, n, B, ldB, A, ldA, m, false, y, T_save, r, status, true, st);
 }
 
 int chain_tc_backward(const void* x, const void* dY, const void* A, const void* B,
@@ -1026,21 +885,14 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
   bool after_chain = false;   // the dT/dX chain kernel is the launch right before the gradient kernel
   const bf16* T = static_cast<const bf16*>(T_saved);
   if (dA && !T) {   // recompute T = x B^T (first product only)
-    AB_TRY(launch_row_chain(x, N, n, B, ldB, nullptr, 0, 0, nullptr, w.T, r, w.status, first, st));
+    AB_TRY(launch_chain(x, N, n, B, ldB, nullptr, 0, 0, false, nullptr, w.T, r, w.status, first, st));
     first = false;
     T = w.T;
   }
   if (dX || dB) {
-    {
-      const int nA = ((m + 31) / 32) * ((r + 31) / 32);
-      const int nB = dX ? ((r + 31) / 32) * ((n + 31) / 32) : 0;
-      AB_LAUNCH_DEP(transpose_factors_kernel, dim3(nA + nB), dim3(256), 0, st, static_cast<const bf16*>(A), m, r, ldA, w.At,
-                 nA, static_cast<const bf16*>(B), n, ldB, w.Bt, first ? w.status : static_cast<int*>(nullptr));
-      AB_LAUNCH_OK();
-      first = false;
-    }
-    // dT = dY A (kept for dB), dX = dT B
-    AB_TRY(launch_row_chain(dY, N, m, w.At, m, w.Bt, r, n, dX, dB ? w.dT : nullptr, r, w.status, false, st));
+    // dT = dY A (kept for dB), dX = dT B: the chain with F1 = A^T and F2 = B^T, i.e. A and B as they lie
+    AB_TRY(launch_chain(dY, N, m, A, ldA, B, ldB, n, true, dX, dB ? w.dT : nullptr, r, w.status, first, st));
+    first = false;
     after_chain = true;
   }
   if (dA || dB) {

@@ -93,6 +93,35 @@ struct GemmDesc {
 };
 int gemm_simt_batched(const GemmDesc* d_descs, int count, int max_M, int max_N, cudaStream_t st);
 
+// ---- general tensor-core GEMM (ab_gemm_tc.cu) --------------------------------------------------
+// C[M x N] = sum over terms of A_t B_t^T on the tensor cores; see the head of ab_gemm_tc.cu.
+struct TcOperand {
+  const void* p[3];   // bf16 pieces: one (plain product) or three (hi, mid, lo of an fp32 matrix)
+  int pieces;
+  int64_t ld;         // row stride in elements, a multiple of 8
+  bool mn;            // false: stored M x K (resp. N x K); true: stored K x M (resp. K x N)
+};
+struct TcProblem {
+  TcOperand A, B;
+  void* C;            // fp32 or bf16, row stride ldc; with ksplit > 1: ksplit partial results, each
+  int64_t ldc;        //   round_up(M, 128) rows, one after the other (fp32 only)
+  int M, N, K;
+  bool c_f32;
+  int ksplit;
+  const int* live_rows;   // optional device ints: rows / columns at or beyond them are written as zero
+  const int* live_cols;
+};
+bool gemm_tc_available();
+bool gemm_tc_problem_ok(const TcProblem& q);
+size_t gemm_tc_table_bytes(int count);
+// table_dev: device memory of gemm_tc_table_bytes(count); status: device int that receives AB_ERR_TIMEOUT
+// if a bounded wait ran out (never cleared here).
+int gemm_tc_batched(const TcProblem* probs, int count, void* table_dev, int* status, cudaStream_t st);
+struct SplitJob { const float* src; int64_t ld_src; int rows, cols; bf16 *hi, *mid, *lo; int64_t ld_dst; int64_t first_block; };
+int64_t split_job_blocks(int rows, int cols);
+int split3_batched(const SplitJob* d_jobs, int njobs, int64_t total_blocks, cudaStream_t st);
+int sum_slices(const float* part, float* out, int64_t count, int64_t slice_stride, int slices, cudaStream_t st);
+
 // ---- fused tensor-core chain (ab_chain_tc.cu) --------------------------------------------------
 bool chain_tc_supported(int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
                         const void* x, const void* A, const void* B, const void* y);
@@ -107,6 +136,8 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
                       void* ws, size_t ws_bytes, cudaStream_t st);
 
 int bounded_wait_selftest(int* dev_status, unsigned limit_us, cudaStream_t st);
+size_t chain_stall_selftest_ws();
+int chain_stall_selftest(void* ws, size_t ws_bytes, unsigned limit_us, cudaStream_t st);
 
 // ---- SVD pipeline (ab_svd.cu) ------------------------------------------------------------------
 struct SvdItem {

@@ -37,6 +37,10 @@ constexpr int kMaxSweeps = 30;
 constexpr int kInnerSweeps = 2;
 constexpr float kCountRel2 = 1e-8f;  // rows below 1e-4 of the largest norm do not hold up convergence
 constexpr float kDeadRel2 = 1e-12f;   // rows below 1e-6 of the largest norm count as zero
+// Accuracy domain of this route: a kept singular value between kZeroRel and kDomainRel of the largest has lost
+// relative accuracy to the squaring in the Gram matrix (measured: 5e-6 at 1-2 %, 5e-3 at 0.5-1 %); the status
+// word then says so.  Below kZeroRel a value is zero to working precision (a W of lower rank than asked for).
+constexpr float kDomainRel = 1e-2f, kZeroRel = 1e-5f;
 
 // Rows count as orthogonal when |x_i.x_j| <= tol |x_i||x_j|.  An fp32 dot product of length s
 // carries rounding noise of about 6e-8 sqrt(s) relative to |x_i||x_j|; the maximum over all
@@ -488,7 +492,13 @@ __global__ void rank_rule_kernel(const float* __restrict__ sigma, int r_cap, flo
   for (int k = 0; k < r_cap; ++k) keep += (sigma[k] >= thr) ? 1 : 0;
   if (keep < 1) keep = 1;
   *r_out = keep;
-  if (dev_status) *dev_status = st->status;
+  if (dev_status) {
+    int code = st->status;
+    if (code == AB_OK)
+      for (int k = 0; k < keep; ++k)
+        if (sigma[k] < kDomainRel * top && sigma[k] > kZeroRel * top) code = AB_ERR_ACCURACY;
+    *dev_status = code;
+  }
 }
 
 // long factor: F(t,k) = Ylong(k,t) / sqrt(sigma_k); short factor: F(k,u) = sqrt(sigma_k) Vr[k][u].

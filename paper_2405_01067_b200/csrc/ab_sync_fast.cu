@@ -33,6 +33,11 @@ constexpr float kJCount2 = 1e-8f;    // rows below 1e-4 of the largest norm do n
 constexpr float kJEarly2 = 9e-8f;    // a sweep whose largest rotated cosine was below 3e-4 is the last one: one-sided
                                      // Jacobi converges quadratically, so what it leaves is of the order 1e-7 < tol
 constexpr float kEigThr = 1e-6f;     // relative pivot cut of G_A, G_B (and of sigma in the scalings)
+// Accuracy domain of the factored route: the relative error of a singular value grows as it falls below the
+// largest (measured: 5e-5 down to 1 %, 1e-4 at 4e-4, 1e-3 at 6e-5 of the largest); a kept value between
+// kFZeroRel and kFDomainRel of the largest, or a Cholesky pivot that was dropped although it was not exactly
+// zero, is reported through the status word.
+constexpr float kFDomainRel = 1e-3f, kFZeroRel = 1e-6f;
 constexpr int kCThreads = 512;
 
 struct JacobiJob {
@@ -411,7 +416,8 @@ __global__ void __launch_bounds__(kCThreads, 1) chol_inv_kernel(const CholJob* _
   __shared__ float maxdiag;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = kCThreads / 32;
 
-  if (tid == 0) maxdiag = 0.f;
+  __shared__ int dropped_live;          // pivots taken as zero although they were not exactly zero
+  if (tid == 0) { maxdiag = 0.f; dropped_live = 0; }
   {
     const float* __restrict__ G = job.G;
     const size_t part = (size_t)r * r;
@@ -443,7 +449,10 @@ __global__ void __launch_bounds__(kCThreads, 1) chol_inv_kernel(const CholJob* _
       const float inv = live ? 1.f / sqrtf(dj) : 0.f;
       for (int k = j + 1 + tid; k < r; k += kCThreads) S[j * ld + k] *= inv;   // a dropped row becomes zero
       __syncthreads();
-      if (tid == 0) { S[j * ld + j] = dj * inv; dinv[j] = inv; }                // nobody reads the pivot below
+      if (tid == 0) {
+        S[j * ld + j] = dj * inv; dinv[j] = inv;                                // nobody reads the pivot below
+        if (!live && dj != 0.f) dropped_live = 1;
+      }
       {                                              // panel rows still open: 64 threads per row
         const int i = j + 1 + (tid >> 6);
         if (i < jend) {
@@ -508,7 +517,7 @@ __global__ void __launch_bounds__(kCThreads, 1) chol_inv_kernel(const CholJob* _
     job.R[idx] = (k >= i) ? S[i * ld + k] : 0.f;
     job.Rinv[idx] = (k > i) ? S[k * ld + i] : (k == i ? dinv[i] : 0.f);
   }
-  if (tid == 0 && job.status) *job.status = AB_OK;
+  if (tid == 0 && job.status) *job.status = dropped_live ? (int)AB_ERR_ACCURACY : (int)AB_OK;
 }
 
 size_t chol_smem_bytes(int r) { return sizeof(float) * ((size_t)r * (r + 1) + r) + 64; }
@@ -529,7 +538,11 @@ __global__ void fast_rank_rule_kernel(const float* const* __restrict__ sigma, co
   *r_out[i] = keep;
   if (dev_status) {
     int st = AB_OK;
-    for (int j = 0; j < 3; ++j) if (jstatus[3 * i + j] != AB_OK) st = jstatus[3 * i + j];
+    for (int k = 0; k < keep; ++k)
+      if (sg[k] < kFDomainRel * top && sg[k] > kFZeroRel * top) st = AB_ERR_ACCURACY;
+    for (int j = 0; j < 3; ++j) if (jstatus[3 * i + j] == AB_ERR_ACCURACY) st = AB_ERR_ACCURACY;
+    for (int j = 0; j < 3; ++j)          // a solver that did not converge outranks the accuracy note
+      if (jstatus[3 * i + j] != AB_OK && jstatus[3 * i + j] != AB_ERR_ACCURACY) st = jstatus[3 * i + j];
     dev_status[i] = st;
   }
 }

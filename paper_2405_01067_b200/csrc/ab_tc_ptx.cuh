@@ -162,4 +162,11 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N, int a_mn_ma
 }
 
 }  // namespace tc
+
+// Host side (ab_chain_tc.cu): 2-D tensor map of a row-major bf16 (or fp32) matrix [rows x cols], row stride
+// ld elements, boxes of box_cols x box_rows with the 128-byte swizzle; and whether the current device and
+// driver can run these kernels at all.
+int make_tensor_map_2d(CUtensorMap* m, const void* ptr, bool f32, uint64_t rows, uint64_t cols, uint64_t ld,
+                       uint32_t box_cols, uint32_t box_rows);
+bool tc_device_ok();
 }  // namespace ab

@@ -31,7 +31,7 @@ def test_every_declared_symbol_is_exported(L):
 def test_status_strings(L):
     from paper_2405_01067_b200 import binding as b
     assert b.status_string(0) == "ok"
-    for code in range(-6, 0):
+    for code in range(-7, 0):
         assert b.status_string(code) not in ("ok", "unknown status")
     assert b.status_string(-99) == "unknown status"
     assert L.ab_version().decode().count(".") == 1
