@@ -638,12 +638,19 @@ def main():
                     help="rows of the CPU checker's bounded sample timed once beside the GPU run (cpu_baseline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-model-sync", action="store_true", help="skip the full-ViT group-sync measurement")
+    ap.add_argument("--only-model-sync", action="store_true",
+                    help="run only the full-ViT group-sync measurement and print its figures (for profiling that part)")
     ap.add_argument("--no-other-workloads", action="store_true",
                     help="skip the ResNet-50 / VGG16 / small fp32 layer measurements")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         raise SystemExit(spawn_ranks(args.gpus))
+    if args.only_model_sync:
+        import torch
+        from paper_2405_01067_b200 import binding as ab
+        print(json.dumps(dict(group_sync_model=vit_model_sync(ab, torch, steps=args.steps))))
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -53,7 +53,9 @@ typedef enum {
   AB_OP_LAYER_BACKWARD = 1,
   AB_OP_GROUP_AVERAGE = 2,
   AB_OP_RECOMBINE = 3,
-  AB_OP_SVD_SPLIT = 4
+  AB_OP_SVD_SPLIT = 4,
+  AB_OP_DENSE_FORWARD = 5,
+  AB_OP_DENSE_BACKWARD = 6
 } ab_op;
 
 /* Human-readable name of a status code (static storage, never NULL). */
@@ -146,6 +148,22 @@ int ab_layer_backward(const void* x, const void* dY, const void* A, const void* 
                       void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Dense layer of the full-rank phases of a training cycle (Algorithm 1: the warm-up steps before the
+ * first decomposition and the full-rank rebound steps after W <- A B; Section "Methodology", full-rank
+ * rebound): the same linear map with W held dense.
+ *   forward : y [N,m] = x [N,n] W^T, W [m,n] dense (row stride n); all of storage type dt.
+ *   backward: dX [N,n] = dY [N,m] W (type dt), dW [m,n] = dY^T x (fp32, sums over N in a fixed order).
+ *   Either of dX, dW may be NULL.  bf16 storage with m, n multiples of 8 runs on the tensor cores
+ *   (fp32 accumulation); other shapes and fp32 storage take the general kernel.  N = 0 is a no-op
+ *   (dW is zeroed).  Workspace: ab_workspace_bytes(AB_OP_DENSE_FORWARD / AB_OP_DENSE_BACKWARD, N, m, n,
+ *   0, 0, dt); its first int receives AB_OK or AB_ERR_TIMEOUT as for ab_layer_forward.
+ */
+int ab_dense_forward(const void* x, const void* W, void* y, int64_t N, int m, int n, int dt,
+                     void* ws, size_t ws_bytes, void* cuda_stream);
+int ab_dense_backward(const void* x, const void* dY, const void* W, void* dX, float* dW,
+                      int64_t N, int m, int n, int dt, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * One AdamW update of a factor from the gradient ab_layer_backward left (the paper trains with
  * AdamW, Section "Experiments"; decoupled weight decay):
  *   p <- p (1 - lr wd);  m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;
@@ -180,7 +198,11 @@ int ab_group_average(const void* base, int64_t stride_elems, int K, int64_t coun
 
 /*
  * Recombination (Algorithm 1: W <- A B): W [m,n] fp32 (dense) = Abar [m,r] Bbar [r,n],
- * factors of type dt, product accumulated in fp32 without reduced-precision passes.
+ * factors of type dt, product accurate to fp32 rounding.  With a workspace of
+ * ab_workspace_bytes(AB_OP_RECOMBINE, 0, m, n, r, 0, dt) bytes and n a multiple of 4 it runs on the tensor
+ * cores: bf16 factors multiply exactly in fp32; fp32 factors are cut into three bf16 pieces each (24 bits)
+ * and multiplied as six bf16 products accumulated in fp32.  With ws = NULL (or too small) the same product
+ * runs on the fp32 pipes.
  */
 int ab_recombine(const void* Abar, const void* Bbar, float* W, int m, int n, int r,
                  int ldA, int ldB, int dt, void* ws, size_t ws_bytes, void* cuda_stream);
@@ -194,9 +216,9 @@ int ab_recombine(const void* Abar, const void* Bbar, float* W, int m, int n, int
  *   descending up to rounding; r_out: device int that receives r'; dev_status: device
  *   int that receives AB_OK, AB_ERR_NOT_CONVERGED or AB_ERR_ACCURACY.  sigma_cutoff = 0 keeps r_cap.
  *   Accuracy domain: the decomposition works on the Gram matrix of the shorter side in fp32, so
- *   singular values below 1% of the largest lose relative accuracy (they keep absolute accuracy
- *   1e-6 * s_0).  If a value between 1e-5 and 1e-2 of the largest is among the kept ones,
- *   dev_status says AB_ERR_ACCURACY (outputs are still written); with sigma_cutoff >= 0.01 every
+ *   singular values below 2% of the largest lose relative accuracy (they keep absolute accuracy
+ *   1e-6 * s_0).  If a value between 1e-5 and 2e-2 of the largest is among the kept ones,
+ *   dev_status says AB_ERR_ACCURACY (outputs are still written); with sigma_cutoff >= 0.02 every
  *   kept value is inside the domain.  Values below 1e-5 * s_0 count as zero (a W of lower rank
  *   than r_max).  min(m,n) <= 3072.
  */
@@ -233,13 +255,13 @@ typedef enum {
  * r x r core, each solved inside shared memory (one CTA, or a cluster of CTAs, per matrix); W
  * itself is only written if W_out asks for it.  It needs r <= 236 (shared-memory capacity);
  * AB_SYNC_FACTORED returns AB_ERR_UNSUPPORTED when r is too large, AB_SYNC_AUTO falls back to the
- * dense path.  Accuracy domain of the factored path: singular values down to 1e-3 of the largest
+ * dense path.  Accuracy domain of the factored path: singular values down to 1e-2 of the largest
  * come out to 1e-4 relative.  dev_status[i] says AB_ERR_ACCURACY (outputs still written) when a
- * kept value lies between 1e-6 and 1e-3 of the largest, or when a Cholesky pivot of a Gram matrix
+ * kept value lies between 1e-6 and 1e-2 of the largest, or when a Cholesky pivot of a Gram matrix
  * fell under 1e-6 of its largest diagonal entry without being exactly zero (exactly zero pivots
  * are the columns of A / rows of B that an earlier rank rule removed: dropping them is exact).
  * A caller that gets this status can rerun that matrix with AB_SYNC_DENSE, whose domain is
- * stated at ab_svd_split; with sigma_cutoff >= 0.01 neither path keeps a value outside its domain.
+ * stated at ab_svd_split; with sigma_cutoff >= 0.02 neither path keeps a value outside its domain.
  * Workspace: ab_sync_workspace_bytes (covers either path).  When a W_out is given, the factored
  * path runs that product on a helper stream of the library (one per device, lowest priority,
  * created on first use) beside its Jacobi kernel and joins it before the call's last kernel, so

@@ -8,6 +8,8 @@ What each function follows:
 
 * ``forward`` / ``backward``   the layer W = A B of Eq. 3 used as a linear map
   y = x W^T, and the chain rule through the rank-r intermediate.
+* ``dense_forward`` / ``dense_backward``  the same layer with W dense (Algorithm 1's
+  full-rank steps: warm-up and rebound).
 * ``group_average*``           Algorithm 1, the two allReduce(./worldSize) lines.
 * ``recombine``                Algorithm 1, "W <- AB".
 * ``jacobi_svd``               the SVD that Eq. 3 refers to (one-sided Jacobi,
@@ -54,6 +56,18 @@ def backward(x, dY, A, B):
     dA = dY.T @ T
     dB = dT.T @ x
     return dX, dA, dB, dT
+
+
+def dense_forward(x, W):
+    """y = x W^T: the layer with W held dense (Algorithm 1's full-rank steps before the first decomposition
+    and after W <- A B)."""
+    return _f64(x) @ _f64(W).T
+
+
+def dense_backward(x, dY, W):
+    """Chain rule of L(y) through y = x W^T: dX = dY W, dW = dY^T x.  Returns (dX, dW)."""
+    x, dY, W = _f64(x), _f64(dY), _f64(W)
+    return dY @ W, dY.T @ x
 
 
 # ------------------------------------------------------------------ group mean (Algorithm 1)

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libab.so")
 
 AB_F32, AB_BF16 = 0, 1
 AB_OP_LAYER_FORWARD, AB_OP_LAYER_BACKWARD, AB_OP_GROUP_AVERAGE, AB_OP_RECOMBINE, AB_OP_SVD_SPLIT = range(5)
+AB_OP_DENSE_FORWARD, AB_OP_DENSE_BACKWARD = 5, 6
 AB_OK = 0
 AB_ERR_INVALID_ARG, AB_ERR_UNSUPPORTED, AB_ERR_WORKSPACE = -1, -2, -3
 AB_ERR_NOT_CONVERGED, AB_ERR_TIMEOUT, AB_ERR_CUDA, AB_ERR_ACCURACY = -4, -5, -6, -7
@@ -24,7 +25,8 @@ AB_SYNC_AUTO, AB_SYNC_DENSE, AB_SYNC_FACTORED = 0, 1, 2
 EXPORTS = ["ab_status_string", "ab_version", "ab_launch_count", "ab_workspace_bytes", "ab_layer_forward", "ab_layer_backward",
            "ab_group_average", "ab_recombine", "ab_svd_split", "ab_group_sync", "ab_sync_workspace_bytes",
            "ab_layer_forward_static", "ab_static_scratch_elems", "ab_adamw_step", "ab_lr_rebound_factor", "ab_selftest_bounded_wait",
-           "ab_selftest_chain_stall", "ab_selftest_chain_stall_workspace_bytes"]
+           "ab_selftest_chain_stall", "ab_selftest_chain_stall_workspace_bytes",
+           "ab_dense_forward", "ab_dense_backward"]
 
 
 class AbError(RuntimeError):
@@ -85,6 +87,10 @@ def lib() -> ctypes.CDLL:
     L.ab_selftest_chain_stall.restype = c_int
     L.ab_selftest_chain_stall.argtypes = [c_void_p, c_size_t, ctypes.c_uint, c_void_p]
     L.ab_selftest_chain_stall_workspace_bytes.restype = c_size_t
+    L.ab_dense_forward.restype = c_int
+    L.ab_dense_forward.argtypes = [c_void_p] * 3 + [c_int64, c_int, c_int, c_int, c_void_p, c_size_t, c_void_p]
+    L.ab_dense_backward.restype = c_int
+    L.ab_dense_backward.argtypes = [c_void_p] * 5 + [c_int64, c_int, c_int, c_int, c_void_p, c_size_t, c_void_p]
     _lib = L
     return L
 
@@ -207,6 +213,39 @@ def ab_layer_backward(x, dY, A, B, T_saved=None, want=("dX", "dA", "dB"), dX=Non
     return dX, dA, dB
 
 
+def ab_dense_forward(x, W, y=None, ws=None, stream=None):
+    """y = x W^T with W held dense (the full-rank phases of a cycle)."""
+    _dev_ok(x, W, y)
+    N, n = x.shape
+    m = W.shape[0]
+    dt = _dt(x)
+    if y is None:
+        y = torch.empty((N, m), dtype=x.dtype, device=x.device)
+    if ws is None:
+        ws = workspace(ab_workspace_bytes(AB_OP_DENSE_FORWARD, N, m, n, 0, 1, dt), x.device)
+    st = lib().ab_dense_forward(_ptr(x), _ptr(W), _ptr(y), N, m, n, dt, _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "ab_dense_forward")
+    return y
+
+
+def ab_dense_backward(x, dY, W, want=("dX", "dW"), dX=None, dW=None, ws=None, stream=None):
+    """dX = dY W, dW = dY^T x (fp32).  Returns (dX, dW); entries not in `want` are None."""
+    _dev_ok(x, dY, W, dX, dW)
+    N, n = x.shape
+    m = W.shape[0]
+    dt = _dt(x)
+    if "dX" in want and dX is None:
+        dX = torch.empty((N, n), dtype=x.dtype, device=x.device)
+    if "dW" in want and dW is None:
+        dW = torch.empty((m, n), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = workspace(ab_workspace_bytes(AB_OP_DENSE_BACKWARD, N, m, n, 0, 1, dt), x.device)
+    st = lib().ab_dense_backward(_ptr(x), _ptr(dY), _ptr(W), _ptr(dX), _ptr(dW), N, m, n, dt, _ptr(ws), ws.numel(),
+                                 _stream(stream))
+    _check(st, "ab_dense_backward")
+    return dX, dW
+
+
 def ab_adamw_step(param, grad, m, v, lr, step, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=1e-2, param_bf16=None,
                   stream=None):
     """One AdamW update in place (param, m, v fp32; grad fp32); param_bf16 optionally receives the rounded copy."""
@@ -239,15 +278,17 @@ def ab_group_average(copies, out=None, out_dtype=None, stream=None):
     return out
 
 
-def ab_recombine(Abar, Bbar, W=None, stream=None):
+def ab_recombine(Abar, Bbar, W=None, ws=None, stream=None):
     """W = Abar Bbar in fp32."""
     _dev_ok(Abar, Bbar, W)
     m, r = Abar.shape
     n = Bbar.shape[1]
     if W is None:
         W = torch.empty((m, n), dtype=torch.float32, device=Abar.device)
+    if ws is None:
+        ws = workspace(ab_workspace_bytes(AB_OP_RECOMBINE, 0, m, n, r, 1, _dt(Abar)), Abar.device)
     st = lib().ab_recombine(_ptr(Abar), _ptr(Bbar), _ptr(W), m, n, r, Abar.stride(0), Bbar.stride(0), _dt(Abar),
-                            None, 0, _stream(stream))
+                            _ptr(ws), ws.numel(), _stream(stream))
     _check(st, "ab_recombine")
     return W
 

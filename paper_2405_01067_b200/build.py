@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libab.so")
-SOURCES = ["ab_api.cu", "ab_gemm_simt.cu", "ab_average.cu", "ab_svd.cu", "ab_chain_tc.cu", "ab_gemm_tc.cu", "ab_noalloc.cu", "ab_sync_fast.cu", "ab_optim.cu"]
+SOURCES = ["ab_api.cu", "ab_gemm_simt.cu", "ab_average.cu", "ab_svd.cu", "ab_chain_tc.cu", "ab_gemm_tc.cu", "ab_dense.cu", "ab_noalloc.cu", "ab_sync_fast.cu", "ab_optim.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
          "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

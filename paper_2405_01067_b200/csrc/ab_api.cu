@@ -62,6 +62,23 @@ int check_layer_args(const void* x, const void* A, const void* B, int64_t N, int
 size_t general_forward_ws(int64_t N, int r) { return 256 + align_up((size_t)N * r * sizeof(float), 256); }
 size_t general_backward_ws(int64_t N, int r) { return 256 + 2 * align_up((size_t)N * r * sizeof(float), 256); }
 
+// Workspace of the tensor-core route of ab_recombine: status word, problem table, two split jobs and the three
+// bf16 pieces of each factor.
+struct RecombWs { int* status; void* table; SplitJob* jobs; bf16 *Asp, *Bsp; size_t ea, eb; int r8, n8; size_t bytes; };
+RecombWs recombine_ws(void* ws, int m, int n, int r) {
+  Arena ar(ws, 0);
+  RecombWs w;
+  w.r8 = (r + 7) & ~7; w.n8 = (n + 7) & ~7;
+  w.ea = (size_t)m * w.r8; w.eb = (size_t)r * w.n8;
+  w.status = ar.take_n<int>(64);
+  w.table = ar.take(gemm_tc_table_bytes(1));
+  w.jobs = ar.take_n<SplitJob>(2);
+  w.Asp = ar.take_n<bf16>(3 * w.ea);
+  w.Bsp = ar.take_n<bf16>(3 * w.eb);
+  w.bytes = align_up(ar.used, 256);
+  return w;
+}
+
 int general_forward(const void* x, const void* A, const void* B, void* y, void* T_save,
                     int64_t N, int m, int n, int r, int ldA, int ldB, int dt, void* ws, size_t ws_bytes,
                     cudaStream_t st) {
@@ -128,7 +145,8 @@ long long ab_launch_count(void) { return g_launches.load(std::memory_order_relax
 
 size_t ab_workspace_bytes(int op, int64_t N, int m, int n, int r, int K, int dt) {
   (void)K;
-  if (m <= 0 || n <= 0 || r <= 0 || N < 0) return 0;
+  if (m <= 0 || n <= 0 || N < 0) return 0;
+  if (r <= 0 && op != AB_OP_DENSE_FORWARD && op != AB_OP_DENSE_BACKWARD) return 0;
   switch (op) {
     case AB_OP_LAYER_FORWARD: {
       size_t g = general_forward_ws(N, r), t = chain_tc_forward_ws(N, m, n, r);
@@ -138,6 +156,9 @@ size_t ab_workspace_bytes(int op, int64_t N, int m, int n, int r, int K, int dt)
       size_t g = general_backward_ws(N, r), t = chain_tc_backward_ws(N, m, n, r);
       return (g > t ? g : t) + 256;
     }
+    case AB_OP_RECOMBINE: return recombine_ws(nullptr, m, n, r).bytes + 256;
+    case AB_OP_DENSE_FORWARD: return dense_forward_ws(N, m, n) + 256;
+    case AB_OP_DENSE_BACKWARD: return dense_backward_ws(N, m, n) + 256;
     case AB_OP_SVD_SPLIT: {
       SvdItem it;
       memset(&it, 0, sizeof(it));
@@ -227,11 +248,34 @@ int ab_group_average(const void* base, int64_t stride_elems, int K, int64_t coun
 
 int ab_recombine(const void* Abar, const void* Bbar, float* W, int m, int n, int r,
                  int ldA, int ldB, int dt, void* ws, size_t ws_bytes, void* cuda_stream) {
-  (void)ws; (void)ws_bytes;
   if (!dtype_ok(dt) || m <= 0 || n <= 0 || r <= 0 || ldA < r || ldB < n) return AB_ERR_INVALID_ARG;
   if (!Abar || !Bbar || !W) return AB_ERR_INVALID_ARG;
   if (!have_device()) return AB_ERR_CUDA;
-  return gemm_simt(Abar, dt, ldA, 1, Bbar, dt, ldB, 1, W, AB_F32, n, m, n, r, static_cast<cudaStream_t>(cuda_stream));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // Tensor-core route: bf16 factors multiply exactly in fp32 (one term); fp32 factors are cut into three bf16
+  // pieces and multiplied as six terms.  It needs the workspace and 16-byte rows; without them the product
+  // runs on the fp32 pipes.
+  RecombWs w = recombine_ws(ws, m, n, r);
+  const bool tc = ws && aligned(ws, 256) && ws_bytes >= w.bytes && gemm_tc_available() && n % 4 == 0 && aligned(W, 16) &&
+                  (dt == AB_F32 || (ldA % 8 == 0 && ldB % 8 == 0 && aligned(Abar, 16) && aligned(Bbar, 16)));
+  if (!tc) return gemm_simt(Abar, dt, ldA, 1, Bbar, dt, ldB, 1, W, AB_F32, n, m, n, r, st);
+  AB_CUDA_OK(cudaMemsetAsync(w.status, 0, sizeof(int), st));
+  TcProblem q;
+  q.C = W; q.ldc = n; q.M = m; q.N = n; q.K = r; q.c_f32 = true; q.ksplit = 1; q.live_rows = q.live_cols = nullptr;
+  if (dt == AB_BF16) {
+    q.A.p[0] = Abar; q.A.p[1] = q.A.p[2] = nullptr; q.A.pieces = 1; q.A.ld = ldA; q.A.mn = false;
+    q.B.p[0] = Bbar; q.B.p[1] = q.B.p[2] = nullptr; q.B.pieces = 1; q.B.ld = ldB; q.B.mn = true;
+  } else {
+    SplitJob jobs[2];
+    jobs[0] = SplitJob{static_cast<const float*>(Abar), ldA, m, r, w.Asp, w.Asp + w.ea, w.Asp + 2 * w.ea, w.r8, 0};
+    jobs[1] = SplitJob{static_cast<const float*>(Bbar), ldB, r, n, w.Bsp, w.Bsp + w.eb, w.Bsp + 2 * w.eb, w.n8,
+                       split_job_blocks(m, r)};
+    AB_CUDA_OK(cudaMemcpyAsync(w.jobs, jobs, sizeof(jobs), cudaMemcpyHostToDevice, st));
+    AB_TRY(split3_batched(w.jobs, 2, split_job_blocks(m, r) + split_job_blocks(r, n), st));
+    for (int k = 0; k < 3; ++k) { q.A.p[k] = w.Asp + k * w.ea; q.B.p[k] = w.Bsp + k * w.eb; }
+    q.A.pieces = q.B.pieces = 3; q.A.ld = w.r8; q.B.ld = w.n8; q.A.mn = false; q.B.mn = true;
+  }
+  return gemm_tc_batched(&q, 1, w.table, w.status, st);
 }
 
 int ab_svd_split(const void* W, int m, int n, int r_max, float sigma_cutoff,

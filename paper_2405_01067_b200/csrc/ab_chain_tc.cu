@@ -13,6 +13,7 @@
 // All operand tiles are TMA boxes of 64 bf16 (128 bytes) x rows with 128-byte swizzle.  Every mbarrier
 // wait gives up after about a second, raises AB_ERR_TIMEOUT in the status word and unwinds to the common
 // exit, where TMEM is released.
+#include <cstring>
 #include <mutex>
 
 #include "ab_common.cuh"
@@ -41,6 +42,25 @@ constexpr int kGroupRows = 32;                   // rows are dealt to CTAs, load
 constexpr int kGroupBytes = kGroupRows * 128;    // one group of one 64-column tile
 constexpr int kF1AtomBytes = 8192;               // 64 x 64 box of an MN-major factor
 
+// Convolution mode (3 x 3, stride 1, padding 1, activations NHWC): the rows of In are never materialised.  A
+// block is a tile of whole image rows (bh rows of one image, or bb whole images when an image has at most 128
+// pixels), i.e. a run of consecutive pixels; slab kr of the reduction is tap kr / cslabs and 64 channels, and the
+// block's In tile for it is the 4-D box of the activation shifted by the tap (what falls outside an image
+// arrives as zeros: the padding).  The factor's slab is found at column tap * tap_stride (+ f1_col_off).
+struct ConvGeom {
+  int on;
+  int B, H, W;
+  int in_ch;       // channels of the In tensor
+  int cslabs;      // ceil(in_ch / 64)
+  int bh, bb;      // tile: bh image rows (bb == 1) or bb whole images (bh == H)
+  int tpi;         // tiles per image (bb == 1) or 1
+  int box_rows;    // W * bh * bb: rows one In box delivers
+  int sign;        // +1: In pixel = out pixel + (tap - 1); -1: In pixel = out pixel - (tap - 1)
+  int tap_stride;  // columns of the factor between taps
+  int f1_col_off;  // first column of this launch's factor window inside a tap
+  int s_col_off;   // first column of S in the output it is stored to
+};
+
 struct ChainParams {
   int K1;        // width of In (reduction length of the first product)
   int P;         // width of Out (0: first product only)
@@ -54,7 +74,11 @@ struct ChainParams {
   int f1_bytes;            // bytes of one F1 slab as the loads deliver it
   int f1_mn, f2_mn;        // 1: the factor is held with the reduction index as the slow one (MN-major operand)
   int save_s;              // 1: copy S to global through tmS
-  int groups;              // 32-row groups in all
+  int groups;              // work items in all: 32-row groups, or tiles of a convolution (see ConvGeom)
+  ConvGeom cv;
+  bf16* out_ptr;           // convolution mode: Out and S as plain pointers for the rows of a tile's last, partial
+  bf16* s_ptr;             //   group of 32 (row strides P and s_ld)
+  int s_ld, s_cols;        // s_cols: true width of S
   int clear_status;        // 1: this is the first kernel of a call and zeroes the status word (see clear_status_word)
   int stall_selftest;      // 1: the producer loads nothing, so every wait of the kernel runs out (failure-path self-test)
   unsigned long long wait_ns;   // limit of every on-chip wait
@@ -120,6 +144,47 @@ __device__ __forceinline__ void store_bf16x16_swizzled(uint8_t* row_base, int ro
   *p1 = make_uint4(w[4], w[5], w[6], w[7]);
 }
 
+// One unit of a CTA's run: up to two blocks, each with its first row, its count of valid rows and (convolution
+// mode) the image and image row its tile starts at.
+struct Unit { int nt, adv; int row0[2], nrows[2], b0[2], y0[2]; };
+__device__ __forceinline__ Unit make_unit(const ChainParams& p, int it, int it_end) {
+  Unit u;
+  if (!p.cv.on) {
+    const int cap = 4 * p.max_blocks;
+    const int ng = (it_end - it < cap) ? it_end - it : cap;
+    u.nt = ng > 4 ? 2 : 1;
+    u.adv = ng;
+    u.row0[0] = it * kGroupRows; u.row0[1] = u.row0[0] + 128;
+    u.nrows[0] = (ng < 4 ? ng : 4) * kGroupRows; u.nrows[1] = (ng - 4) * kGroupRows;
+    u.b0[0] = u.b0[1] = u.y0[0] = u.y0[1] = 0;
+  } else {
+    u.nt = (it_end - it < p.max_blocks) ? it_end - it : p.max_blocks;
+    u.adv = u.nt;
+    for (int tt = 0; tt < 2; ++tt) {
+      const int t = it + tt;
+      const int grp = t / p.cv.tpi, ty = t - grp * p.cv.tpi;
+      u.b0[tt] = grp * p.cv.bb;
+      u.y0[tt] = ty * p.cv.bh;
+      u.row0[tt] = (u.b0[tt] * p.cv.H + u.y0[tt]) * p.cv.W;
+      int nb = p.cv.B - u.b0[tt]; if (nb > p.cv.bb) nb = p.cv.bb;
+      int nh = p.cv.H - u.y0[tt]; if (nh > p.cv.bh) nh = p.cv.bh;
+      u.nrows[tt] = nb * nh * p.cv.W;
+    }
+  }
+  return u;
+}
+
+// The rows of a partial group (fewer than 32) of a staged 32 x 64 tile go out with plain 16-byte stores.
+__device__ __forceinline__ void store_partial_group(const uint8_t* buf, bf16* dst, int64_t ld, int rows, int cols_left) {
+  const int lane = threadIdx.x & 31;
+  for (int idx = lane; idx < rows * 8; idx += 32) {
+    const int rr = idx >> 3, ch = idx & 7;
+    if (ch * 8 >= cols_left) continue;
+    const uint4 v = *reinterpret_cast<const uint4*>(buf + rr * 128 + ((ch ^ (rr & 7)) << 4));
+    *reinterpret_cast<uint4*>(dst + (int64_t)rr * ld + ch * 8) = v;
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // chain_kernel:  S = In F1^T (rows x r, accumulated in TMEM over the width of In), S rounded to bf16 into
 // shared memory, Out = S F2^T in 256-column chunks, stored as bf16.  One persistent CTA per SM.
@@ -147,7 +212,7 @@ __device__ __forceinline__ void store_bf16x16_swizzled(uint8_t* row_base, int ro
 // reduction index is the slow one -- A and B in the backward pass, where F1 = A^T and F2 = B^T), which the
 // shared-memory descriptors of the MMAs express directly; nothing is transposed in memory.
 __global__ void __launch_bounds__(kChainThreads, 1)
-chain_kernel(const __grid_constant__ CUtensorMap tmIn,
+chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ CUtensorMap tmIn4,
              const __grid_constant__ CUtensorMap tmF1, const __grid_constant__ CUtensorMap tmF2,
              const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmS, const ChainParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -162,7 +227,6 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g_begin = (int)((int64_t)blockIdx.x * p.groups / gridDim.x);
   const int g_end = (int)((int64_t)(blockIdx.x + 1) * p.groups / gridDim.x);
-  const int unit_groups = 4 * p.max_blocks;
   // All CTAs walk the same factor tiles.  Started together they would all ask L2 for the same few lines at
   // the same moment; each CTA therefore starts its walk at a different slab / chunk and wraps round.
   const int rot1 = blockIdx.x % p.nk1;
@@ -178,7 +242,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
     bars->abort_any = 0;
     bars->epi_abort = 0;
     fence_barrier_init();
-    tma_prefetch_desc(&tmIn); tma_prefetch_desc(&tmF1); tma_prefetch_desc(&tmF2);
+    tma_prefetch_desc(&tmIn); tma_prefetch_desc(&tmIn4); tma_prefetch_desc(&tmF1); tma_prefetch_desc(&tmF2);
     tma_prefetch_desc(&tmOut); tma_prefetch_desc(&tmS);
   }
   if (warp == 1) tmem_alloc(&bars->tmem_base, kTmemCols);
@@ -197,25 +261,40 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
       int i1 = 0, i2 = 0, u = 0;
       bool ok = true;
       for (int g = g_begin; g < g_end && ok; ++u) {
-        const int ng = (g_end - g < unit_groups) ? g_end - g : unit_groups;
-        const int nt = ng > 4 ? 2 : 1;
-        const int row0 = g * kGroupRows;
+        const Unit un = make_unit(p, g, g_end);
+        const int nt = un.nt;
         // the shared memory of the last unit is free once its MMAs are done and its stores have been read
         if (u > 0 && !mbar_wait(&bars->unit_done, (u - 1) & 1, lim)) { raise_timeout(bars, p.status); ok = false; break; }
         for (int ks = 0; ks < p.nk1 && ok; ++ks, ++i1) {
           const int slot = i1 % p.ns, ph = (i1 / p.ns) & 1;
           if (!mbar_wait(&bars->empty[slot], ph ^ 1, lim)) { raise_timeout(bars, p.status); ok = false; break; }
           uint8_t* dst = smem + (size_t)slot * p.slot_bytes;
-          mbar_arrive_expect_tx(&bars->full[slot], nt * kAtomBytes + p.f1_bytes);
           const int kr = (ks + rot1) % p.nk1;
-          // a block at the end of the run is loaded whole as well: the rows past the run are a neighbour's
-          // (or zeros past the last row) and cost less than four separate 32-row loads
-          for (int tt = 0; tt < nt; ++tt) tma_load_2d(dst + tt * kAtomBytes, &tmIn, &bars->full[slot], kr * 64, row0 + tt * 128);
           uint8_t* f1 = dst + p.max_blocks * kAtomBytes;
-          if (p.f1_mn)
-            for (int a = 0; a < p.natoms; ++a) tma_load_2d(f1 + a * kF1AtomBytes, &tmF1, &bars->full[slot], a * 64, kr * 64);
-          else
-            tma_load_2d(f1, &tmF1, &bars->full[slot], kr * 64, 0);
+          if (!p.cv.on) {
+            mbar_arrive_expect_tx(&bars->full[slot], nt * kAtomBytes + p.f1_bytes);
+            // a block at the end of the run is loaded whole as well: the rows past the run are a neighbour's
+            // (or zeros past the last row) and cost less than four separate 32-row loads
+            for (int tt = 0; tt < nt; ++tt)
+              tma_load_2d(dst + tt * kAtomBytes, &tmIn, &bars->full[slot], kr * 64, un.row0[tt]);
+            if (p.f1_mn)
+              for (int a = 0; a < p.natoms; ++a) tma_load_2d(f1 + a * kF1AtomBytes, &tmF1, &bars->full[slot], a * 64, kr * 64);
+            else
+              tma_load_2d(f1, &tmF1, &bars->full[slot], kr * 64, 0);
+          } else {
+            // slab kr = (tap, 64 channels): the tile's box of the activation, shifted by the tap
+            const int tap = kr / p.cv.cslabs, cs = kr - tap * p.cv.cslabs;
+            const int dy = (tap / 3 - 1) * p.cv.sign, dx = (tap % 3 - 1) * p.cv.sign;
+            mbar_arrive_expect_tx(&bars->full[slot], nt * p.cv.box_rows * 128 + p.f1_bytes);
+            for (int tt = 0; tt < nt; ++tt)
+              tma_load_4d(dst + tt * kAtomBytes, &tmIn4, &bars->full[slot], cs * 64, dx, un.y0[tt] + dy, un.b0[tt]);
+            const int fcol = tap * p.cv.tap_stride + p.cv.f1_col_off;
+            if (p.f1_mn)
+              for (int a = 0; a < p.natoms; ++a)
+                tma_load_2d(f1 + a * kF1AtomBytes, &tmF1, &bars->full[slot], fcol + a * 64, cs * 64);
+            else
+              tma_load_2d(f1, &tmF1, &bars->full[slot], fcol + cs * 64, 0);
+          }
         }
         // the second product's slots lie over the first product's: wait until its MMAs have read them
         if (ok && !mbar_wait(&bars->t_full, u & 1, lim)) { raise_timeout(bars, p.status); ok = false; }
@@ -232,7 +311,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
               tma_load_2d(d, &tmF2, &bars->full2[slot], j * 64, col0);
           }
         }
-        g += ng;
+        g += un.adv;
       }
     }
   } else if (warp == 1) {
@@ -244,8 +323,8 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
       int q0 = 0, q1 = 0;                      // uses of each accumulator so far
       bool ok = true;
       for (int g = g_begin; g < g_end && ok; ++u) {
-        const int ng = (g_end - g < unit_groups) ? g_end - g : unit_groups;
-        const int nt = ng > 4 ? 2 : 1;
+        const Unit un = make_unit(p, g, g_end);
+        const int nt = un.nt;
         for (int ks = 0; ks < p.nk1; ++ks, ++i1) {
           const int slot = i1 % p.ns, ph = (i1 / p.ns) & 1;
           if (!mbar_wait(&bars->full[slot], ph, lim)) { raise_timeout(bars, p.status); ok = false; break; }
@@ -253,7 +332,8 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
           const uint32_t sa = smem_u32(smem + (size_t)slot * p.slot_bytes);
           const uint32_t sf = sa + p.max_blocks * kAtomBytes;
           const uint64_t da0 = smem_desc_sw128(sa, 16), da1 = smem_desc_sw128(sa + kAtomBytes, 16);
-          int ksteps = (p.K1 - ((ks + rot1) % p.nk1) * 64 + 15) >> 4;
+          const int kr = (ks + rot1) % p.nk1;
+          int ksteps = p.cv.on ? (p.cv.in_ch - (kr % p.cv.cslabs) * 64 + 15) >> 4 : (p.K1 - kr * 64 + 15) >> 4;
           if (ksteps > 4) ksteps = 4;
           for (int kk = 0; kk < ksteps; ++kk) {
             const uint64_t db = p.f1_mn ? smem_desc_sw128(sf + kk * 2048, kF1AtomBytes) : smem_desc_sw128(sf, 16) + 2 * kk;
@@ -294,7 +374,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
           i2 += p.natoms;
         }
         if (ok) tc_commit(&bars->unit_done);
-        g += ng;
+        g += un.adv;
       }
     }
   } else {
@@ -309,9 +389,8 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
     int u = 0;
     bool ok = true;
     for (int g = g_begin; g < g_end && ok; ++u) {
-      const int ng = (g_end - g < unit_groups) ? g_end - g : unit_groups;
-      const int nt = ng > 4 ? 2 : 1;
-      const int row0 = g * kGroupRows;
+      const Unit un = make_unit(p, g, g_end);
+      const int nt = un.nt;
       ok = warp_wait(bars, &bars->t_full, u & 1, lim, p.status);
       if (!ok) break;
       tc_fence_after();
@@ -335,17 +414,23 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->s_ready);
-      if (p.save_s && lane == 0) {           // this warp's tiles, this warp's 32 rows, if the block has them
+      if (p.save_s) {                        // this warp's tiles, this warp's 32 rows, if the block has them
         for (int tt = 0; tt < nt; ++tt) {
-          const int gb = tt == 0 ? (ng < 4 ? ng : 4) : ng - 4;
-          if (qw >= gb) continue;
+          const int grows = un.nrows[tt] - qw * kGroupRows;      // rows of this warp's group in the block
+          if (grows <= 0) continue;
+          const int grow0 = un.row0[tt] + qw * kGroupRows;
           for (int j = 0; j < p.natoms; ++j) {
             if (((tt * p.natoms + j) % kWarpsPerQuarter) != hw) continue;
-            tma_store_2d(&tmS, S0 + ((size_t)tt * p.natoms + j) * kAtomBytes + qw * kGroupBytes, j * 64,
-                         row0 + tt * 128 + qw * kGroupRows);
+            const uint8_t* src = S0 + ((size_t)tt * p.natoms + j) * kAtomBytes + qw * kGroupBytes;
+            if (grows >= kGroupRows) {
+              if (lane == 0) tma_store_2d(&tmS, src, j * 64 + p.cv.s_col_off, grow0);
+            } else {
+              store_partial_group(src, p.s_ptr + (int64_t)grow0 * p.s_ld + p.cv.s_col_off + j * 64, p.s_ld, grows,
+                                  p.s_cols - j * 64);
+            }
           }
         }
-        tma_store_commit();
+        if (lane == 0) tma_store_commit();
       }
       for (int c = 0; c < p.nchunks && ok; ++c) {
         const int col0 = ((c + rot2) % p.nchunks) * kChunk + hw * (64 * kPiecesPerWarp);
@@ -355,8 +440,9 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
           if (!ok) break;
           if (b) ++q1; else ++q0;
           tc_fence_after();
-          const int gb = tt == 0 ? (ng < 4 ? ng : 4) : ng - 4;
-          const bool rows_live = qw < gb;                 // does this block hold this warp's group?
+          const int grows = un.nrows[tt] - qw * kGroupRows;   // rows of this warp's group in the block
+          const bool rows_live = grows > 0;
+          const int grow0 = un.row0[tt] + qw * kGroupRows;
           const uint32_t tacc = tmem_base + kChunk * b + lane_base + hw * (64 * kPiecesPerWarp);
           // the warp's 64-column pieces: each is read from TMEM and rounded to bf16 pairs at once (32
           // registers a piece); they are staged and stored after the accumulator has been handed back
@@ -394,9 +480,14 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
                   make_uint4(w[pc][4 * ch], w[pc][4 * ch + 1], w[pc][4 * ch + 2], w[pc][4 * ch + 3]);
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) {
-              tma_store_2d(&tmOut, buf, col0 + pc * 64, row0 + tt * 128 + qw * kGroupRows);
-              tma_store_commit();
+            if (grows >= kGroupRows) {
+              if (lane == 0) {
+                tma_store_2d(&tmOut, buf, col0 + pc * 64, grow0);
+                tma_store_commit();
+              }
+            } else {        // the last rows of a convolution tile: fewer than 32
+              store_partial_group(buf, p.out_ptr + (int64_t)grow0 * p.P + col0 + pc * 64, p.P, grows, p.P - (col0 + pc * 64));
+              __syncwarp();
             }
           }
         }
@@ -407,7 +498,7 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn,
         if (lane == 0) { tma_store_wait_read<0>(); mbar_arrive(&bars->unit_done); }
         __syncwarp();
       }
-      g += ng;
+      g += un.adv;
     }
     if (lane == 0) tma_store_wait_all();
   }
@@ -543,6 +634,138 @@ grad_kernel(const __grid_constant__ CUtensorMap tmAct0, const __grid_constant__ 
             for (int i = 0; i < 16; ++i) v[i] = 0.f;
           }
           if (prow < job.P) {
+            float4* o = reinterpret_cast<float4*>(out + c0);
+            o[0] = make_float4(v[0], v[1], v[2], v[3]);
+            o[1] = make_float4(v[4], v[5], v[6], v[7]);
+            o[2] = make_float4(v[8], v[9], v[10], v[11]);
+            o[3] = make_float4(v[12], v[13], v[14], v[15]);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*reinterpret_cast<volatile int*>(&bars->abort_any)) {
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// conv_grad_kernel: dB of a 3 x 3 convolution without materialised im2col rows,
+//   dB[j][tap * C + c] = sum over pixels of dT[pixel][j] * x[pixel shifted by the tap][c].
+// Same shape as grad_kernel (two 128-row accumulators per CTA, a slice of the reduction each, fp32 partials),
+// but the reduction runs over boxes of whole image rows (at most 64 pixels: bhk rows of one image, or kb whole
+// images), loaded with 4-D boxes: x shifted by the tap (zeros outside an image: the padding), dT unshifted.
+// A box may hold fewer than 64 pixels; the ring is zeroed once, so the rows no box ever writes stay zero in
+// both operands and add nothing.
+struct ConvGradParams {
+  int B, H, W, C;
+  int r, natoms, ns, slot_bytes;
+  int spi, kb, bhk, box_rows;    // slabs per image (kb == 1) or 1; images per slab; image rows per slab; pixels per box
+  int cpt;                       // 256-channel windows per tap
+  int slices, slabs_per_slice, nslabs;
+  float* partial;                // [slices][9 C][r]
+  int* status;
+};
+
+__global__ void __launch_bounds__(192, 1)
+conv_grad_kernel(const __grid_constant__ CUtensorMap tmX4, const __grid_constant__ CUtensorMap tmT4,
+                 const ConvGradParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* ring = smem;
+  Bars* bars = reinterpret_cast<Bars*>(ring + (size_t)p.ns * p.slot_bytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int tile = blockIdx.x;
+  const int slice = tile % p.slices;
+  const int chunk = tile / p.slices;
+  const int tap = chunk / p.cpt, cwin = (chunk - tap * p.cpt) * 256;
+  const int s_begin = slice * p.slabs_per_slice;
+  int s_end = s_begin + p.slabs_per_slice;
+  if (s_end > p.nslabs) s_end = p.nslabs;
+  const int nk = s_end > s_begin ? s_end - s_begin : 0;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.ns; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
+    mbar_init(&bars->t_full, 1);
+    bars->abort_any = 0;
+    bars->epi_abort = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&tmX4); tma_prefetch_desc(&tmT4);
+  }
+  {
+    uint4* z = reinterpret_cast<uint4*>(ring);
+    const int n16 = p.ns * p.slot_bytes / 16;
+    for (int i = threadIdx.x; i < n16; i += blockDim.x) z[i] = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) tmem_alloc(&bars->tmem_base, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
+  dep_wait();
+  dep_launch();
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const int dy = tap / 3 - 1, dx = tap % 3 - 1;
+      for (int i = 0; i < nk; ++i) {
+        const int slot = i % p.ns, ph = (i / p.ns) & 1;
+        if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { raise_timeout(bars, p.status); break; }
+        uint8_t* dst = ring + (size_t)slot * p.slot_bytes;
+        const int sl = s_begin + i;
+        const int grp = sl / p.spi, ty = sl - grp * p.spi;
+        const int b0 = grp * p.kb, y0 = ty * p.bhk;
+        mbar_arrive_expect_tx(&bars->full[slot], (4 + p.natoms) * p.box_rows * 128);
+        for (int a = 0; a < 4; ++a) tma_load_4d(dst + a * 8192, &tmX4, &bars->full[slot], cwin + a * 64, dx, y0 + dy, b0);
+        for (int a = 0; a < p.natoms; ++a) tma_load_4d(dst + 32768 + a * 8192, &tmT4, &bars->full[slot], a * 64, 0, y0, b0);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_bf16(128, p.r, 1, 1);
+      bool ok = true;
+      for (int i = 0; i < nk; ++i) {
+        const int slot = i % p.ns, ph = (i / p.ns) & 1;
+        if (!mbar_wait(&bars->full[slot], ph)) { raise_timeout(bars, p.status); ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = smem_u32(ring + (size_t)slot * p.slot_bytes);
+        for (int kk = 0; kk < 4; ++kk) {
+          const uint64_t db = smem_desc_sw128(sa + 32768 + kk * 2048, 8192);
+          tc_mma_bf16(tmem_base, smem_desc_sw128(sa + kk * 2048, 8192), db, idesc, (i | kk) != 0);
+          tc_mma_bf16(tmem_base + 256, smem_desc_sw128(sa + 16384 + kk * 2048, 8192), db, idesc, (i | kk) != 0);
+        }
+        tc_commit(&bars->empty[slot]);
+      }
+      if (ok) tc_commit(&bars->t_full);
+    }
+  } else {
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+    bool ok = true;
+    if (nk > 0) ok = epi_wait(bars, &bars->t_full, 0, p.status);
+    if (ok) {
+      tc_fence_after();
+      for (int mt = 0; mt < 2; ++mt) {
+        const int ch = cwin + mt * 128 + row;             // channel within the tap
+        float* out = p.partial + ((size_t)slice * 9 * p.C + (size_t)tap * p.C + ch) * p.r;
+        for (int c0 = 0; c0 < p.r; c0 += 16) {
+          float v[16];
+          if (nk > 0) tmem_ld16(tmem_base + mt * 256 + lane_base + c0, v);
+          else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = 0.f;
+          }
+          if (ch < p.C) {
             float4* o = reinterpret_cast<float4*>(out + c0);
             o[0] = make_float4(v[0], v[1], v[2], v[3]);
             o[1] = make_float4(v[4], v[5], v[6], v[7]);
@@ -758,6 +981,81 @@ BwdWs bwd_ws(void* ws, int64_t N, int m, int n, int r) {
   return w;
 }
 
+// Everything one launch of chain_kernel needs.  Regular mode: In is N x K1.  Convolution mode (cv != null): In is
+// the NHWC activation cv describes, N = B H W pixels, K1 is not used; F1 is the factor that holds the nine taps
+// side by side (r x 9 C as an operand, or, MN-major, stored (reduction index) x (9 C)).
+struct ChainLaunch {
+  const void* In; int64_t N; int K1;
+  const void* F1; int ldF1; int f1_rows, f1_cols;   // extents of F1 as it lies in memory
+  const void* F2; int ldF2; int P;
+  bool f_mn;
+  void* Out; void* Sg; int s_ld, s_cols;   // S is stored to Sg (row stride s_ld) at column cv->s_col_off
+  int r;                                   // width of S
+  const ConvGeom* cv;
+  int* status; bool clear_status;
+  bool stall_selftest; unsigned long long wait_ns;
+};
+
+int launch_chain_ex(const ChainLaunch& L, cudaStream_t st) {
+  const int rp = pad16(L.r);
+  const bool second = L.Out != nullptr && L.P > 0;
+  const int sms = sm_count();
+  if (sms <= 0) return AB_ERR_CUDA;
+  const bool conv = L.cv != nullptr;
+  int64_t items, per_unit;
+  if (conv) {
+    const int groups_of_images = (L.cv->B + L.cv->bb - 1) / L.cv->bb;
+    items = (int64_t)groups_of_images * L.cv->tpi;
+    per_unit = 1;
+  } else {
+    items = (L.N + kGroupRows - 1) / kGroupRows;
+    per_unit = 4;
+  }
+  const int grid = (int)(items < sms ? items : sms);
+  const int64_t per_cta = (items + grid - 1) / grid;
+  ChainPlan pl = chain_plan(rp, per_cta > per_unit ? 2 : 1, L.f_mn);
+  if (!pl.ok && pl.max_blocks == 2) pl = chain_plan(rp, 1, L.f_mn);
+  if (!pl.ok) return AB_ERR_UNSUPPORTED;
+  CUtensorMap tmIn, tmIn4, tmF1, tmF2, tmOut, tmS;
+  if (conv) {
+    AB_TRY(make_tensor_map_nhwc(&tmIn4, L.In, L.cv->B, L.cv->H, L.cv->W, L.cv->in_ch, L.cv->W, L.cv->bh, L.cv->bb));
+    AB_TRY(make_map(&tmF1, L.F1, L.f1_rows, L.f1_cols, L.ldF1, 64, L.f_mn ? 64 : rp));
+    tmIn = tmF1;
+  } else {
+    AB_TRY(make_map(&tmIn, L.In, (uint64_t)L.N, L.K1, L.K1, 64, 128));
+    tmIn4 = tmIn;
+    if (L.f_mn) AB_TRY(make_map(&tmF1, L.F1, L.K1, L.r, L.ldF1, 64, 64));
+    else AB_TRY(make_map(&tmF1, L.F1, L.r, L.K1, L.ldF1, 64, rp));
+  }
+  // unused maps still have to be valid objects: alias them to another operand
+  if (second) {
+    if (L.f_mn) AB_TRY(make_map(&tmF2, L.F2, L.r, L.P, L.ldF2, 64, 64));
+    else AB_TRY(make_map(&tmF2, L.F2, L.P, L.r, L.ldF2, 64, kChunk));
+    AB_TRY(make_map(&tmOut, L.Out, (uint64_t)L.N, L.P, L.P, 64, kGroupRows));
+  } else {
+    tmF2 = tmF1;
+    tmOut = tmF1;
+  }
+  if (L.Sg) AB_TRY(make_map(&tmS, L.Sg, (uint64_t)L.N, conv ? L.cv->s_col_off + L.s_cols : L.s_cols, L.s_ld, 64, kGroupRows));
+  else tmS = tmF1;
+  ChainParams q;
+  std::memset(&q, 0, sizeof(q));
+  q.K1 = L.K1; q.P = second ? L.P : 0; q.r = rp;
+  q.nk1 = conv ? 9 * L.cv->cslabs : (L.K1 + 63) / 64;
+  q.nchunks = second ? (L.P + kChunk - 1) / kChunk : 0;
+  q.natoms = pl.natoms; q.max_blocks = pl.max_blocks; q.ns = pl.ns; q.slot_bytes = pl.slot_bytes; q.ns2 = pl.ns2;
+  q.f1_bytes = pl.f1_bytes; q.f1_mn = L.f_mn ? 1 : 0; q.f2_mn = L.f_mn ? 1 : 0; q.save_s = L.Sg ? 1 : 0;
+  q.groups = (int)items; q.clear_status = L.clear_status ? 1 : 0; q.stall_selftest = L.stall_selftest ? 1 : 0;
+  q.wait_ns = L.wait_ns; q.status = L.status;
+  if (conv) q.cv = *L.cv;
+  q.out_ptr = static_cast<bf16*>(L.Out); q.s_ptr = static_cast<bf16*>(L.Sg); q.s_ld = L.s_ld; q.s_cols = L.s_cols;
+  AB_CUDA_OK(cudaFuncSetAttribute(chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
+  AB_LAUNCH_DEP(chain_kernel, dim3((unsigned)grid), dim3(kChainThreads), pl.smem, st, tmIn, tmIn4, tmF1, tmF2, tmOut,
+                tmS, q);
+  AB_LAUNCH_OK();
+  return AB_OK;
+}
+
 // S = In F1^T (saved to Sg if not null), Out = S F2^T (skipped if Out is null).
 // f_mn = false: F1 is given as r x K1 (row stride ldF1) and F2 as P x r (row stride ldF2);
 // f_mn = true : F1 is given transposed, K1 x r, and F2 transposed, r x P (the factors A and B as they lie in
@@ -765,42 +1063,11 @@ BwdWs bwd_ws(void* ws, int64_t N, int m, int n, int r) {
 int launch_chain(const void* In, int64_t N, int K1, const void* F1, int ldF1, const void* F2, int ldF2, int P,
                  bool f_mn, void* Out, void* Sg, int r, int* status, bool clear_status, cudaStream_t st,
                  bool stall_selftest = false, unsigned long long wait_ns = kWaitLimitNs) {
-  const int rp = pad16(r);
-  const bool second = Out != nullptr && P > 0;
-  const int sms = sm_count();
-  if (sms <= 0) return AB_ERR_CUDA;
-  const int64_t groups = (N + kGroupRows - 1) / kGroupRows;
-  const int grid = (int)(groups < sms ? groups : sms);
-  const int64_t per_cta = (groups + grid - 1) / grid;
-  ChainPlan pl = chain_plan(rp, per_cta > 4 ? 2 : 1, f_mn);
-  if (!pl.ok && pl.max_blocks == 2) pl = chain_plan(rp, 1, f_mn);
-  if (!pl.ok) return AB_ERR_UNSUPPORTED;
-  CUtensorMap tmIn, tmF1, tmF2, tmOut, tmS;
-  AB_TRY(make_map(&tmIn, In, (uint64_t)N, K1, K1, 64, 128));
-  if (f_mn) AB_TRY(make_map(&tmF1, F1, K1, r, ldF1, 64, 64));
-  else AB_TRY(make_map(&tmF1, F1, r, K1, ldF1, 64, rp));
-  // unused maps still have to be valid objects: alias them to the first operand
-  if (second) {
-    if (f_mn) AB_TRY(make_map(&tmF2, F2, r, P, ldF2, 64, 64));
-    else AB_TRY(make_map(&tmF2, F2, P, r, ldF2, 64, kChunk));
-    AB_TRY(make_map(&tmOut, Out, (uint64_t)N, P, P, 64, kGroupRows));
-  } else {
-    tmF2 = tmIn;
-    tmOut = tmIn;
-  }
-  if (Sg) AB_TRY(make_map(&tmS, Sg, (uint64_t)N, r, r, 64, kGroupRows));
-  else tmS = tmIn;
-  ChainParams q;
-  q.K1 = K1; q.P = second ? P : 0; q.r = rp; q.nk1 = (K1 + 63) / 64; q.nchunks = second ? (P + kChunk - 1) / kChunk : 0;
-  q.natoms = pl.natoms; q.max_blocks = pl.max_blocks; q.ns = pl.ns; q.slot_bytes = pl.slot_bytes; q.ns2 = pl.ns2;
-  q.f1_bytes = pl.f1_bytes; q.f1_mn = f_mn ? 1 : 0; q.f2_mn = f_mn ? 1 : 0; q.save_s = Sg ? 1 : 0;
-  q.groups = (int)groups; q.clear_status = clear_status ? 1 : 0; q.stall_selftest = stall_selftest ? 1 : 0;
-  q.wait_ns = wait_ns; q.status = status;
-  AB_CUDA_OK(cudaFuncSetAttribute(chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
-  AB_LAUNCH_DEP(chain_kernel, dim3((unsigned)grid), dim3(kChainThreads), pl.smem, st, tmIn, tmF1, tmF2, tmOut,
-                tmS, q);
-  AB_LAUNCH_OK();
-  return AB_OK;
+  ChainLaunch L;
+  L.In = In; L.N = N; L.K1 = K1; L.F1 = F1; L.ldF1 = ldF1; L.f1_rows = 0; L.f1_cols = 0; L.F2 = F2; L.ldF2 = ldF2; L.P = P;
+  L.f_mn = f_mn; L.Out = Out; L.Sg = Sg; L.s_ld = r; L.s_cols = r; L.r = r; L.cv = nullptr; L.status = status;
+  L.clear_status = clear_status; L.stall_selftest = stall_selftest; L.wait_ns = wait_ns;
+  return launch_chain_ex(L, st);
 }
 
 }  // namespace
@@ -840,6 +1107,20 @@ int make_tensor_map_2d(CUtensorMap* m, const void* ptr, bool f32, uint64_t rows,
   CUresult rc = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr),
                    dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? AB_OK : AB_ERR_CUDA;
+}
+
+int make_tensor_map_nhwc(CUtensorMap* m, const void* ptr, uint64_t B, uint64_t H, uint64_t W, uint64_t C,
+                         uint32_t bw, uint32_t bh, uint32_t bb) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return AB_ERR_CUDA;
+  cuuint64_t dims[4] = {C, W, H, B};
+  cuuint64_t strides[3] = {C * 2, W * C * 2, H * W * C * 2};
+  cuuint32_t box[4] = {64, bw, bh, bb};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult rc = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? AB_OK : AB_ERR_CUDA;
 }
 
@@ -931,6 +1212,177 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
     first = false;
   }
   if (first) AB_CUDA_OK(cudaMemsetAsync(w.status, 0, sizeof(int), st));   // nothing was asked for
+  return AB_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// 3 x 3 convolution (stride 1, padding 1, NHWC) with the factorised weight, im2col rows never materialised.
+namespace {
+
+ConvGeom conv_geom(int B, int H, int W, int in_ch, int sign, int tap_stride, int f1_col_off, int s_col_off) {
+  ConvGeom g;
+  g.on = 1; g.B = B; g.H = H; g.W = W; g.in_ch = in_ch; g.cslabs = (in_ch + 63) / 64;
+  if (H * W <= 128) { g.bb = 128 / (H * W); g.bh = H; g.tpi = 1; }
+  else {
+    const int bhmax = 128 / W;
+    g.bb = 1; g.tpi = (H + bhmax - 1) / bhmax; g.bh = (H + g.tpi - 1) / g.tpi;
+  }
+  g.box_rows = W * g.bh * g.bb;
+  g.sign = sign; g.tap_stride = tap_stride; g.f1_col_off = f1_col_off; g.s_col_off = s_col_off;
+  return g;
+}
+
+struct ConvGradPlan { int natoms, ns, slot_bytes, spi, kb, bhk, box_rows, cpt, slices, slabs_per_slice, nslabs; size_t smem; bool ok; };
+ConvGradPlan conv_grad_plan(int B, int H, int W, int C, int rp) {
+  ConvGradPlan pl;
+  pl.natoms = (rp + 63) / 64;
+  pl.slot_bytes = 32768 + pl.natoms * 8192;
+  const int fixed = (int)sizeof(Bars) + 1024;
+  pl.ns = (kSmemLimit - fixed) / pl.slot_bytes;
+  if (pl.ns > kMaxStages) pl.ns = kMaxStages;
+  pl.smem = (size_t)fixed + (size_t)pl.ns * pl.slot_bytes;
+  pl.ok = W <= 64 && pl.ns >= 2;
+  if (H * W <= 64) { pl.kb = 64 / (H * W); pl.bhk = H; pl.spi = 1; pl.nslabs = (B + pl.kb - 1) / pl.kb; }
+  else { pl.kb = 1; pl.bhk = W <= 64 ? 64 / W : 1; pl.spi = (H + pl.bhk - 1) / pl.bhk; pl.nslabs = B * pl.spi; }
+  pl.box_rows = W * pl.bhk * pl.kb;
+  pl.cpt = (C + 255) / 256;
+  const int chunks = 9 * pl.cpt;
+  int sms = sm_count();
+  if (sms <= 0) sms = 1;
+  int slices = sms / chunks;
+  if (slices < 1) slices = 1;
+  if (slices > pl.nslabs) slices = pl.nslabs;
+  pl.slabs_per_slice = (pl.nslabs + slices - 1) / slices;
+  pl.slices = (pl.nslabs + pl.slabs_per_slice - 1) / pl.slabs_per_slice;
+  return pl;
+}
+
+struct ConvWs { int* status; bf16 *T, *dT; float *pA, *pB; size_t bytes; };
+ConvWs conv_ws(void* ws, int B, int H, int W, int C, int m, int r) {
+  const int64_t N = (int64_t)B * H * W;
+  const int rp = pad16(r);
+  GradPlan ga = grad_plan(N, m, 0, r);
+  ConvGradPlan gb = conv_grad_plan(B, H, W, C, rp);
+  Arena ar(ws, 0);
+  ConvWs w;
+  w.status = ar.take_n<int>(64);
+  w.T = ar.take_n<bf16>((size_t)N * r);
+  w.dT = ar.take_n<bf16>((size_t)N * r);
+  w.pA = ar.take_n<float>((size_t)ga.slices * m * rp);
+  w.pB = ar.take_n<float>((size_t)gb.slices * 9 * C * rp);
+  w.bytes = align_up(ar.used, 256);
+  return w;
+}
+
+}  // namespace
+
+bool conv_tc_supported(int B, int H, int W, int C, int m, int r, int ldA, int ldB, int dt,
+                       const void* x, const void* A, const void* Bf) {
+  if (dt != AB_BF16) return false;
+  if (r % 8 != 0 || r < 8 || r > 256 || C % 8 != 0 || m % 8 != 0 || ldA % 8 != 0 || ldB % 8 != 0) return false;
+  if (B < 1 || H < 1 || W < 1 || W > 64 || H > 256 || (int64_t)B * H * W > ((int64_t)1 << 30)) return false;
+  if (!aligned(x, 16) || !aligned(A, 16) || !aligned(Bf, 16)) return false;
+  if (!device_is_sm100() || !encode_fn()) return false;
+  const int cw = C < 256 ? C : 256;
+  return chain_plan(pad16(r), 1, false).ok && chain_plan(pad16(r), 1, true).ok && chain_plan(pad16(cw), 1, true).ok &&
+         conv_grad_plan(B, H, W, C, pad16(r)).ok;
+}
+
+size_t conv_tc_ws(int B, int H, int W, int C, int m, int r) { return conv_ws(nullptr, B, H, W, C, m, r).bytes; }
+
+// y[pixel][:] = (sum over taps of x[pixel + tap][:] B_tap^T) A^T, B_tap = columns tap C .. tap C + C of B
+int conv_tc_forward(const void* x, const void* A, const void* Bf, void* y, void* T_save, int B, int H, int W, int C,
+                    int m, int r, int ldA, int ldB, void* ws, size_t ws_bytes, cudaStream_t st) {
+  if (!ws || ws_bytes < 256) return AB_ERR_WORKSPACE;
+  if ((T_save && !aligned(T_save, 16)) || !aligned(y, 16)) return AB_ERR_INVALID_ARG;
+  const ConvGeom g = conv_geom(B, H, W, C, +1, C, 0, 0);
+  ChainLaunch L;
+  L.In = x; L.N = (int64_t)B * H * W; L.K1 = 0; L.F1 = Bf; L.ldF1 = ldB; L.f1_rows = r; L.f1_cols = 9 * C;
+  L.F2 = A; L.ldF2 = ldA; L.P = m; L.f_mn = false; L.Out = y; L.Sg = T_save; L.s_ld = r; L.s_cols = r; L.r = r; L.cv = &g;
+  L.status = static_cast<int*>(ws); L.clear_status = true; L.stall_selftest = false; L.wait_ns = kWaitLimitNs;
+  return launch_chain_ex(L, st);
+}
+
+// dT = dY A; dX[pixel][c] = sum over taps of dT[pixel - tap][:] B[:, tap C + c] (the col2im sum, folded into the
+// reduction); dA = dY^T T; dB[j][tap C + c] = sum over pixels of dT[pixel][j] x[pixel + tap][c].
+int conv_tc_backward(const void* x, const void* dY, const void* A, const void* Bf, const void* T_saved, void* dX,
+                     float* dA, float* dB, int B, int H, int W, int C, int m, int r, int ldA, int ldB,
+                     void* ws, size_t ws_bytes, cudaStream_t st) {
+  if (!ws) return AB_ERR_WORKSPACE;
+  ConvWs w = conv_ws(ws, B, H, W, C, m, r);
+  if (w.bytes > ws_bytes) return AB_ERR_WORKSPACE;
+  if ((dX && !aligned(dX, 16)) || (T_saved && !aligned(T_saved, 16)) || (dA && !aligned(dA, 16)) || (dB && !aligned(dB, 16)))
+    return AB_ERR_INVALID_ARG;
+  const int64_t N = (int64_t)B * H * W;
+  const int rp = pad16(r);
+  bool first = true;
+  const bf16* T = static_cast<const bf16*>(T_saved);
+  if (dA && !T) {      // T rebuilt from x (first product of the forward pass only)
+    const ConvGeom g = conv_geom(B, H, W, C, +1, C, 0, 0);
+    ChainLaunch L;
+    L.In = x; L.N = N; L.K1 = 0; L.F1 = Bf; L.ldF1 = ldB; L.f1_rows = r; L.f1_cols = 9 * C; L.F2 = nullptr; L.ldF2 = 0; L.P = 0;
+    L.f_mn = false; L.Out = nullptr; L.Sg = w.T; L.s_ld = r; L.s_cols = r; L.r = r; L.cv = &g; L.status = w.status;
+    L.clear_status = first; L.stall_selftest = false; L.wait_ns = kWaitLimitNs;
+    AB_TRY(launch_chain_ex(L, st));
+    first = false;
+    T = w.T;
+  }
+  if (dX || dB) {
+    AB_TRY(launch_chain(dY, N, m, A, ldA, nullptr, 0, 0, true, nullptr, w.dT, r, w.status, first, st));   // dT = dY A
+    first = false;
+  }
+  if (dX) {
+    for (int c0 = 0; c0 < C; c0 += 256) {      // 256 channels of dX per launch: the width of one accumulator
+      const int cw = C - c0 < 256 ? C - c0 : 256;
+      const ConvGeom g = conv_geom(B, H, W, r, -1, C, c0, c0);
+      ChainLaunch L;
+      L.In = w.dT; L.N = N; L.K1 = 0; L.F1 = Bf; L.ldF1 = ldB; L.f1_rows = r; L.f1_cols = 9 * C; L.F2 = nullptr; L.ldF2 = 0;
+      L.P = 0; L.f_mn = true; L.Out = nullptr; L.Sg = dX; L.s_ld = C; L.s_cols = cw; L.r = cw; L.cv = &g; L.status = w.status;
+      L.clear_status = false; L.stall_selftest = false; L.wait_ns = kWaitLimitNs;
+      AB_TRY(launch_chain_ex(L, st));
+    }
+  }
+  if (dA) {
+    GradPlan gp = grad_plan(N, m, 0, r);
+    GradParams p;
+    std::memset(&p, 0, sizeof(p));
+    CUtensorMap tmAct, tmSmall;
+    AB_TRY(make_map(&tmAct, dY, (uint64_t)N, m, m, 64, 64));
+    AB_TRY(make_map(&tmSmall, T, (uint64_t)N, r, r, 64, 64));
+    p.job[0].P = m; p.job[0].chunks = (m + 255) / 256; p.job[0].partial = w.pA;
+    p.job[1] = p.job[0]; p.job[1].chunks = 0;
+    p.njobs = 1; p.r = rp; p.natoms = gp.natoms; p.ns = gp.ns; p.slot_bytes = gp.slot_bytes;
+    p.slices = gp.slices; p.rows_per_slice = gp.rows_per_slice; p.N = (int)N; p.clear_status = first ? 1 : 0;
+    p.status = w.status; p.job0_independent = 0;
+    AB_CUDA_OK(cudaFuncSetAttribute(grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gp.smem));
+    AB_LAUNCH_DEP(grad_kernel, dim3((unsigned)(p.job[0].chunks * gp.slices)), dim3(192), gp.smem, st, tmAct, tmSmall, tmAct,
+                  tmSmall, p);
+    AB_LAUNCH_OK();
+    first = false;
+    const int nA = (int)(((int64_t)m * r / 4 + 255) / 256);
+    AB_LAUNCH_DEP(reduce_partials_kernel, dim3(nA), dim3(256), 0, st, static_cast<const float*>(w.pA), dA, m, nA,
+                  static_cast<const float*>(w.pA), static_cast<float*>(nullptr), 0, gp.slices, r, rp);
+    AB_LAUNCH_OK();
+  }
+  if (dB) {
+    ConvGradPlan gp = conv_grad_plan(B, H, W, C, rp);
+    ConvGradParams p;
+    std::memset(&p, 0, sizeof(p));
+    CUtensorMap tmX4, tmT4;
+    AB_TRY(make_tensor_map_nhwc(&tmX4, x, B, H, W, C, W, gp.bhk, gp.kb));
+    AB_TRY(make_tensor_map_nhwc(&tmT4, w.dT, B, H, W, r, W, gp.bhk, gp.kb));
+    p.B = B; p.H = H; p.W = W; p.C = C; p.r = rp; p.natoms = gp.natoms; p.ns = gp.ns; p.slot_bytes = gp.slot_bytes;
+    p.spi = gp.spi; p.kb = gp.kb; p.bhk = gp.bhk; p.box_rows = gp.box_rows; p.cpt = gp.cpt; p.slices = gp.slices;
+    p.slabs_per_slice = gp.slabs_per_slice; p.nslabs = gp.nslabs; p.partial = w.pB; p.status = w.status;
+    AB_CUDA_OK(cudaFuncSetAttribute(conv_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gp.smem));
+    AB_LAUNCH_DEP(conv_grad_kernel, dim3((unsigned)(9 * gp.cpt * gp.slices)), dim3(192), gp.smem, st, tmX4, tmT4, p);
+    AB_LAUNCH_OK();
+    const int nB = ((9 * C + 31) / 32) * ((r + 31) / 32);
+    AB_LAUNCH_DEP(reduce_partials_kernel, dim3(nB), dim3(256), 0, st, static_cast<const float*>(w.pB), static_cast<float*>(nullptr),
+                  0, 0, static_cast<const float*>(w.pB), dB, 9 * C, gp.slices, r, rp);
+    AB_LAUNCH_OK();
+  }
+  if (first) AB_CUDA_OK(cudaMemsetAsync(w.status, 0, sizeof(int), st));
   return AB_OK;
 }
 

@@ -122,6 +122,10 @@ int64_t split_job_blocks(int rows, int cols);
 int split3_batched(const SplitJob* d_jobs, int njobs, int64_t total_blocks, cudaStream_t st);
 int sum_slices(const float* part, float* out, int64_t count, int64_t slice_stride, int slices, cudaStream_t st);
 
+// ---- dense layer of the full-rank phases (ab_dense.cu) ------------------------------------------
+size_t dense_forward_ws(int64_t N, int m, int n);
+size_t dense_backward_ws(int64_t N, int m, int n);
+
 // ---- fused tensor-core chain (ab_chain_tc.cu) --------------------------------------------------
 bool chain_tc_supported(int64_t N, int m, int n, int r, int ldA, int ldB, int dt,
                         const void* x, const void* A, const void* B, const void* y);
@@ -134,6 +138,16 @@ int chain_tc_backward(const void* x, const void* dY, const void* A, const void* 
                       const void* T_saved, void* dX, float* dA, float* dB,
                       int64_t N, int m, int n, int r, int ldA, int ldB,
                       void* ws, size_t ws_bytes, cudaStream_t st);
+
+// 3 x 3 convolution with the factorised weight on NHWC activations, im2col rows never formed (ab_chain_tc.cu)
+bool conv_tc_supported(int B, int H, int W, int C, int m, int r, int ldA, int ldB, int dt,
+                       const void* x, const void* A, const void* Bf);
+size_t conv_tc_ws(int B, int H, int W, int C, int m, int r);
+int conv_tc_forward(const void* x, const void* A, const void* Bf, void* y, void* T_save, int B, int H, int W, int C,
+                    int m, int r, int ldA, int ldB, void* ws, size_t ws_bytes, cudaStream_t st);
+int conv_tc_backward(const void* x, const void* dY, const void* A, const void* Bf, const void* T_saved, void* dX,
+                     float* dA, float* dB, int B, int H, int W, int C, int m, int r, int ldA, int ldB,
+                     void* ws, size_t ws_bytes, cudaStream_t st);
 
 int bounded_wait_selftest(int* dev_status, unsigned limit_us, cudaStream_t st);
 size_t chain_stall_selftest_ws();

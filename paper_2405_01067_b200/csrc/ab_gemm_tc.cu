@@ -39,7 +39,7 @@ constexpr int kMaxTerms = 6;
 
 struct TcBars {
   uint64_t full[kStages], empty[kStages];
-  uint64_t acc_full;
+  uint64_t acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   int abort_any;
 };
@@ -57,7 +57,7 @@ struct alignas(64) TcProblemDev {
   int ksplit;               // slices of K
   int kslice;               // K per slice, a multiple of 64
   int c_rows;               // rows of one partial result in the output map (M when ksplit == 1)
-  int first_tile;           // first block of this problem in the grid
+  int first_tile;           // index of this problem's first tile among all tiles of the batch
   const int* live_rows;     // optional device ints: rows / columns at or beyond them are written as zero
   const int* live_cols;
 };
@@ -67,8 +67,39 @@ __device__ __forceinline__ void tc_raise(TcBars* b, int* status) {
   atomicExch(status, (int)AB_ERR_TIMEOUT);
 }
 
+// What one tile of the batch is: its problem, its corner, its slice of K.
+struct TileInfo {
+  const TcProblemDev* P;
+  int m0, n0, slice, k_begin, k_end, nslab, ncols, nmma;
+};
+__device__ __forceinline__ TileInfo decode_tile(const TcProblemDev* __restrict__ probs, int nprobs, int tile) {
+  int lo = 0, hi = nprobs - 1;
+  while (lo < hi) {                       // the last problem whose first tile is <= tile
+    const int mid = (lo + hi + 1) >> 1;
+    if (probs[mid].first_tile <= tile) lo = mid; else hi = mid - 1;
+  }
+  TileInfo ti;
+  ti.P = probs + lo;
+  int t = tile - ti.P->first_tile;
+  ti.slice = t % ti.P->ksplit;
+  t /= ti.P->ksplit;
+  ti.n0 = (t % ti.P->tiles_n) * kBN;
+  ti.m0 = (t / ti.P->tiles_n) * kBM;
+  ti.k_begin = ti.slice * ti.P->kslice;
+  ti.k_end = ti.k_begin + ti.P->kslice;
+  if (ti.k_end > ti.P->K) ti.k_end = ti.P->K;
+  ti.nslab = ti.k_end > ti.k_begin ? (ti.k_end - ti.k_begin + kBK - 1) / kBK : 0;
+  ti.ncols = ti.P->N - ti.n0;
+  if (ti.ncols > kBN) ti.ncols = kBN;
+  ti.nmma = (ti.ncols + 15) & ~15;
+  return ti;
+}
+
+// Persistent CTAs: CTA b takes the tiles b, b + gridDim.x, ... of the batch.  Two 256-column accumulators in
+// TMEM alternate between a CTA's tiles, so the epilogue of one tile (TMEM -> staging -> TMA stores) runs
+// beside the loads and MMAs of the next.
 __global__ void __launch_bounds__(kTcThreads, 1)
-gemm_tc_kernel(const TcProblemDev* __restrict__ probs, int nprobs, int* status) {
+gemm_tc_kernel(const TcProblemDev* __restrict__ probs, int nprobs, int ntiles, int* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* ring = smem;
@@ -76,35 +107,13 @@ gemm_tc_kernel(const TcProblemDev* __restrict__ probs, int nprobs, int* status) 
   TcBars* bars = reinterpret_cast<TcBars*>(stg + 4 * 2 * kStgBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  // which problem: the last one whose first tile is <= blockIdx.x
-  int lo = 0, hi = nprobs - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (probs[mid].first_tile <= (int)blockIdx.x) lo = mid; else hi = mid - 1;
-  }
-  const TcProblemDev* P = probs + lo;
-  int t = (int)blockIdx.x - P->first_tile;
-  const int slice = t % P->ksplit;
-  t /= P->ksplit;
-  const int tn = t % P->tiles_n, tm = t / P->tiles_n;
-  const int m0 = tm * kBM, n0 = tn * kBN;
-  const int k_begin = slice * P->kslice;
-  int k_end = k_begin + P->kslice;
-  if (k_end > P->K) k_end = P->K;
-  const int nslab = k_end > k_begin ? (k_end - k_begin + kBK - 1) / kBK : 0;
-  const int nterms = P->nterms;
-  const int a_mn = P->a_mn, b_mn = P->b_mn;
-  int ncols = P->N - n0;                       // columns of this tile, rounded up to the MMA's granularity
-  if (ncols > kBN) ncols = kBN;
-  const int nmma = (ncols + 15) & ~15;
-
   if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
-    mbar_init(&bars->acc_full, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 4); }
     bars->abort_any = 0;
     fence_barrier_init();
   }
-  if (warp == 1) tmem_alloc(&bars->tmem_base, 256);
+  if (warp == 1) tmem_alloc(&bars->tmem_base, 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -115,74 +124,96 @@ gemm_tc_kernel(const TcProblemDev* __restrict__ probs, int nprobs, int* status) 
     if (lane == 0) {
       int i = 0;
       bool ok = true;
-      for (int tix = 0; tix < nterms && ok; ++tix) {
-        const CUtensorMap* ma = &P->a[P->term_a[tix]];
-        const CUtensorMap* mb = &P->b[P->term_b[tix]];
-        for (int ks = 0; ks < nslab; ++ks, ++i) {
-          const int slot = i % kStages, ph = (i / kStages) & 1;
-          if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { tc_raise(bars, status); ok = false; break; }
-          uint8_t* da = ring + (size_t)slot * kStage;
-          uint8_t* db = da + kAStage;
-          const int k0 = k_begin + ks * kBK;
-          mbar_arrive_expect_tx(&bars->full[slot], kStage);
-          if (a_mn) { for (int h = 0; h < 2; ++h) tma_load_2d(da + h * 8192, ma, &bars->full[slot], m0 + 64 * h, k0); }
-          else tma_load_2d(da, ma, &bars->full[slot], k0, m0);
-          if (b_mn) { for (int h = 0; h < 4; ++h) tma_load_2d(db + h * 8192, mb, &bars->full[slot], n0 + 64 * h, k0); }
-          else tma_load_2d(db, mb, &bars->full[slot], k0, n0);
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+        const TileInfo ti = decode_tile(probs, nprobs, tile);
+        const TcProblemDev* P = ti.P;
+        const int a_mn = P->a_mn, b_mn = P->b_mn;
+        for (int tix = 0; tix < P->nterms && ok; ++tix) {
+          const CUtensorMap* ma = &P->a[P->term_a[tix]];
+          const CUtensorMap* mb = &P->b[P->term_b[tix]];
+          for (int ks = 0; ks < ti.nslab; ++ks, ++i) {
+            const int slot = i % kStages, ph = (i / kStages) & 1;
+            if (!mbar_wait(&bars->empty[slot], ph ^ 1)) { tc_raise(bars, status); ok = false; break; }
+            uint8_t* da = ring + (size_t)slot * kStage;
+            uint8_t* db = da + kAStage;
+            const int k0 = ti.k_begin + ks * kBK;
+            mbar_arrive_expect_tx(&bars->full[slot], kStage);
+            if (a_mn) { for (int h = 0; h < 2; ++h) tma_load_2d(da + h * 8192, ma, &bars->full[slot], ti.m0 + 64 * h, k0); }
+            else tma_load_2d(da, ma, &bars->full[slot], k0, ti.m0);
+            if (b_mn) { for (int h = 0; h < 4; ++h) tma_load_2d(db + h * 8192, mb, &bars->full[slot], ti.n0 + 64 * h, k0); }
+            else tma_load_2d(db, mb, &bars->full[slot], k0, ti.n0);
+          }
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = instr_desc_bf16(kBM, nmma, a_mn, b_mn);
-      int i = 0;
+      int i = 0, it = 0;
       bool ok = true;
-      for (int tix = 0; tix < nterms && ok; ++tix) {
-        for (int ks = 0; ks < nslab; ++ks, ++i) {
-          const int slot = i % kStages, ph = (i / kStages) & 1;
-          if (!mbar_wait(&bars->full[slot], ph)) { tc_raise(bars, status); ok = false; break; }
-          tc_fence_after();
-          const uint32_t sa = smem_u32(ring + (size_t)slot * kStage), sb = sa + kAStage;
-          int ksteps = (k_end - (k_begin + ks * kBK) + 15) >> 4;
-          if (ksteps > 4) ksteps = 4;
-          for (int kk = 0; kk < ksteps; ++kk) {
-            const uint64_t da = a_mn ? smem_desc_sw128(sa + kk * 2048, 8192) : smem_desc_sw128(sa, 16) + 2 * kk;
-            const uint64_t db = b_mn ? smem_desc_sw128(sb + kk * 2048, 8192) : smem_desc_sw128(sb, 16) + 2 * kk;
-            tc_mma_bf16(tmem_base, da, db, idesc, (i | kk) != 0);
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+        const TileInfo ti = decode_tile(probs, nprobs, tile);
+        const TcProblemDev* P = ti.P;
+        const int a_mn = P->a_mn, b_mn = P->b_mn;
+        const uint32_t idesc = instr_desc_bf16(kBM, ti.nmma, a_mn, b_mn);
+        const int b = it & 1;
+        if (!mbar_wait(&bars->acc_empty[b], ((it >> 1) & 1) ^ 1)) { tc_raise(bars, status); ok = false; break; }
+        tc_fence_after();
+        const uint32_t tacc = tmem_base + 256 * b;
+        int first = 1;
+        for (int tix = 0; tix < P->nterms && ok; ++tix) {
+          for (int ks = 0; ks < ti.nslab; ++ks, ++i) {
+            const int slot = i % kStages, ph = (i / kStages) & 1;
+            if (!mbar_wait(&bars->full[slot], ph)) { tc_raise(bars, status); ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = smem_u32(ring + (size_t)slot * kStage), sb = sa + kAStage;
+            int ksteps = (ti.k_end - (ti.k_begin + ks * kBK) + 15) >> 4;
+            if (ksteps > 4) ksteps = 4;
+            for (int kk = 0; kk < ksteps; ++kk) {
+              const uint64_t da = a_mn ? smem_desc_sw128(sa + kk * 2048, 8192) : smem_desc_sw128(sa, 16) + 2 * kk;
+              const uint64_t db = b_mn ? smem_desc_sw128(sb + kk * 2048, 8192) : smem_desc_sw128(sb, 16) + 2 * kk;
+              tc_mma_bf16(tacc, da, db, idesc, first ? 0u : 1u);
+              first = 0;
+            }
+            tc_commit(&bars->empty[slot]);
           }
-          tc_commit(&bars->empty[slot]);
         }
+        if (ok) tc_commit(&bars->acc_full[b]);
       }
-      if (ok) tc_commit(&bars->acc_full);
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int qw = warp & 3;
     const uint32_t lane_base = (uint32_t)(qw * 32) << 16;
     uint8_t* mystg = stg + (size_t)(warp - 2) * 2 * kStgBytes;
-    const int grow = m0 + qw * 32 + lane;           // row of C this thread holds
-    const int live_r = P->live_rows ? *P->live_rows : P->M;
-    const int live_c = P->live_cols ? *P->live_cols : P->N;
-    const bool rows_in = m0 + qw * 32 < P->M;
+    int nst = 0, it = 0;
     bool ok = true;
-    if (nslab > 0 && nterms > 0) {
-      int w = 1;
-      if (lane == 0) { w = mbar_wait(&bars->acc_full, 0) ? 1 : 0; if (!w) tc_raise(bars, status); }
-      ok = __shfl_sync(0xffffffffu, w, 0) != 0;
-    }
-    if (ok && rows_in) {
+    for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+      const TileInfo ti = decode_tile(probs, nprobs, tile);
+      const TcProblemDev* P = ti.P;
+      const int b = it & 1;
+      const bool have_acc = ti.nslab > 0 && P->nterms > 0;      // an empty reduction leaves zeros
+      {
+        int w = 1;
+        if (lane == 0) { w = mbar_wait(&bars->acc_full[b], (it >> 1) & 1) ? 1 : 0; if (!w) tc_raise(bars, status); }
+        ok = __shfl_sync(0xffffffffu, w, 0) != 0;
+      }
+      if (!ok) break;
       tc_fence_after();
-      const int pcols = P->c_f32 ? 32 : 64;          // columns of one 128-byte piece
-      const int crow = slice * P->c_rows + m0 + qw * 32;
-      int nst = 0;
-      for (int c0 = 0; c0 < ncols; c0 += pcols, ++nst) {
+      const int grow = ti.m0 + qw * 32 + lane;           // row of C this thread holds
+      const int live_r = P->live_rows ? *P->live_rows : P->M;
+      const int live_c = P->live_cols ? *P->live_cols : P->N;
+      const bool rows_in = ti.m0 + qw * 32 < P->M;
+      const int c_f32 = P->c_f32;
+      const int pcols = c_f32 ? 32 : 64;                 // columns of one 128-byte piece
+      const int crow = ti.slice * P->c_rows + ti.m0 + qw * 32;
+      const uint32_t tacc = tmem_base + 256 * b + lane_base;
+      for (int c0 = 0; c0 < ti.ncols; c0 += pcols) {
         uint32_t v[4][16];
-        const int nld = pcols / 16;
-        if (nslab > 0 && nterms > 0) {
+        if (have_acc && rows_in) {
 #pragma unroll
           for (int gq = 0; gq < 4; ++gq)
-            if (gq < nld) tmem_ld16_nowait(tmem_base + lane_base + c0 + gq * 16, v[gq]);
+            if (gq * 16 < pcols) tmem_ld16_nowait(tacc + c0 + gq * 16, v[gq]);
           tmem_wait_ld();
         } else {
 #pragma unroll
@@ -190,17 +221,24 @@ gemm_tc_kernel(const TcProblemDev* __restrict__ probs, int nprobs, int* status) 
 #pragma unroll
             for (int e = 0; e < 16; ++e) v[gq][e] = 0u;
         }
+        if (c0 + pcols >= ti.ncols) {                    // the last piece is in registers: hand the accumulator back
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->acc_empty[b]);
+        }
+        if (!rows_in) continue;
         const bool row_dead = grow >= live_r;
 #pragma unroll
         for (int gq = 0; gq < 4; ++gq)
 #pragma unroll
           for (int e = 0; e < 16; ++e)
-            if (row_dead || n0 + c0 + gq * 16 + e >= live_c) v[gq][e] = 0u;
+            if (row_dead || ti.n0 + c0 + gq * 16 + e >= live_c) v[gq][e] = 0u;
         uint8_t* buf = mystg + (nst & 1) * kStgBytes;
+        ++nst;
         if (lane == 0) tma_store_wait_read<1>();
         __syncwarp();
         uint8_t* rowp = buf + lane * 128;
-        if (P->c_f32) {
+        if (c_f32) {
 #pragma unroll
           for (int ch = 0; ch < 8; ++ch)
             *reinterpret_cast<uint4*>(rowp + ((ch ^ (lane & 7)) << 4)) =
@@ -223,7 +261,7 @@ gemm_tc_kernel(const TcProblemDev* __restrict__ probs, int nprobs, int* status) 
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_2d(&P->c, buf, n0 + c0, crow);
+          tma_store_2d(&P->c, buf, ti.n0 + c0, crow);
           tma_store_commit();
         }
       }
@@ -240,10 +278,9 @@ gemm_tc_kernel(const TcProblemDev* __restrict__ probs, int nprobs, int* status) 
   }
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 256);
+    tmem_dealloc(tmem_base, 512);
   }
 }
-
 
 // ---------------------------------------------------------------------------------------------
 // fp32 -> three bf16 pieces: hi = bf16(x), mid = bf16(x - hi), lo = bf16(x - hi - mid); hi + mid + lo = x to
@@ -256,19 +293,42 @@ split3_kernel(const SplitJob* __restrict__ jobs, int njobs) {
     if (jobs[mid].first_block <= (int64_t)blockIdx.x) lo = mid; else hi = mid - 1;
   }
   const SplitJob j = jobs[lo];
-  const int64_t i = ((int64_t)blockIdx.x - j.first_block) * 256 + threadIdx.x;
-  const int64_t total = (int64_t)j.rows * j.cols;
-  if (i >= total) return;
-  const int64_t r = i / j.cols, c = i - r * j.cols;
-  const float x = j.src[r * j.ld_src + c];
-  const bf16 h = __float2bfloat16_rn(x);
-  const float r1 = x - __bfloat162float(h);
-  const bf16 m = __float2bfloat16_rn(r1);
-  const float r2 = r1 - __bfloat162float(m);
-  const int64_t o = r * j.ld_dst + c;
-  j.hi[o] = h;
-  j.mid[o] = m;
-  j.lo[o] = __float2bfloat16_rn(r2);
+  // four consecutive elements of a row per thread when the rows allow 16-byte loads and 8-byte stores
+  const bool vec = (j.cols & 3) == 0 && (j.ld_src & 3) == 0 && (j.ld_dst & 3) == 0 &&
+                   ((reinterpret_cast<uintptr_t>(j.src) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(j.hi) & 7u) == 0) &&
+                   ((reinterpret_cast<uintptr_t>(j.mid) & 7u) == 0) && ((reinterpret_cast<uintptr_t>(j.lo) & 7u) == 0);
+  const unsigned cols4 = (unsigned)(j.cols + 3) >> 2;
+  const unsigned total4 = (unsigned)j.rows * cols4;
+  const unsigned i = (unsigned)((int64_t)blockIdx.x - j.first_block) * 256u + threadIdx.x;
+  if (i >= total4) return;
+  const unsigned r = i / cols4, c = (i - r * cols4) * 4u;
+  float x[4];
+  const float* src = j.src + (int64_t)r * j.ld_src + c;
+  if (vec) {
+    const float4 q = *reinterpret_cast<const float4*>(src);
+    x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w;
+  } else {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) x[e] = (c + e < (unsigned)j.cols) ? src[e] : 0.f;
+  }
+  bf16 h[4], m[4], l[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    h[e] = __float2bfloat16_rn(x[e]);
+    const float r1 = x[e] - __bfloat162float(h[e]);
+    m[e] = __float2bfloat16_rn(r1);
+    l[e] = __float2bfloat16_rn(r1 - __bfloat162float(m[e]));
+  }
+  const int64_t o = (int64_t)r * j.ld_dst + c;
+  if (vec) {
+    *reinterpret_cast<uint2*>(j.hi + o) = *reinterpret_cast<const uint2*>(h);
+    *reinterpret_cast<uint2*>(j.mid + o) = *reinterpret_cast<const uint2*>(m);
+    *reinterpret_cast<uint2*>(j.lo + o) = *reinterpret_cast<const uint2*>(l);
+  } else {
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (c + e < (unsigned)j.cols) { j.hi[o + e] = h[e]; j.mid[o + e] = m[e]; j.lo[o + e] = l[e]; }
+  }
 }
 
 // out[i] = sum over slices of part[s][i], ascending s (fixed order); partials are rows_pad x ld, out is rows x ld
@@ -283,7 +343,7 @@ sum_slices_kernel(const float* __restrict__ part, float* __restrict__ out, int64
 
 }  // namespace
 
-int64_t split_job_blocks(int rows, int cols) { return ((int64_t)rows * cols + 255) / 256; }
+int64_t split_job_blocks(int rows, int cols) { return ((int64_t)rows * ((cols + 3) / 4) + 255) / 256; }
 
 int split3_batched(const SplitJob* d_jobs, int njobs, int64_t total_blocks, cudaStream_t st) {
   if (njobs <= 0 || total_blocks <= 0) return AB_OK;
@@ -353,7 +413,10 @@ int gemm_tc_batched(const TcProblem* probs, int count, void* table_dev, int* sta
   AB_CUDA_OK(cudaMemcpyAsync(table_dev, tab.data(), tab.size() * sizeof(TcProblemDev), cudaMemcpyHostToDevice, st));
   const size_t smem = (size_t)kStages * kStage + 4 * 2 * kStgBytes + sizeof(TcBars) + 1024;
   AB_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  gemm_tc_kernel<<<(unsigned)tiles, kTcThreads, smem, st>>>(static_cast<const TcProblemDev*>(table_dev), count, status);
+  int sms = sm_count();
+  if (sms <= 0) return AB_ERR_CUDA;
+  const int grid = tiles < sms ? tiles : sms;
+  gemm_tc_kernel<<<(unsigned)grid, kTcThreads, smem, st>>>(static_cast<const TcProblemDev*>(table_dev), count, tiles, status);
   AB_LAUNCH_OK();
   return AB_OK;
 }

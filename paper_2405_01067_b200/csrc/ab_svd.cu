@@ -38,9 +38,9 @@ constexpr int kInnerSweeps = 2;
 constexpr float kCountRel2 = 1e-8f;  // rows below 1e-4 of the largest norm do not hold up convergence
 constexpr float kDeadRel2 = 1e-12f;   // rows below 1e-6 of the largest norm count as zero
 // Accuracy domain of this route: a kept singular value between kZeroRel and kDomainRel of the largest has lost
-// relative accuracy to the squaring in the Gram matrix (measured: 5e-6 at 1-2 %, 5e-3 at 0.5-1 %); the status
-// word then says so.  Below kZeroRel a value is zero to working precision (a W of lower rank than asked for).
-constexpr float kDomainRel = 1e-2f, kZeroRel = 1e-5f;
+// relative accuracy to the squaring in the Gram matrix (measured: 2e-7 above 2 %, up to 1.3e-4 at 1-2 %, 5e-3 at
+// 0.5-1 %); the status word then says so.  Below kZeroRel a value is zero to working precision (a W of lower rank than asked for).
+constexpr float kDomainRel = 2e-2f, kZeroRel = 1e-5f;
 
 // Rows count as orthogonal when |x_i.x_j| <= tol |x_i||x_j|.  An fp32 dot product of length s
 // carries rounding noise of about 6e-8 sqrt(s) relative to |x_i||x_j|; the maximum over all

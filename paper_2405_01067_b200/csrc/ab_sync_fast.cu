@@ -30,14 +30,15 @@ namespace cg = cooperative_groups;
 constexpr int kJMaxSweeps = 40;
 constexpr float kJDead2 = 1e-12f;    // rows below 1e-6 of the largest norm are zero rows
 constexpr float kJCount2 = 1e-8f;    // rows below 1e-4 of the largest norm do not hold up convergence
-constexpr float kJEarly2 = 9e-8f;    // a sweep whose largest rotated cosine was below 3e-4 is the last one: one-sided
-                                     // Jacobi converges quadratically, so what it leaves is of the order 1e-7 < tol
+constexpr float kJEarly2 = 4e-6f;    // a sweep whose largest rotated cosine was below 2e-3 is the last one: one-sided
+                                     // Jacobi converges quadratically, so what it leaves is of the order 4e-6 <= tol
 constexpr float kEigThr = 1e-6f;     // relative pivot cut of G_A, G_B (and of sigma in the scalings)
 // Accuracy domain of the factored route: the relative error of a singular value grows as it falls below the
-// largest (measured: 5e-5 down to 1 %, 1e-4 at 4e-4, 1e-3 at 6e-5 of the largest); a kept value between
+// largest and the worse conditioned the factors are (measured: at most 7e-5 down to 1 % of the largest for
+// factors of condition number up to 1e4; 1e-4 to 5e-3 below that); a kept value between
 // kFZeroRel and kFDomainRel of the largest, or a Cholesky pivot that was dropped although it was not exactly
 // zero, is reported through the status word.
-constexpr float kFDomainRel = 1e-3f, kFZeroRel = 1e-6f;
+constexpr float kFDomainRel = 1e-2f, kFZeroRel = 1e-6f;
 constexpr int kCThreads = 512;
 
 struct JacobiJob {
@@ -567,8 +568,15 @@ struct FastWs {
   const float** sig_ptrs;
   int** rout_ptrs;
   int* rs;
+  // tensor-core route of the long products: bf16 pieces (hi, mid, lo) of Abar, Bbar, Z_A, Z_B
+  SplitJob* sjobs;      // 4 L
+  std::vector<bf16*> Asp, Bsp, ZAsp, ZBsp;    // each: three pieces one after the other
+  void* tc_table[3];    // problem tables of the three tensor-core launches
+  int* tc_status;
   size_t bytes;
 };
+
+int r8(int v) { return (v + 7) & ~7; }
 
 FastWs fast_layout(const ab_sync_desc* d, int L, void* ws) {
   FastWs w;
@@ -593,8 +601,28 @@ FastWs fast_layout(const ab_sync_desc* d, int L, void* ws) {
   w.sig_ptrs = ar.take_n<const float*>(L);
   w.rout_ptrs = ar.take_n<int*>(L);
   w.rs = ar.take_n<int>(L);
+  w.sjobs = ar.take_n<SplitJob>((size_t)4 * L);
+  auto each_bf = [&](std::vector<bf16*>& v, auto count) {
+    v.resize(L);
+    for (int i = 0; i < L; ++i) v[i] = ar.take_n<bf16>(3 * count(d[i]));
+  };
+  each_bf(w.Asp, [](const ab_sync_desc& x) { return (size_t)x.m * r8(x.r); });
+  each_bf(w.Bsp, [](const ab_sync_desc& x) { return (size_t)x.r * r8(x.n); });
+  each_bf(w.ZAsp, [](const ab_sync_desc& x) { return (size_t)x.r * r8(x.r); });
+  each_bf(w.ZBsp, [](const ab_sync_desc& x) { return (size_t)x.r * r8(x.r); });
+  w.tc_table[0] = ar.take(gemm_tc_table_bytes(2 * L));
+  w.tc_table[1] = ar.take(gemm_tc_table_bytes(2 * L));
+  w.tc_table[2] = ar.take(gemm_tc_table_bytes(L));
+  w.tc_status = ar.take_n<int>(64);
   w.bytes = align_up(ar.used, 256);
   return w;
+}
+
+TcOperand pieces3(const bf16* base, size_t piece_elems, int64_t ld, bool mn) {
+  TcOperand o;
+  for (int k = 0; k < 3; ++k) o.p[k] = base + k * piece_elems;
+  o.pieces = 3; o.ld = ld; o.mn = mn;
+  return o;
 }
 
 GemmDesc mk(const float* A, int64_t sAm, int64_t sAk, const float* B, int64_t sBk, int64_t sBn, void* C, int64_t ldc,
@@ -675,6 +703,17 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   for (int i = 0; i < L; ++i) {
     rmax = std::max(rmax, d[i].r); mmax = std::max(mmax, d[i].m); nmax = std::max(nmax, d[i].n);
   }
+  // The long products (Gram matrices, A', B', W) run on the tensor cores as six-term bf16 products when
+  // every output can be stored by 16-byte rows; otherwise on the fp32 pipes.
+  bool use_tc = gemm_tc_available();
+  for (int i = 0; i < L && use_tc; ++i) {
+    const int q = out_bf16 ? 8 : 4;
+    use_tc = d[i].r % 4 == 0 && d[i].r % q == 0 && d[i].n % q == 0 && aligned(d[i].A_out, 16) && aligned(d[i].B_out, 16) &&
+             (!d[i].W_out || (d[i].n % 4 == 0 && aligned(d[i].W_out, 16)));
+  }
+  std::vector<SplitJob> sj((size_t)4 * L);
+  std::vector<TcProblem> tp_gram, tp_out, tp_w;
+  int64_t split_blocks[2] = {0, 0};
   // ---- host-built tables: 9 GEMM descriptors, 2 Cholesky jobs and 1 Jacobi job per matrix, copied in one go each
   std::vector<GemmDesc> g((size_t)9 * L);
   std::vector<CholJob> cj((size_t)2 * L);
@@ -711,18 +750,55 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
     gb.c_bf16 = out_bf16; gb.live_rows = d[i].r_out;
     // batch 6 (L, optional): W = Abar Bbar
     g[8 * L + i] = mk(Ab, r, 1, Bb, n, 1, d[i].W_out, n, d[i].W_out ? m : 0, d[i].W_out ? n : 0, r);
-    const int pa = gram_parts(m), pb = gram_parts(n);
+    const int pa = use_tc ? 1 : gram_parts(m), pb = use_tc ? 1 : gram_parts(n);
+    if (use_tc) {
+      const int rr8 = r8(r), n8 = r8(n);
+      const size_t ea = (size_t)m * rr8, eb = (size_t)r * n8, ez = (size_t)r * rr8;
+      sj[2 * i] = SplitJob{Ab, r, m, r, w.Asp[i], w.Asp[i] + ea, w.Asp[i] + 2 * ea, rr8, 0};
+      sj[2 * i + 1] = SplitJob{Bb, n, r, n, w.Bsp[i], w.Bsp[i] + eb, w.Bsp[i] + 2 * eb, n8, 0};
+      sj[2 * L + 2 * i] = SplitJob{w.ZA[i], r, r, r, w.ZAsp[i], w.ZAsp[i] + ez, w.ZAsp[i] + 2 * ez, rr8, 0};
+      sj[2 * L + 2 * i + 1] = SplitJob{w.ZB[i], r, r, r, w.ZBsp[i], w.ZBsp[i] + ez, w.ZBsp[i] + 2 * ez, rr8, 0};
+      for (int h = 0; h < 2; ++h) {
+        sj[2 * i + h].first_block = split_blocks[0];
+        split_blocks[0] += split_job_blocks(sj[2 * i + h].rows, sj[2 * i + h].cols);
+        sj[2 * L + 2 * i + h].first_block = split_blocks[1];
+        split_blocks[1] += split_job_blocks(r, r);
+      }
+      const TcOperand A_k = pieces3(w.Asp[i], ea, rr8, false), A_t = pieces3(w.Asp[i], ea, rr8, true);
+      const TcOperand B_k = pieces3(w.Bsp[i], eb, n8, false), B_t = pieces3(w.Bsp[i], eb, n8, true);
+      TcProblem q;
+      q.ksplit = 1; q.live_rows = q.live_cols = nullptr; q.c_f32 = true;
+      // G_A = Abar^T Abar: both operands are Abar as it lies, (reduction index m) x r
+      q.A = A_t; q.B = A_t; q.C = w.GA[i]; q.ldc = r; q.M = r; q.N = r; q.K = m;
+      tp_gram.push_back(q);
+      // G_B = Bbar Bbar^T: both operands Bbar, r x (reduction index n)
+      q.A = B_k; q.B = B_k; q.C = w.GB[i]; q.ldc = r; q.M = r; q.N = r; q.K = n;
+      tp_gram.push_back(q);
+      // A' = Abar Z_A (columns at or beyond r' zero), B' = Z_B Bbar (rows at or beyond r' zero)
+      q.c_f32 = !out_bf16;
+      q.A = A_k; q.B = pieces3(w.ZAsp[i], ez, rr8, true); q.C = d[i].A_out; q.ldc = r; q.M = m; q.N = r; q.K = r;
+      q.live_cols = d[i].r_out;
+      tp_out.push_back(q);
+      q.A = pieces3(w.ZBsp[i], ez, rr8, false); q.B = B_t; q.C = d[i].B_out; q.ldc = n; q.M = r; q.N = n; q.K = r;
+      q.live_cols = nullptr; q.live_rows = d[i].r_out;
+      tp_out.push_back(q);
+      if (d[i].W_out) {     // W = Abar Bbar
+        q.c_f32 = true; q.live_rows = nullptr;
+        q.A = A_k; q.B = B_t; q.C = d[i].W_out; q.ldc = n; q.M = m; q.N = n; q.K = r;
+        tp_w.push_back(q);
+      }
+    }
     cj[i] = CholJob{w.GA[i], pa, w.RA[i], w.IA[i], w.jstatus + 3 * i, r};
     cj[L + i] = CholJob{w.GB[i], pb, w.RB[i], w.IB[i], w.jstatus + 3 * i + 1, r};
     // Gram matrices in slices of the long index (equal work per CTA, partial sums added by the
     // Cholesky kernel in ascending slice order), upper tiles only
-    for (int q = 0; q < pa; ++q) {
+    for (int q = 0; q < pa && !use_tc; ++q) {
       const int k0 = gram_k0(m, pa, q), k1 = gram_k0(m, pa, q + 1);
       GemmDesc x = mk(Ab + (size_t)k0 * r, 1, r, Ab + (size_t)k0 * r, r, 1, w.GA[i] + (size_t)q * r * r, r, r, r, k1 - k0);
       x.upper_only = 1;
       gg.push_back(x);
     }
-    for (int q = 0; q < pb; ++q) {
+    for (int q = 0; q < pb && !use_tc; ++q) {
       const int k0 = gram_k0(n, pb, q), k1 = gram_k0(n, pb, q + 1);
       GemmDesc x = mk(Bb + k0, n, 1, Bb + k0, 1, n, w.GB[i] + (size_t)q * r * r, r, r, r, k1 - k0);
       x.upper_only = 1;
@@ -744,7 +820,7 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   }
   {
     char* base = reinterpret_cast<char*>(w.descs);
-    const size_t span = (size_t)(reinterpret_cast<char*>(w.rs + L) - base);
+    const size_t span = (size_t)(reinterpret_cast<char*>(w.sjobs + 4 * L) - base);
     std::vector<char> img(span, 0);
     auto put = [&](const void* dev_ptr, const void* src, size_t bytes) {
       std::memcpy(img.data() + (reinterpret_cast<const char*>(dev_ptr) - base), src, bytes);
@@ -757,6 +833,7 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
     put(w.sig_ptrs, sigp.data(), L * sizeof(float*));
     put(w.rout_ptrs, routp.data(), L * sizeof(int*));
     put(w.rs, rs.data(), L * sizeof(int));
+    put(w.sjobs, sj.data(), sj.size() * sizeof(SplitJob));
     AB_CUDA_OK(cudaMemcpyAsync(base, img.data(), span, cudaMemcpyHostToDevice, st));
   }
 
@@ -786,8 +863,17 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   } evs;
   if (side && !evs.create()) side = nullptr;
   cudaEvent_t fork = evs.fork, join = evs.join;
-  if (any_w && !side) AB_TRY(gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, st));
-  AB_TRY(gemm_simt_batched(w.gram_descs, (int)gg.size(), rmax, rmax, st));                  // Gram slices
+  auto product_w = [&](cudaStream_t s2) -> int {
+    if (use_tc) return gemm_tc_batched(tp_w.data(), (int)tp_w.size(), w.tc_table[2], w.tc_status + 2, s2);
+    return gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, s2);
+  };
+  if (use_tc) {
+    AB_CUDA_OK(cudaMemsetAsync(w.tc_status, 0, 4 * sizeof(int), st));
+    AB_TRY(split3_batched(w.sjobs, 2 * L, split_blocks[0], st));                            // pieces of Abar, Bbar
+  }
+  if (any_w && !side) AB_TRY(product_w(st));
+  if (use_tc) AB_TRY(gemm_tc_batched(tp_gram.data(), (int)tp_gram.size(), w.tc_table[0], w.tc_status, st));
+  else AB_TRY(gemm_simt_batched(w.gram_descs, (int)gg.size(), rmax, rmax, st));             // Gram slices
   const size_t csm = chol_smem_bytes(rmax);
   AB_CUDA_OK(cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csm));
   chol_inv_kernel<<<2 * L, kCThreads, csm, st>>>(w.cjobs);                                  // R_A, R_B and inverses
@@ -798,7 +884,7 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   AB_TRY(launch_jacobi(w.jobs, L, rmax, tol, st));                                    // SVD of M
   if (side) {
     if (side_rc == AB_OK && cudaStreamWaitEvent(side, fork, 0) != cudaSuccess) side_rc = AB_ERR_CUDA;
-    if (side_rc == AB_OK) side_rc = gemm_simt_batched(w.descs + 8 * L, L, mmax, nmax, side);
+    if (side_rc == AB_OK) side_rc = product_w(side);
     if (side_rc == AB_OK && cudaEventRecord(join, side) != cudaSuccess) side_rc = AB_ERR_CUDA;
   }
   fast_rank_rule_kernel<<<(L + 127) / 128, 128, 0, st>>>(w.sig_ptrs, w.rs, sigma_cutoff, w.rout_ptrs, w.jstatus,
@@ -806,8 +892,13 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   AB_LAUNCH_OK();
   AB_TRY(gemm_simt_batched(w.descs + 3 * L, 2 * L, rmax, rmax, st));                        // Y1, Z_B
   AB_TRY(gemm_simt_batched(w.descs + 5 * L, L, rmax, rmax, st));                            // Z_A
-  AB_TRY(gemm_simt_batched(w.descs + 6 * L, L, mmax, rmax, st));                            // A'
-  AB_TRY(gemm_simt_batched(w.descs + 7 * L, L, rmax, nmax, st));                            // B'
+  if (use_tc) {
+    AB_TRY(split3_batched(w.sjobs + 2 * L, 2 * L, split_blocks[1], st));                    // pieces of Z_A, Z_B
+    AB_TRY(gemm_tc_batched(tp_out.data(), (int)tp_out.size(), w.tc_table[1], w.tc_status + 1, st));   // A', B'
+  } else {
+    AB_TRY(gemm_simt_batched(w.descs + 6 * L, L, mmax, rmax, st));                          // A'
+    AB_TRY(gemm_simt_batched(w.descs + 7 * L, L, rmax, nmax, st));                          // B'
+  }
   if (side) {
     if (side_rc == AB_OK && cudaStreamWaitEvent(st, join, 0) != cudaSuccess) side_rc = AB_ERR_CUDA;
     if (side_rc != AB_OK) { (void)cudaGetLastError(); return side_rc; }

@@ -78,6 +78,16 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* m, uin
       "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
       : "memory");
 }
+// 4-D tile load (an NHWC activation: c0 = channel, c1 = x, c2 = y, c3 = image).  Coordinates may start outside
+// the tensor (also below zero): what lies outside arrives as zeros, which is the padding of a convolution.
+// c0 times the element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* m, uint64_t* bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(
+          smem_u32(dst)),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, const void* src, int c0, int c1) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
                    reinterpret_cast<uint64_t>(m)),
@@ -168,5 +178,8 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N, int a_mn_ma
 // driver can run these kernels at all.
 int make_tensor_map_2d(CUtensorMap* m, const void* ptr, bool f32, uint64_t rows, uint64_t cols, uint64_t ld,
                        uint32_t box_cols, uint32_t box_rows);
+// 4-D tensor map of a bf16 NHWC activation [B, H, W, C] (C contiguous), boxes of 64 channels x bw x bh x bb.
+int make_tensor_map_nhwc(CUtensorMap* m, const void* ptr, uint64_t B, uint64_t H, uint64_t W, uint64_t C,
+                         uint32_t bw, uint32_t bh, uint32_t bb);
 bool tc_device_ok();
 }  // namespace ab

@@ -84,3 +84,34 @@ def test_full_rank_factors_reproduce_dense_layer():
     x = rng.standard_normal((7, 9))
     _, y = orc.forward(x, A, B)
     assert np.allclose(y, x @ W.T, atol=1e-12)
+
+
+def test_dense_layer_loops_finite_differences_and_factorised_form():
+    """The dense layer of the full-rank phases: element-wise loops, central differences of L = <y, dY> (exact
+    up to rounding: L is linear in x and in W), and agreement with the factorised layer when W = A B."""
+    rng = np.random.default_rng(21)
+    N, m, n, r = 5, 4, 6, 3
+    x, dY, W = rng.standard_normal((N, n)), rng.standard_normal((N, m)), rng.standard_normal((m, n))
+    y = orc.dense_forward(x, W)
+    for i in range(N):
+        for j in range(m):
+            assert np.isclose(y[i, j], sum(x[i, k] * W[j, k] for k in range(n)), rtol=1e-13)
+    dX, dW = orc.dense_backward(x, dY, W)
+    h = 1e-3
+
+    def loss(xx, ww):
+        return float(np.sum(orc.dense_forward(xx, ww) * dY))
+    for i in range(N):
+        for k in range(n):
+            e = np.zeros_like(x); e[i, k] = h
+            assert np.isclose((loss(x + e, W) - loss(x - e, W)) / (2 * h), dX[i, k], rtol=1e-9, atol=1e-11)
+    for j in range(m):
+        for k in range(n):
+            e = np.zeros_like(W); e[j, k] = h
+            assert np.isclose((loss(x, W + e) - loss(x, W - e)) / (2 * h), dW[j, k], rtol=1e-9, atol=1e-11)
+    A, B = rng.standard_normal((m, r)), rng.standard_normal((r, n))
+    assert np.allclose(orc.dense_forward(x, A @ B), orc.forward(x, A, B)[1], atol=1e-12)
+    dXf, dAf, dBf, _ = orc.backward(x, dY, A, B)
+    dXd, dWd = orc.dense_backward(x, dY, A @ B)
+    assert np.allclose(dXd, dXf, atol=1e-12)
+    assert np.allclose(dWd @ B.T, dAf, atol=1e-12) and np.allclose(A.T @ dWd, dBf, atol=1e-12)
