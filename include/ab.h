@@ -148,6 +148,30 @@ int ab_layer_backward(const void* x, const void* dY, const void* A, const void* 
                       void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Factorised 3 x 3 convolution (stride 1, zero padding 1) on NHWC activations, without materialised im2col
+ * rows.  The paper flattens the trailing dimensions of a convolution weight into a matrix before Eq. 3
+ * (Section "Methodology", after Eq. 3); here the flattened weight is W [m, 9 C] = A B with column
+ * (ky * 3 + kx) * C + c for tap (ky, kx) and input channel c, and
+ *   forward : y [B,H,W,m] = (rows(x) B^T) A^T, where rows(x) are the 9 C-wide im2col rows of x [B,H,W,C]; they
+ *             are never formed: every tap's shifted view of x is loaded straight from the activation (what
+ *             falls outside an image is zero), so x is read from device memory once instead of nine times.
+ *             T_save: NULL, or [B H W, r] that receives T for the backward call.
+ *   backward: dT = dY A;  dX [B,H,W,C] = the col2im sum of dT B over the nine taps (folded into the
+ *             reduction: no 9 C-wide gradient rows are formed);  dA [m,r] = dY^T T;  dB [r,9C] = dT^T rows(x).
+ *             Any of dX, dA, dB may be NULL; T_saved NULL recomputes T.  dA, dB fp32, fixed summation order.
+ *   Supported: dt = AB_BF16, C, m, r multiples of 8, 8 <= r <= 256, W <= 64, H <= 256; anything else returns
+ *   AB_ERR_UNSUPPORTED (materialise the rows and call ab_layer_forward / ab_layer_backward instead).
+ *   Workspace: ab_conv3x3_workspace_bytes; its first int is the device status word as for ab_layer_forward.
+ */
+int ab_conv3x3_forward(const void* x, const void* A, const void* B, void* y, void* T_save,
+                       int batch, int H, int W, int C, int m, int r, int ldA, int ldB, int dt,
+                       void* ws, size_t ws_bytes, void* cuda_stream);
+int ab_conv3x3_backward(const void* x, const void* dY, const void* A, const void* B, const void* T_saved,
+                        void* dX, float* dA, float* dB, int batch, int H, int W, int C, int m, int r,
+                        int ldA, int ldB, int dt, void* ws, size_t ws_bytes, void* cuda_stream);
+size_t ab_conv3x3_workspace_bytes(int batch, int H, int W, int C, int m, int r);
+
+/*
  * Dense layer of the full-rank phases of a training cycle (Algorithm 1: the warm-up steps before the
  * first decomposition and the full-rank rebound steps after W <- A B; Section "Methodology", full-rank
  * rebound): the same linear map with W held dense.

@@ -8,6 +8,8 @@ What each function follows:
 
 * ``forward`` / ``backward``   the layer W = A B of Eq. 3 used as a linear map
   y = x W^T, and the chain rule through the rank-r intermediate.
+* ``im2col_3x3`` / ``col2im_3x3`` / ``conv3x3_*``  the flattening of a convolution weight's
+  trailing dimensions (Methodology, after Eq. 3) applied to NHWC activations.
 * ``dense_forward`` / ``dense_backward``  the same layer with W dense (Algorithm 1's
   full-rank steps: warm-up and rebound).
 * ``group_average*``           Algorithm 1, the two allReduce(./worldSize) lines.
@@ -56,6 +58,46 @@ def backward(x, dY, A, B):
     dA = dY.T @ T
     dB = dT.T @ x
     return dX, dA, dB, dT
+
+
+def im2col_3x3(x):
+    """Rows of a 3 x 3 convolution with stride 1 and zero padding 1 over an NHWC activation x [B, H, W, C]:
+    row (b, oy, ox) holds x[b, oy + ky - 1, ox + kx - 1, c] at column (ky * 3 + kx) * C + c (zeros outside
+    the image).  This is the flattening of the trailing weight dimensions (Methodology, after Eq. 3) seen
+    from the activation side: a convolution weight [m, ky, kx, C] flattened to m x 9C multiplies these rows."""
+    x = _f64(x)
+    B, H, W, C = x.shape
+    xp = np.zeros((B, H + 2, W + 2, C))
+    xp[:, 1:H + 1, 1:W + 1] = x
+    rows = np.empty((B, H, W, 9, C))
+    for ky in range(3):
+        for kx in range(3):
+            rows[:, :, :, ky * 3 + kx] = xp[:, ky:ky + H, kx:kx + W]
+    return rows.reshape(B * H * W, 9 * C)
+
+
+def col2im_3x3(rows, B, H, W, C):
+    """The transpose of ``im2col_3x3``: every entry of a row is added back to the pixel it was taken from
+    (entries taken from the padding are dropped).  Turns the gradient of the rows into that of x."""
+    r = _f64(rows).reshape(B, H, W, 9, C)
+    xp = np.zeros((B, H + 2, W + 2, C))
+    for ky in range(3):
+        for kx in range(3):
+            xp[:, ky:ky + H, kx:kx + W] += r[:, :, :, ky * 3 + kx]
+    return xp[:, 1:H + 1, 1:W + 1].copy()
+
+
+def conv3x3_forward(x, A, B):
+    """Factorised 3 x 3 convolution: the layer of Eq. 3 applied to the im2col rows.  Returns (T, y) as
+    [pixels, r] and [pixels, m]."""
+    return forward(im2col_3x3(x), A, B)
+
+
+def conv3x3_backward(x, dY, A, B):
+    """Chain rule of the factorised convolution.  Returns (dX [B,H,W,C], dA, dB, dT)."""
+    Bn, H, W, C = np.shape(x)
+    dXr, dA, dB, dT = backward(im2col_3x3(x), dY, A, B)
+    return col2im_3x3(dXr, Bn, H, W, C), dA, dB, dT
 
 
 def dense_forward(x, W):

@@ -26,7 +26,8 @@ EXPORTS = ["ab_status_string", "ab_version", "ab_launch_count", "ab_workspace_by
            "ab_group_average", "ab_recombine", "ab_svd_split", "ab_group_sync", "ab_sync_workspace_bytes",
            "ab_layer_forward_static", "ab_static_scratch_elems", "ab_adamw_step", "ab_lr_rebound_factor", "ab_selftest_bounded_wait",
            "ab_selftest_chain_stall", "ab_selftest_chain_stall_workspace_bytes",
-           "ab_dense_forward", "ab_dense_backward"]
+           "ab_dense_forward", "ab_dense_backward", "ab_conv3x3_forward", "ab_conv3x3_backward",
+           "ab_conv3x3_workspace_bytes"]
 
 
 class AbError(RuntimeError):
@@ -91,6 +92,12 @@ def lib() -> ctypes.CDLL:
     L.ab_dense_forward.argtypes = [c_void_p] * 3 + [c_int64, c_int, c_int, c_int, c_void_p, c_size_t, c_void_p]
     L.ab_dense_backward.restype = c_int
     L.ab_dense_backward.argtypes = [c_void_p] * 5 + [c_int64, c_int, c_int, c_int, c_void_p, c_size_t, c_void_p]
+    L.ab_conv3x3_forward.restype = c_int
+    L.ab_conv3x3_forward.argtypes = [c_void_p] * 5 + [c_int] * 9 + [c_void_p, c_size_t, c_void_p]
+    L.ab_conv3x3_backward.restype = c_int
+    L.ab_conv3x3_backward.argtypes = [c_void_p] * 8 + [c_int] * 9 + [c_void_p, c_size_t, c_void_p]
+    L.ab_conv3x3_workspace_bytes.restype = c_size_t
+    L.ab_conv3x3_workspace_bytes.argtypes = [c_int] * 6
     _lib = L
     return L
 
@@ -210,6 +217,48 @@ def ab_layer_backward(x, dY, A, B, T_saved=None, want=("dX", "dA", "dB"), dX=Non
     st = lib().ab_layer_backward(_ptr(x), _ptr(dY), _ptr(A), _ptr(B), _ptr(T_saved), _ptr(dX), _ptr(dA), _ptr(dB),
                                  N, m, n, r, A.stride(0), B.stride(0), dt, _ptr(ws), ws.numel(), _stream(stream))
     _check(st, "ab_layer_backward")
+    return dX, dA, dB
+
+
+def ab_conv3x3_workspace_bytes(batch, H, W, C, m, r) -> int:
+    return int(lib().ab_conv3x3_workspace_bytes(batch, H, W, C, m, r))
+
+
+def ab_conv3x3_forward(x, A, B, y=None, T_save=None, ws=None, stream=None, save_T=False):
+    """Factorised 3 x 3 convolution on an NHWC activation x [batch, H, W, C].  Returns (y [batch,H,W,m], T or None)."""
+    _dev_ok(x, A, B, y, T_save)
+    batch, H, W, C = x.shape
+    m, r = A.shape
+    if y is None:
+        y = torch.empty((batch, H, W, m), dtype=x.dtype, device=x.device)
+    if save_T and T_save is None:
+        T_save = torch.empty((batch * H * W, r), dtype=x.dtype, device=x.device)
+    if ws is None:
+        ws = workspace(ab_conv3x3_workspace_bytes(batch, H, W, C, m, r), x.device)
+    st = lib().ab_conv3x3_forward(_ptr(x), _ptr(A), _ptr(B), _ptr(y), _ptr(T_save), batch, H, W, C, m, r,
+                                  A.stride(0), B.stride(0), _dt(x), _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "ab_conv3x3_forward")
+    return y, T_save
+
+
+def ab_conv3x3_backward(x, dY, A, B, T_saved=None, want=("dX", "dA", "dB"), dX=None, dA=None, dB=None, ws=None,
+                        stream=None):
+    """dX [batch,H,W,C], dA [m,r], dB [r,9C] of the factorised convolution; dY is [batch,H,W,m]."""
+    _dev_ok(x, dY, A, B, T_saved, dX, dA, dB)
+    batch, H, W, C = x.shape
+    m, r = A.shape
+    if "dX" in want and dX is None:
+        dX = torch.empty_like(x)
+    if "dA" in want and dA is None:
+        dA = torch.empty((m, r), dtype=torch.float32, device=x.device)
+    if "dB" in want and dB is None:
+        dB = torch.empty((r, 9 * C), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = workspace(ab_conv3x3_workspace_bytes(batch, H, W, C, m, r), x.device)
+    st = lib().ab_conv3x3_backward(_ptr(x), _ptr(dY), _ptr(A), _ptr(B), _ptr(T_saved), _ptr(dX), _ptr(dA), _ptr(dB),
+                                   batch, H, W, C, m, r, A.stride(0), B.stride(0), _dt(x), _ptr(ws), ws.numel(),
+                                   _stream(stream))
+    _check(st, "ab_conv3x3_backward")
     return dX, dA, dB
 
 

@@ -216,6 +216,49 @@ int ab_layer_backward(const void* x, const void* dY, const void* A, const void* 
   return general_backward(x, dY, A, B, T_saved, dX, dA, dB, N, m, n, r, ldA, ldB, dt, ws, ws_bytes, st);
 }
 
+size_t ab_conv3x3_workspace_bytes(int batch, int H, int W, int C, int m, int r) {
+  if (batch <= 0 || H <= 0 || W <= 0 || C <= 0 || m <= 0 || r <= 0) return 0;
+  return conv_tc_ws(batch, H, W, C, m, r) + 256;
+}
+
+static int check_conv_args(const void* x, const void* A, const void* B, int batch, int H, int W, int C, int m, int r,
+                           int ldA, int ldB, int dt) {
+  if (!dtype_ok(dt)) return AB_ERR_INVALID_ARG;
+  if (batch < 0 || H <= 0 || W <= 0 || C <= 0 || m <= 0 || r <= 0) return AB_ERR_INVALID_ARG;
+  if (r > m || r > 9 * C || ldA < r || ldB < 9 * C) return AB_ERR_INVALID_ARG;
+  if (!A || !B || (batch > 0 && !x)) return AB_ERR_INVALID_ARG;
+  return AB_OK;
+}
+
+int ab_conv3x3_forward(const void* x, const void* A, const void* B, void* y, void* T_save,
+                       int batch, int H, int W, int C, int m, int r, int ldA, int ldB, int dt,
+                       void* ws, size_t ws_bytes, void* cuda_stream) {
+  AB_TRY(check_conv_args(x, A, B, batch, H, W, C, m, r, ldA, ldB, dt));
+  if (batch > 0 && !y) return AB_ERR_INVALID_ARG;
+  if (!have_device()) return AB_ERR_CUDA;
+  if (batch == 0) return AB_OK;
+  if (!ws || !aligned(ws, 256)) return AB_ERR_WORKSPACE;
+  if (!conv_tc_supported(batch, H, W, C, m, r, ldA, ldB, dt, x, A, B)) return AB_ERR_UNSUPPORTED;
+  return conv_tc_forward(x, A, B, y, T_save, batch, H, W, C, m, r, ldA, ldB, ws, ws_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ab_conv3x3_backward(const void* x, const void* dY, const void* A, const void* B, const void* T_saved,
+                        void* dX, float* dA, float* dB, int batch, int H, int W, int C, int m, int r,
+                        int ldA, int ldB, int dt, void* ws, size_t ws_bytes, void* cuda_stream) {
+  AB_TRY(check_conv_args(x, A, B, batch, H, W, C, m, r, ldA, ldB, dt));
+  if (batch > 0 && !dY) return AB_ERR_INVALID_ARG;
+  if (!have_device()) return AB_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (batch == 0) {
+    if (dA) AB_CUDA_OK(cudaMemsetAsync(dA, 0, (size_t)m * r * sizeof(float), st));
+    if (dB) AB_CUDA_OK(cudaMemsetAsync(dB, 0, (size_t)r * 9 * C * sizeof(float), st));
+    return AB_OK;
+  }
+  if (!ws || !aligned(ws, 256)) return AB_ERR_WORKSPACE;
+  if (!conv_tc_supported(batch, H, W, C, m, r, ldA, ldB, dt, x, A, B) || !aligned(dY, 16)) return AB_ERR_UNSUPPORTED;
+  return conv_tc_backward(x, dY, A, B, T_saved, dX, dA, dB, batch, H, W, C, m, r, ldA, ldB, ws, ws_bytes, st);
+}
+
 int ab_adamw_step(float* param, const float* grad, float* m, float* v, void* param_bf16, int64_t count,
                   float lr, float beta1, float beta2, float eps, float weight_decay, int step,
                   void* cuda_stream) {

@@ -20,7 +20,7 @@ def L():
 def test_every_declared_symbol_is_exported(L):
     hdr = open(os.path.join(ROOT, "include", "ab.h")).read()
     hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
-    names = set(re.findall(r"\b(ab_[a-z_]+)\s*\(", hdr))
+    names = set(re.findall(r"\b(ab_[a-z0-9_]+)\s*\(", hdr))
     assert {"ab_layer_forward", "ab_layer_backward", "ab_group_average", "ab_recombine", "ab_svd_split"} <= names
     for nm in names:
         assert hasattr(L, nm), nm

@@ -115,3 +115,35 @@ def test_dense_layer_loops_finite_differences_and_factorised_form():
     dXd, dWd = orc.dense_backward(x, dY, A @ B)
     assert np.allclose(dXd, dXf, atol=1e-12)
     assert np.allclose(dWd @ B.T, dAf, atol=1e-12) and np.allclose(A.T @ dWd, dBf, atol=1e-12)
+
+
+def test_conv3x3_rows_against_direct_convolution_and_adjoint():
+    """im2col rows times a flattened weight equal the convolution written as loops; col2im is the exact
+    transpose of im2col (<im2col(x), R> = <x, col2im(R)>); the factorised convolution's dX matches central
+    differences."""
+    rng = np.random.default_rng(31)
+    B, H, W, C, m, r = 2, 3, 4, 3, 4, 2
+    x = rng.standard_normal((B, H, W, C))
+    Wt = rng.standard_normal((m, 3, 3, C))
+    y = orc.im2col_3x3(x) @ Wt.reshape(m, 9 * C).T
+    for b in range(B):
+        for oy in range(H):
+            for ox in range(W):
+                for o in range(m):
+                    acc = 0.0
+                    for ky in range(3):
+                        for kx in range(3):
+                            iy, ix = oy + ky - 1, ox + kx - 1
+                            if 0 <= iy < H and 0 <= ix < W:
+                                acc += float(np.dot(x[b, iy, ix], Wt[o, ky, kx]))
+                    assert np.isclose(y[(b * H + oy) * W + ox, o], acc, rtol=1e-12, atol=1e-13)
+    R = rng.standard_normal((B * H * W, 9 * C))
+    assert np.isclose(np.sum(orc.im2col_3x3(x) * R), np.sum(x * orc.col2im_3x3(R, B, H, W, C)), rtol=1e-12)
+    A, Bf = rng.standard_normal((m, r)), rng.standard_normal((r, 9 * C))
+    dY = rng.standard_normal((B * H * W, m))
+    dX, dA, dB, _ = orc.conv3x3_backward(x, dY, A, Bf)
+    h = 1e-3
+    for idx in [(0, 0, 0, 0), (1, 2, 3, 2), (0, 1, 2, 1), (1, 0, 3, 0)]:
+        e = np.zeros_like(x); e[idx] = h
+        num = (np.sum(orc.conv3x3_forward(x + e, A, Bf)[1] * dY) - np.sum(orc.conv3x3_forward(x - e, A, Bf)[1] * dY)) / (2 * h)
+        assert np.isclose(num, dX[idx], rtol=1e-8, atol=1e-10)
