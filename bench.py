@@ -309,6 +309,53 @@ def other_workloads(ab, torch, iters=10):
     return out
 
 
+def conv_workloads(ab, torch, iters=10):
+    """The two convolution shapes through the implicit-im2col entry points (NHWC activation in, no 9x inflated
+    rows in memory): forward + backward (dX with col2im folded in, dA, dB).  Bytes are counted against the
+    un-inflated activation: x in forward and backward, dX out, y out, dY in (bf16)."""
+    pk = measured_peaks()
+    out = {}
+    bf = torch.bfloat16
+    for name, (B, H, W, C, m, r) in (("resnet50_layer3_conv3x3_r128", (128, 14, 14, 256, 256, 128)),
+                                     ("vgg16_512_4x4_r8", (1024, 4, 4, 512, 512, 8)),
+                                     ("vgg16_512_4x4_r16", (1024, 4, 4, 512, 512, 16)),
+                                     ("vgg16_512_4x4_r32", (1024, 4, 4, 512, 512, 32)),
+                                     ("vgg16_512_4x4_r64", (1024, 4, 4, 512, 512, 64))):
+        g = torch.Generator(device="cuda").manual_seed(5)
+        x = torch.randn((B, H, W, C), device="cuda", generator=g).abs().to(bf)
+        dY = torch.randn((B, H, W, m), device="cuda", generator=g).to(bf)
+        A = (torch.randn((m, r), device="cuda", generator=g) * 0.05).to(bf)
+        Bf = (torch.randn((r, 9 * C), device="cuda", generator=g) * 0.05).to(bf)
+        y = torch.empty((B, H, W, m), dtype=bf, device="cuda")
+        T = torch.empty((B * H * W, r), dtype=bf, device="cuda")
+        dX = torch.empty_like(x)
+        dA = torch.empty((m, r), device="cuda")
+        dB = torch.empty((r, 9 * C), device="cuda")
+        ws = ab.workspace(ab.ab_conv3x3_workspace_bytes(B, H, W, C, m, r), "cuda")
+
+        def fn():
+            ab.ab_conv3x3_forward(x, A, Bf, y=y, T_save=T, ws=ws)
+            ab.ab_conv3x3_backward(x, dY, A, Bf, T_saved=T, dX=dX, dA=dA, dB=dB, ws=ws)
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        N = B * H * W
+        flop = 6.0 * N * r * (m + 9 * C)
+        nbytes = 2.0 * N * (3 * C + 2 * m)
+        out[name] = dict(batch=B, H=H, W=W, C=C, m=m, r=r, ms=ms, tflops=flop / (ms * 1e-3) / 1e12,
+                         activation_gbs=nbytes / (ms * 1e-3) / 1e9, frac_of_hbm=nbytes / (ms * 1e-3) / 1e9 / pk["hbm"],
+                         bytes_vs_materialised_rows=nbytes / (2.0 * N * (3 * 9 * C + 2 * m)),
+                         device_status=ab.workspace_status(ws))
+    return out
+
+
 def dense_split_times(ab, torch, iters=3):
     """The decomposition Algorithm 1 runs after the full-rank rebound phase: W is dense and no longer of rank
     <= r, so the factored route does not apply.  ab_svd_split (r_max 192, fixed rank) of one matrix of each
@@ -604,6 +651,7 @@ def run_ours(args):
             line["other_workloads"] = other_workloads(ab, torch)
             line["adamw_update_vit_factors"] = optimizer_step(ab, torch)
             line["dense_split_ms"] = dense_split_times(ab, torch)
+            line["implicit_conv"] = conv_workloads(ab, torch)
         if world == 1 and not args.no_cpu_baseline:
             cb = cpu_baseline(inputs, min(N, args.baseline_rows), sync_scale=4)    # about 10 s of host work
             line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}

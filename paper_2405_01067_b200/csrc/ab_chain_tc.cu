@@ -75,6 +75,7 @@ struct ChainParams {
   int f1_mn, f2_mn;        // 1: the factor is held with the reduction index as the slow one (MN-major operand)
   int save_s;              // 1: copy S to global through tmS
   int groups;              // work items in all: 32-row groups, or tiles of a convolution (see ConvGeom)
+  int deal;                // items are dealt to the CTAs in runs of this many
   ConvGeom cv;
   bf16* out_ptr;           // convolution mode: Out and S as plain pointers for the rows of a tile's last, partial
   bf16* s_ptr;             //   group of 32 (row strides P and s_ld)
@@ -217,16 +218,23 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
              const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmS, const ChainParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  // [ second-product ring | S of block 0 | S of block 1 | one staging tile per epilogue warp | barriers ]; the
-  // first product's ring lies over the first three regions, which it has to itself while it runs
+  // [ second-product ring | S of block 0 | S of block 1 | staging tiles of the epilogue warps | barriers ]; the
+  // first product's ring lies over all of the first four regions, which it has to itself while it runs (the
+  // staging tiles are written only after the unit's first product is complete, and a unit ends only when the
+  // stores that read them are done)
   uint8_t* ring = smem;
   uint8_t* S0 = smem + (size_t)p.ns2 * kAtom2Bytes;
   uint8_t* stg = S0 + (size_t)p.max_blocks * p.natoms * kAtomBytes;
   Bars* bars = reinterpret_cast<Bars*>(stg + kEpiWarps * kStgTiles * kGroupBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g_begin = (int)((int64_t)blockIdx.x * p.groups / gridDim.x);
-  const int g_end = (int)((int64_t)(blockIdx.x + 1) * p.groups / gridDim.x);
+  // items are dealt in runs of p.deal (1, or 4 = whole 128-row blocks when every CTA gets at least two blocks:
+  // a block costs the same whether full or not, so whole blocks waste none, and the CTAs with one block fewer
+  // leave their SMs to the kernel that follows)
+  const int nruns = (p.groups + p.deal - 1) / p.deal;
+  const int g_begin = (int)((int64_t)blockIdx.x * nruns / gridDim.x) * p.deal;
+  int g_end = (int)((int64_t)(blockIdx.x + 1) * nruns / gridDim.x) * p.deal;
+  if (g_end > p.groups) g_end = p.groups;
   // All CTAs walk the same factor tiles.  Started together they would all ask L2 for the same few lines at
   // the same moment; each CTA therefore starts its walk at a different slab / chunk and wraps round.
   const int rot1 = blockIdx.x % p.nk1;
@@ -316,31 +324,54 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
+    // One thread feeds the tensor pipe; its own instruction count per MMA is kept small: the descriptors of
+    // slot 0 are built once, a slot is an addition, a K step is an addition (32 bytes along a K-major row,
+    // 2048 bytes -- 16 rows -- down an MN-major tile), and the four K steps are unrolled.  (Measured: a second
+    // issuing thread, one per block of a unit, changes nothing -- 100.7 against 102.2 us for a ViT forward:
+    // the pipe itself takes about 200 cycles per 128 x 256 x 16 MMA here.)
     if (lane == 0) {
       const uint32_t idesc1 = instr_desc_bf16(128, p.r, 0, p.f1_mn);
       const uint32_t idesc2 = instr_desc_bf16(128, kChunk, 0, p.f2_mn);
-      int i1 = 0, i2 = 0, u = 0;
+      const uint32_t s_base = smem_u32(smem);
+      const uint64_t dA1 = smem_desc_sw128(s_base, 16);                          // In tile of block 0, slot 0
+      const uint64_t dF1 = p.f1_mn ? smem_desc_sw128(s_base + p.max_blocks * kAtomBytes, kF1AtomBytes)
+                                   : smem_desc_sw128(s_base + p.max_blocks * kAtomBytes, 16);
+      const uint64_t f1_step = p.f1_mn ? (2048u >> 4) : 2u;
+      const uint64_t slot_step = (uint64_t)(p.slot_bytes >> 4);
+      const uint64_t dS = smem_desc_sw128(smem_u32(S0), 16);                     // S tile 0 of block 0
+      const uint64_t dF2 = p.f2_mn ? smem_desc_sw128(s_base, kF1AtomBytes) : smem_desc_sw128(s_base, 16);
+      const uint64_t f2_step = p.f2_mn ? (2048u >> 4) : 2u;
+      const uint64_t blk_step = (uint64_t)(kAtomBytes >> 4);
+      int i2 = 0, u = 0;
+      int slot1 = 0, ph1 = 0;                  // first-product ring position
       int q0 = 0, q1 = 0;                      // uses of each accumulator so far
       bool ok = true;
       for (int g = g_begin; g < g_end && ok; ++u) {
         const Unit un = make_unit(p, g, g_end);
         const int nt = un.nt;
-        for (int ks = 0; ks < p.nk1; ++ks, ++i1) {
-          const int slot = i1 % p.ns, ph = (i1 / p.ns) & 1;
-          if (!mbar_wait(&bars->full[slot], ph, lim)) { raise_timeout(bars, p.status); ok = false; break; }
+        int kr = rot1;
+        for (int ks = 0; ks < p.nk1; ++ks) {
+          if (!mbar_wait(&bars->full[slot1], ph1, lim)) { raise_timeout(bars, p.status); ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_u32(smem + (size_t)slot * p.slot_bytes);
-          const uint32_t sf = sa + p.max_blocks * kAtomBytes;
-          const uint64_t da0 = smem_desc_sw128(sa, 16), da1 = smem_desc_sw128(sa + kAtomBytes, 16);
-          const int kr = (ks + rot1) % p.nk1;
-          int ksteps = p.cv.on ? (p.cv.in_ch - (kr % p.cv.cslabs) * 64 + 15) >> 4 : (p.K1 - kr * 64 + 15) >> 4;
-          if (ksteps > 4) ksteps = 4;
-          for (int kk = 0; kk < ksteps; ++kk) {
-            const uint64_t db = p.f1_mn ? smem_desc_sw128(sf + kk * 2048, kF1AtomBytes) : smem_desc_sw128(sf, 16) + 2 * kk;
-            tc_mma_bf16(tmem_base, da0 + 2 * kk, db, idesc1, (ks | kk) != 0);
-            if (nt == 2) tc_mma_bf16(tmem_base + 256, da1 + 2 * kk, db, idesc1, (ks | kk) != 0);
+          const uint64_t da0 = dA1 + slot_step * slot1, db0 = dF1 + slot_step * slot1;
+          const int ksteps = p.cv.on ? (p.cv.in_ch - (kr % p.cv.cslabs) * 64 + 15) >> 4 : (p.K1 - kr * 64 + 15) >> 4;
+          const uint32_t acc0 = ks != 0;
+          if (nt == 2) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              if (kk < ksteps) {
+                tc_mma_bf16(tmem_base, da0 + 2 * kk, db0 + f1_step * kk, idesc1, kk ? 1u : acc0);
+                tc_mma_bf16(tmem_base + 256, da0 + blk_step + 2 * kk, db0 + f1_step * kk, idesc1, kk ? 1u : acc0);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              if (kk < ksteps) tc_mma_bf16(tmem_base, da0 + 2 * kk, db0 + f1_step * kk, idesc1, kk ? 1u : acc0);
           }
-          tc_commit(&bars->empty[slot]);
+          tc_commit(&bars->empty[slot1]);
+          if (++slot1 == p.ns) { slot1 = 0; ph1 ^= 1; }
+          if (++kr == p.nk1) kr = 0;
         }
         if (!ok) break;
         tc_commit(&bars->t_full);
@@ -354,19 +385,18 @@ chain_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ C
             if (!mbar_wait(&bars->acc_empty[b], ((b ? q1 : q0) & 1) ^ 1, lim)) { raise_timeout(bars, p.status); ok = false; break; }
             tc_fence_after();
             const uint32_t tacc = tmem_base + kChunk * b;
-            const uint8_t* Sb = S0 + (size_t)tt * p.natoms * kAtomBytes;
+            const uint64_t dSb = dS + blk_step * (uint64_t)(tt * p.natoms);
             for (int j = 0; j < p.natoms; ++j) {
               const int idx = i2 + j, slot = idx % p.ns2, ph = (idx / p.ns2) & 1;
               if (!mbar_wait(&bars->full2[slot], ph, lim)) { raise_timeout(bars, p.status); ok = false; break; }
               tc_fence_after();
-              const uint64_t da = smem_desc_sw128(smem_u32(Sb + j * kAtomBytes), 16);
-              const uint32_t sb = smem_u32(ring + (size_t)slot * kAtom2Bytes);
-              int ksteps = (p.r - j * 64) >> 4;
-              if (ksteps > 4) ksteps = 4;
-              for (int kk = 0; kk < ksteps; ++kk) {
-                const uint64_t db = p.f2_mn ? smem_desc_sw128(sb + kk * 2048, kF1AtomBytes) : smem_desc_sw128(sb, 16) + 2 * kk;
-                tc_mma_bf16(tacc, da + 2 * kk, db, idesc2, (j | kk) != 0);
-              }
+              const uint64_t da = dSb + blk_step * j;
+              const uint64_t db = dF2 + (uint64_t)(kAtom2Bytes >> 4) * slot;
+              const int ksteps = (p.r - j * 64) >> 4;
+              const uint32_t acc0 = j != 0;
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk)
+                if (kk < ksteps) tc_mma_bf16(tacc, da + 2 * kk, db + f2_step * kk, idesc2, kk ? 1u : acc0);
               if (tt == nt - 1) tc_commit(&bars->empty2[slot]);     // the last block of the unit is done with this tile
             }
             if (ok) { tc_commit(&bars->acc_full[b]); if (b) ++q1; else ++q0; }
@@ -939,7 +969,8 @@ ChainPlan chain_plan(int rp, int max_blocks, bool f1_mn) {
   pl.ns2 = (kSmemLimit - fixed) / kAtom2Bytes;
   if (pl.ns2 > kMaxStages2) pl.ns2 = kMaxStages2;
   if (pl.ns2 < 0) pl.ns2 = 0;
-  pl.ns = (pl.ns2 * kAtom2Bytes + s_bytes) / pl.slot_bytes;
+  // the first product's ring lies over the second product's ring, S and the staging tiles (all idle while it runs)
+  pl.ns = (pl.ns2 * kAtom2Bytes + s_bytes + kEpiWarps * kStgTiles * kGroupBytes) / pl.slot_bytes;
   if (pl.ns > kMaxStages) pl.ns = kMaxStages;
   pl.smem = (size_t)fixed + (size_t)pl.ns2 * kAtom2Bytes;
   // a two-block unit keeps every tile of a chunk of F2 until its second block has used it
@@ -1045,7 +1076,9 @@ int launch_chain_ex(const ChainLaunch& L, cudaStream_t st) {
   q.nchunks = second ? (L.P + kChunk - 1) / kChunk : 0;
   q.natoms = pl.natoms; q.max_blocks = pl.max_blocks; q.ns = pl.ns; q.slot_bytes = pl.slot_bytes; q.ns2 = pl.ns2;
   q.f1_bytes = pl.f1_bytes; q.f1_mn = L.f_mn ? 1 : 0; q.f2_mn = L.f_mn ? 1 : 0; q.save_s = L.Sg ? 1 : 0;
-  q.groups = (int)items; q.clear_status = L.clear_status ? 1 : 0; q.stall_selftest = L.stall_selftest ? 1 : 0;
+  q.groups = (int)items;
+  q.deal = (!conv && items >= (int64_t)8 * grid) ? 4 : 1;
+  q.clear_status = L.clear_status ? 1 : 0; q.stall_selftest = L.stall_selftest ? 1 : 0;
   q.wait_ns = L.wait_ns; q.status = L.status;
   if (conv) q.cv = *L.cv;
   q.out_ptr = static_cast<bf16*>(L.Out); q.s_ptr = static_cast<bf16*>(L.Sg); q.s_ld = L.s_ld; q.s_cols = L.s_cols;
