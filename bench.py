@@ -229,10 +229,21 @@ def vit_model_sync(ab, torch, steps=5):
         torch.cuda.synchronize()
         res[name] = e0.elapsed_time(e1) / steps
     bad = int(plan.status.abs().sum().item())
+    # the same model through the dense route (W formed, block Jacobi at short side 768): what a decomposition
+    # costs when W is not of rank <= r any more; one warm-up, one timed call
+    ab.ab_group_sync(plan_now, path=ab.AB_SYNC_DENSE)
+    torch.cuda.synchronize()
+    e0, e1 = ev(), ev()
+    e0.record()
+    ab.ab_group_sync(plan_now, path=ab.AB_SYNC_DENSE)
+    e1.record()
+    torch.cuda.synchronize()
+    res["dense"] = e0.elapsed_time(e1)
+    bad += int(plan_now.status.abs().sum().item())
     pk = measured_peaks()
     mean_bytes = (K + 1) * 4.0 * total
     return dict(workload="vit_b16_full_sync_72_matrices_fp32_K8_cutoff0.1", ms_per_model=res["sync"],
-                ms_per_model_without_W=res["sync_now"], ms_per_matrix=res["sync"] / len(shapes),
+                ms_per_model_without_W=res["sync_now"], ms_per_model_dense_route=res["dense"], ms_per_matrix=res["sync"] / len(shapes),
                 mean_ms=res["mean"], mean_gbs=mean_bytes / (res["mean"] * 1e-3) / 1e9,
                 mean_frac_of_measured_hbm=mean_bytes / (res["mean"] * 1e-3) / 1e9 / pk["hbm"],
                 mean_frac_of_nominal_8tbs=mean_bytes / (res["mean"] * 1e-3) / 1e9 / 8000.0,
@@ -353,6 +364,98 @@ def conv_workloads(ab, torch, iters=10):
                          activation_gbs=nbytes / (ms * 1e-3) / 1e9, frac_of_hbm=nbytes / (ms * 1e-3) / 1e9 / pk["hbm"],
                          bytes_vs_materialised_rows=nbytes / (2.0 * N * (3 * 9 * C + 2 * m)),
                          device_status=ab.workspace_status(ws))
+    return out
+
+
+def training_cycle(ab, torch, N=256 * 197, n_ab=4, n_dense=1, K=K_GROUPS):
+    """One whole cycle of Algorithm 1 on one GPU for the ViT-B/16 MLP pair, every step through the library:
+    decomposition of the dense weights (ab_svd_split, rank 192) -> n_ab factorised steps (forward, backward,
+    AdamW on A and B) -> group synchronisation of K copies (mean, W = Abar Bbar, written) -> n_dense full-rank
+    steps (dense forward, backward, AdamW on W) -> decomposition again.  The paper's ratio of factorised to
+    rebound steps is 4 : 1.  Event-timed per phase; the K copies are the trained factors plus N(0, 1e-3) noise."""
+    from paper_2405_01067_b200 import synth
+    bf = torch.bfloat16
+    w = synth.vit_mlp_weights(seed=1)
+    layers = []
+    for li, (m, n) in enumerate(LAYERS):
+        d = synth.vit_mlp(li + 1, seed=7, N=N, K=K)
+        g = dict(m=m, n=n, W=torch.from_numpy(w["W1" if li == 0 else "W2"]).cuda(),
+                 x=torch.from_numpy(d["x"]).to(bf).cuda(), dY=torch.from_numpy(d["dY"]).to(bf).cuda(),
+                 noise_A=torch.from_numpy(np.stack(d["noise_A"])).cuda(), noise_B=torch.from_numpy(np.stack(d["noise_B"])).cuda(),
+                 y=torch.empty((N, m), dtype=bf, device="cuda"), T=torch.empty((N, R), dtype=bf, device="cuda"),
+                 dX=torch.empty((N, n), dtype=bf, device="cuda"), dA=torch.empty((m, R), device="cuda"),
+                 dB=torch.empty((R, n), device="cuda"), dW=torch.empty((m, n), device="cuda"),
+                 W_lp=torch.empty((m, n), dtype=bf, device="cuda"), A_lp=torch.empty((m, R), dtype=bf, device="cuda"),
+                 B_lp=torch.empty((R, n), dtype=bf, device="cuda"))
+        for nm, shape in (("A", (m, R)), ("B", (R, n)), ("W", (m, n))):
+            g["m_" + nm] = torch.zeros(shape, device="cuda")
+            g["v_" + nm] = torch.zeros(shape, device="cuda")
+        g["ws_f"] = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_FORWARD, N, m, n, R, 1, ab.AB_BF16), "cuda")
+        g["ws_b"] = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_LAYER_BACKWARD, N, m, n, R, 1, ab.AB_BF16), "cuda")
+        g["ws_df"] = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_DENSE_FORWARD, N, m, n, 0, 1, ab.AB_BF16), "cuda")
+        g["ws_db"] = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_DENSE_BACKWARD, N, m, n, 0, 1, ab.AB_BF16), "cuda")
+        g["ws_s"] = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_SVD_SPLIT, 0, m, n, R, 1, ab.AB_F32), "cuda")
+        layers.append(g)
+
+    def decompose():
+        for g in layers:
+            g["A"], g["B"], g["sigma"], g["r_out"], g["st"] = ab.ab_svd_split(g["W"], R, 0.0, ws=g["ws_s"])
+            ab.ab_group_average(g["A"][None], out=g["A_lp"])        # the bf16 copies the chain reads (a mean of one)
+            ab.ab_group_average(g["B"][None], out=g["B_lp"])
+
+    def ab_steps():
+        for step in range(1, n_ab + 1):
+            lr = 1e-3 * ab.ab_lr_rebound_factor(step, 2, 0.05)
+            for g in layers:
+                ab.ab_layer_forward(g["x"], g["A_lp"], g["B_lp"], y=g["y"], T_save=g["T"], ws=g["ws_f"])
+                ab.ab_layer_backward(g["x"], g["dY"], g["A_lp"], g["B_lp"], T_saved=g["T"], dX=g["dX"], dA=g["dA"], dB=g["dB"],
+                                     ws=g["ws_b"])
+                ab.ab_adamw_step(g["A"], g["dA"], g["m_A"], g["v_A"], lr, step, param_bf16=g["A_lp"])
+                ab.ab_adamw_step(g["B"], g["dB"], g["m_B"], g["v_B"], lr, step, param_bf16=g["B_lp"])
+
+    def sync():
+        copies_A = [g["A"][None] + g["noise_A"] for g in layers]      # input assembly: the K groups' copies
+        copies_B = [g["B"][None] + g["noise_B"] for g in layers]
+        plan = ab.SyncPlan(copies_A, copies_B, 0.0, want_W=True)
+        return plan
+
+    def sync_run(plan):
+        ab.ab_group_sync(plan)
+        for g, Wn in zip(layers, plan.W_out):
+            g["W"] = Wn
+            ab.ab_group_average(Wn[None], out=g["W_lp"])
+
+    def dense_steps():
+        for step in range(1, n_dense + 1):
+            lr = 1e-3 * ab.ab_lr_rebound_factor(step, 2, 0.05)
+            for g in layers:
+                ab.ab_dense_forward(g["x"], g["W_lp"], y=g["y"], ws=g["ws_df"])
+                ab.ab_dense_backward(g["x"], g["dY"], g["W_lp"], dX=g["dX"], dW=g["dW"], ws=g["ws_db"])
+                ab.ab_adamw_step(g["W"], g["dW"], g["m_W"], g["v_W"], lr, step, param_bf16=g["W_lp"])
+
+    def timed(fn):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    decompose()                      # warm-up of every kernel on the way
+    ab_steps()
+    plan = sync()
+    sync_run(plan)
+    dense_steps()
+    out = dict(workload="vit_b16_mlp_pair, one cycle", rows=N, n_ab_steps=n_ab, n_dense_steps=n_dense, K=K)
+    out["decompose_ms"] = timed(decompose)
+    out["ab_steps_ms"] = timed(ab_steps)
+    plan = sync()
+    out["sync_ms"] = timed(lambda: sync_run(plan))
+    out["dense_steps_ms"] = timed(dense_steps)
+    out["decompose_again_ms"] = timed(decompose)
+    out["cycle_ms"] = sum(out[k] for k in ("decompose_ms", "ab_steps_ms", "sync_ms", "dense_steps_ms"))
+    out["device_status"] = [int(g["st"].item()) for g in layers] + [int(plan.status.abs().sum().item())]
     return out
 
 
@@ -652,6 +755,8 @@ def run_ours(args):
             line["adamw_update_vit_factors"] = optimizer_step(ab, torch)
             line["dense_split_ms"] = dense_split_times(ab, torch)
             line["implicit_conv"] = conv_workloads(ab, torch)
+            torch.cuda.empty_cache()
+            line["training_cycle"] = training_cycle(ab, torch)
         if world == 1 and not args.no_cpu_baseline:
             cb = cpu_baseline(inputs, min(N, args.baseline_rows), sync_scale=4)    # about 10 s of host work
             line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}

@@ -6,7 +6,7 @@
 //   * vectors are stored as ROWS (X is s x s, V^T is s x s), split into blocks of b rows;
 //   * a sweep is nb-1 rounds of disjoint block pairs (round-robin); one CTA per pair keeps the
 //     2b x s panel in shared memory (b = 16), forms its 32 x 32 Gram matrix M, runs a few
-//     sweeps of a two-sided cyclic Jacobi on M inside one warp's registers (accumulating Q),
+//     sweeps of a two-sided cyclic Jacobi on M in shared memory (accumulating Q),
 //     applies Q^T to the panel and to the matching panel of V^T;
 //   * sweeps repeat until no pair of rows has |x_i.x_j| > tol |x_i||x_j| (a device flag; the
 //     host enqueues a fixed number of sweeps and converged matrices return at once).
@@ -17,6 +17,8 @@
 #include <vector>
 #include <algorithm>
 #include <map>
+
+#include <cooperative_groups.h>
 
 #include "ab_common.cuh"
 
@@ -34,7 +36,7 @@ struct JState {
 };
 
 constexpr int kMaxSweeps = 30;
-constexpr int kInnerSweeps = 2;
+constexpr int kInnerSweeps = 1;
 constexpr float kCountRel2 = 1e-8f;  // rows below 1e-4 of the largest norm do not hold up convergence
 constexpr float kDeadRel2 = 1e-12f;   // rows below 1e-6 of the largest norm count as zero
 // Accuracy domain of this route: a kept singular value between kZeroRel and kDomainRel of the largest has lost
@@ -87,108 +89,123 @@ __device__ __forceinline__ void rr_pair(int ne, int t, int k, int& p, int& q) {
   if (p > q) { int tmp = p; p = q; q = tmp; }
 }
 
-// ---- 32 x 32 symmetric eigenproblem in one warp ------------------------------------------------
-// Two-sided cyclic Jacobi with the tournament ordering: pairs always sit at positions (2k, 2k+1),
-// and after every step all positions but 0 move one place round the cycle
-// 2 -> 4 -> ... -> 30 -> 31 -> 29 -> ... -> 3 -> 1 -> 2, so that in 31 steps every pair has met
-// once and everything is back in place.  Lane l holds column l of the working matrix and of Q
-// (rows in registers): column rotations and the column moves are warp shuffles, row rotations
-// and the row moves act on registers with compile-time indices.  No shared memory, no barrier.
-__host__ __device__ constexpr int tour_cycle(int i) { return i < 15 ? 2 * (i + 1) : 31 - 2 * (i - 15); }
-__host__ __device__ constexpr int tour_index(int pos) { return (pos & 1) ? 15 + (31 - pos) / 2 : pos / 2 - 1; }
-__host__ __device__ constexpr int tour_next(int pos) { return pos == 0 ? 0 : tour_cycle((tour_index(pos) + 1) % 31); }
-__host__ __device__ constexpr int tour_prev(int pos) { return pos == 0 ? 0 : tour_cycle((tour_index(pos) + 30) % 31); }
-
-template <int J> struct TourMove {
-  __device__ static __forceinline__ void run(const float (&y)[32], float (&ny)[32]) {
-    ny[tour_next(J)] = y[J];
-    TourMove<J + 1>::run(y, ny);
-  }
-};
-template <> struct TourMove<32> {
-  __device__ static __forceinline__ void run(const float (&)[32], float (&)[32]) {}
-};
-
-// y: column `lane` of the symmetric matrix, q: column `lane` of Q (identity on entry).
-// Rotates pairs whose |m_pq| > thr sqrt(m_pp m_qq); rows whose diagonal is <= dead2 are left alone.
-__device__ __forceinline__ void warp_eig32(float (&y)[32], float (&q)[32], float thr, float dead2, int max_sweeps) {
-  constexpr unsigned FULL = 0xffffffffu;
-  const int lane = threadIdx.x & 31;
-  const bool even = (lane & 1) == 0;
-  const int src = tour_prev(lane);     // the lane whose column moves here after a step
-  for (int sweep = 0; sweep < max_sweeps; ++sweep) {
-    bool rotated = false;
-    for (int step = 0; step < 31; ++step) {
-      float d = 0.f, e = 0.f;
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        if (j == lane) d = y[j];
-        if (j == (lane ^ 1)) e = y[j];
-      }
-      const float dpart = __shfl_xor_sync(FULL, d, 1);
-      const float g = __shfl_sync(FULL, e, lane & ~1);
-      const float app = even ? d : dpart, aqq = even ? dpart : d;
-      float c = 1.f, sn = 0.f;
-      if (app > dead2 && aqq > dead2 && app > 0.f && aqq > 0.f && fabsf(g) > thr * sqrtf(app) * sqrtf(aqq)) {
-        const float zeta = (aqq - app) / (2.f * g);
-        const float t = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
-        c = 1.f / sqrtf(1.f + t * t);   // IEEE sqrt and divide: c^2 + s^2 = 1 to an ulp, no drift
-        sn = c * t;
-      }
-      const bool any = __any_sync(FULL, sn != 0.f);
-      if (any) {
-        rotated = true;
-        const float ss = even ? -sn : sn;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {   // columns p, q of M and of Q
-          const float o = __shfl_xor_sync(FULL, y[j], 1);
-          y[j] = c * y[j] + ss * o;
-          const float oq = __shfl_xor_sync(FULL, q[j], 1);
-          q[j] = c * q[j] + ss * oq;
-        }
-#pragma unroll
-        for (int k = 0; k < 16; ++k) {   // rows 2k, 2k+1 of M with that pair's rotation
-          const float ck = __shfl_sync(FULL, c, 2 * k), sk = __shfl_sync(FULL, sn, 2 * k);
-          const float a = y[2 * k], b = y[2 * k + 1];
-          y[2 * k] = ck * a - sk * b;
-          y[2 * k + 1] = sk * a + ck * b;
-        }
-      }
-      float ny[32];
-      TourMove<0>::run(y, ny);
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        y[j] = __shfl_sync(FULL, ny[j], src);
-        q[j] = __shfl_sync(FULL, q[j], src);
-      }
-    }
-    if (!rotated) break;
+// ---- 32 x 32 symmetric eigenproblem of a panel ---------------------------------------------------
+// Two-sided cyclic Jacobi: 31 steps of 16 disjoint pairs (round-robin tournament) cover every pair once.
+// Solved by the whole CTA (256 threads) in shared memory, two barriers and a few dozen instructions per thread
+// and step; an earlier version that kept the matrix
+// in one warp's registers and moved columns by shuffles took a few hundred dependent shuffles per step
+// (measured on the 3072 x 768 split: 118 us per round of the block Jacobi with it).
+// Ms: the symmetric matrix (leading dimension ldm), Qs: receives Q (identity on entry is set here).
+// Rotation that annihilates M[p][q].  Approximate reciprocal and square-root units are enough here: an error in
+// c scales both rotated vectors alike (their orthogonality is untouched, and the singular vectors are
+// normalised at the end), an error in t leaves a residue of second order that the next sweep removes.
+__device__ __forceinline__ void jacobi_rotation(const float* Ms, int ldm, int pp, int qq, float thr, float dead2,
+                                                float& c, float& sn) {
+  const float app = Ms[pp * ldm + pp], aqq = Ms[qq * ldm + qq], g = Ms[pp * ldm + qq];
+  c = 1.f; sn = 0.f;
+  if (app > dead2 && aqq > dead2 && app > 0.f && aqq > 0.f && g * g > thr * thr * app * aqq) {
+    float zeta = __fdividef(aqq - app, 2.f * g);
+    zeta = fminf(fmaxf(zeta, -1e15f), 1e15f);
+    const float h = fmaf(zeta, zeta, 1.f);
+    const float t = __fdividef(copysignf(1.f, zeta), fabsf(zeta) + h * rsqrtf(h));
+    c = rsqrtf(fmaf(t, t, 1.f));
+    sn = c * t;
   }
 }
 
-// One CTA per block pair: PB = 32 rows (16 + 16) or PB = 16 (8 + 8, for long vectors).
-template <int PB>
+// Thread (k, k2) of the 16 x 16 grid owns the 2 x 2 block of M at the rows of pair k and the columns of pair k2.
+// Per step: 16 threads work out the 16 rotations (the pairs of all 31 steps come from a table built once); after
+// a barrier every thread reads its block, applies J_k^T B J_k2 and writes it back (the blocks of a step are
+// disjoint), and carries two rows of Q through the column rotation of pair k2; a second barrier ends the step.
+struct EigScratch {
+  unsigned char pp[31 * 16], qq[31 * 16];
+  float c[16], s[16];
+  int flag;
+};
+__device__ __forceinline__ void cta_eig32(float* Ms, float* Qs, int ldm, float thr, float dead2, int max_sweeps, EigScratch* es) {
+  const int tid = threadIdx.x;
+  const int k = tid >> 4, k2 = tid & 15;
+  for (int idx = tid; idx < 32 * 32; idx += 256) Qs[(idx >> 5) * ldm + (idx & 31)] = ((idx >> 5) == (idx & 31)) ? 1.f : 0.f;
+  for (int idx = tid; idx < 31 * 16; idx += 256) {
+    int a, b;
+    rr_pair(32, idx >> 4, idx & 15, a, b);
+    es->pp[idx] = (unsigned char)a; es->qq[idx] = (unsigned char)b;
+  }
+  __syncthreads();
+  for (int sweep = 0; sweep < max_sweeps; ++sweep) {
+    if (tid == 0) es->flag = 0;
+    __syncthreads();
+    for (int step = 0; step < 31; ++step) {
+      if (tid < 16) {
+        float c, sn;
+        jacobi_rotation(Ms, ldm, es->pp[step * 16 + tid], es->qq[step * 16 + tid], thr, dead2, c, sn);
+        es->c[tid] = c; es->s[tid] = sn;
+        if (sn != 0.f) es->flag = 1;
+      }
+      __syncthreads();
+      const float c1 = es->c[k], s1 = es->s[k], c2 = es->c[k2], s2 = es->s[k2];
+      const int p1 = es->pp[step * 16 + k], q1 = es->qq[step * 16 + k], p2 = es->pp[step * 16 + k2], q2 = es->qq[step * 16 + k2];
+      if (s1 != 0.f || s2 != 0.f) {
+        const float b00 = Ms[p1 * ldm + p2], b01 = Ms[p1 * ldm + q2], b10 = Ms[q1 * ldm + p2], b11 = Ms[q1 * ldm + q2];
+        // rows (pair k), then columns (pair k2)
+        const float r00 = c1 * b00 - s1 * b10, r10 = s1 * b00 + c1 * b10;
+        const float r01 = c1 * b01 - s1 * b11, r11 = s1 * b01 + c1 * b11;
+        Ms[p1 * ldm + p2] = c2 * r00 - s2 * r01; Ms[p1 * ldm + q2] = s2 * r00 + c2 * r01;
+        Ms[q1 * ldm + p2] = c2 * r10 - s2 * r11; Ms[q1 * ldm + q2] = s2 * r10 + c2 * r11;
+      }
+      if (s2 != 0.f) {
+        const int i0 = k, i1 = k + 16;                // the two rows of Q this thread rotates (columns p2, q2)
+        const float qa0 = Qs[i0 * ldm + p2], qb0 = Qs[i0 * ldm + q2], qa1 = Qs[i1 * ldm + p2], qb1 = Qs[i1 * ldm + q2];
+        Qs[i0 * ldm + p2] = c2 * qa0 - s2 * qb0; Qs[i0 * ldm + q2] = s2 * qa0 + c2 * qb0;
+        Qs[i1 * ldm + p2] = c2 * qa1 - s2 * qb1; Qs[i1 * ldm + q2] = s2 * qa1 + c2 * qb1;
+      }
+      __syncthreads();
+    }
+    if (!es->flag) break;
+  }
+}
+
+// One cluster of kCl CTAs (8, or 1 when a batch already fills the device) per block pair: PB = 32 rows (16 + 16)
+// or PB = 16 (8 + 8).  A panel is only PB rows, so
+// one CTA per pair would leave most of the device idle (24 CTAs for a 768 x 768 matrix: 116 us per round); the
+// columns of the panel are cut into kCl slices instead, one per CTA of the cluster.  Each CTA forms the Gram matrix
+// of its slice; the partial matrices are added through distributed shared memory in ascending CTA order, so every
+// CTA of the cluster holds the same M to the bit, solves the same small eigenproblem and rotates its own slice of
+// the X panel and of the V^T panel.  No wait spins: the only waits are cluster barriers that every CTA of the
+// cluster reaches (all early exits depend on values the whole cluster agrees on).
+template <int PB, int kCl>
 __global__ void __launch_bounds__(256, 2)
 jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, int nb, int round,
                    float tol, JState* __restrict__ states) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
   constexpr int HB = PB / 2;          // rows per block
-  constexpr int RT = PB / 16;         // register tile of the panel Gram
   constexpr int LDM = 33;
   constexpr int LDQ = PB + 4;
   extern __shared__ __align__(16) float smem[];
   const int mat = blockIdx.y;
+  const int pair = blockIdx.x / kCl, crank = blockIdx.x % kCl;
   JState* st = states + mat;
-  if (st->done) return;
+  if (st->done) return;               // the same for the whole cluster
   const int nbe = nb + (nb & 1);
   int bi, bj;
-  rr_pair(nbe, round, blockIdx.x, bi, bj);
-  if (bj >= nb && nb > 1) return;     // this block sits the round out
-  const int ldp = ((s + 3) & ~3) + 4;
+  rr_pair(nbe, round, pair, bi, bj);
+  if (bj >= nb && nb > 1) return;     // this block sits the round out (whole cluster)
+  // this CTA's slice of the columns: multiples of 4, as equal as they come
+  const int s4 = (s + 3) >> 2;
+  const int c_lo = (int)((long long)crank * s4 / kCl) * 4;
+  int c_hi = (int)((long long)(crank + 1) * s4 / kCl) * 4;
+  if (c_hi > s) c_hi = s;
+  const int w = c_hi > c_lo ? c_hi - c_lo : 0;     // width of the slice
+  const int ldp = (((s4 + kCl - 1) / kCl) * 4) + 4;  // the same in every CTA
   float* P = smem;                    // PB x ldp
-  float* Ms = P + (size_t)PB * ldp;   // 32 x LDM (zero beyond PB)
-  float* Qt = Ms + 32 * LDM + 3;      // PB x LDQ, Qt[c][i] = Q[i][c]; (32*33+3) % 4 == 3 -> realigned below
+  float* Mp = P + (size_t)PB * ldp;   // 32 x LDM: this CTA's partial Gram matrix (zero beyond PB)
+  float* Ms = Mp + 32 * LDM;          // 32 x LDM: the sum
+  float* Qs = Ms + 32 * LDM;          // 32 x LDM
+  float* Qt = Qs + 32 * LDM + 1;      // PB x LDQ, Qt[c][i] = Q[i][c]; realigned below
   Qt = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(Qt) + 15) & ~(uintptr_t)15);
   __shared__ int any_rot;
+  __shared__ EigScratch eig_scratch;
   const int tid = threadIdx.x;
   float* X = Xall + (size_t)mat * s * s;
   float* V = Vall + (size_t)mat * s * s;
@@ -202,22 +219,21 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
     return g < s ? g : -1;
   };
   auto load_panel = [&](const float* src) {
-    const int s4 = ldp - 4;           // padded row length handled, multiple of 4
     for (int lr = tid >> 5; lr < PB; lr += 8) {      // a warp per row: coalesced
       const int g = grow(lr);
-      for (int k = tid & 31; k < s4; k += 32)
-        P[(size_t)lr * ldp + k] = (g >= 0 && k < s) ? src[(size_t)g * s + k] : 0.f;
+      for (int k = tid & 31; k < ldp - 4; k += 32)
+        P[(size_t)lr * ldp + k] = (g >= 0 && k < w) ? src[(size_t)g * s + c_lo + k] : 0.f;
     }
   };
   auto store_panel = [&](float* dst) {
     for (int lr = tid >> 5; lr < PB; lr += 8) {
       const int g = grow(lr);
       if (g < 0) continue;
-      for (int k = tid & 31; k < s; k += 32) dst[(size_t)g * s + k] = P[(size_t)lr * ldp + k];
+      for (int k = tid & 31; k < w; k += 32) dst[(size_t)g * s + c_lo + k] = P[(size_t)lr * ldp + k];
     }
   };
   auto apply_q = [&]() {              // P <- Q^T P, one panel column per thread at a time
-    for (int k = tid; k < s; k += 256) {
+    for (int k = tid; k < w; k += 256) {
       float col[PB];
 #pragma unroll
       for (int j = 0; j < PB; ++j) col[j] = P[(size_t)j * ldp + k];
@@ -239,52 +255,47 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
   };
 
   load_panel(X);
-  for (int idx = tid; idx < 32 * LDM; idx += 256) Ms[idx] = 0.f;
+  for (int idx = tid; idx < 32 * LDM; idx += 256) Mp[idx] = 0.f;
   if (tid == 0) any_rot = 0;
   __syncthreads();
 
-  // ---- M = P P^T
-  {
-    const int tx = tid & 15, ty = tid >> 4;
-    float acc[RT][RT];
-#pragma unroll
-    for (int i = 0; i < RT; ++i)
-#pragma unroll
-      for (int j = 0; j < RT; ++j) acc[i][j] = 0.f;
-    const int s4 = ldp - 4;
-    for (int k = 0; k < s4; k += 4) {
-      float4 a[RT], b[RT];
-#pragma unroll
-      for (int i = 0; i < RT; ++i) a[i] = *reinterpret_cast<const float4*>(P + (size_t)(ty + 16 * i) * ldp + k);
-#pragma unroll
-      for (int j = 0; j < RT; ++j) b[j] = *reinterpret_cast<const float4*>(P + (size_t)(tx + 16 * j) * ldp + k);
-#pragma unroll
-      for (int i = 0; i < RT; ++i)
-#pragma unroll
-        for (int j = 0; j < RT; ++j) {
-          acc[i][j] = fmaf(a[i].x, b[j].x, acc[i][j]);
-          acc[i][j] = fmaf(a[i].y, b[j].y, acc[i][j]);
-          acc[i][j] = fmaf(a[i].z, b[j].z, acc[i][j]);
-          acc[i][j] = fmaf(a[i].w, b[j].w, acc[i][j]);
-        }
+  // ---- partial Gram matrix of this slice: entry (i, j) by thread i * PB + j (and + 256 ...), k ascending
+  for (int e = tid; e < PB * PB; e += 256) {
+    const int i = e / PB, jj = e - i * PB;
+    if (jj < i) continue;             // symmetric: the upper triangle is computed, the lower mirrored
+    const float4* a = reinterpret_cast<const float4*>(P + (size_t)i * ldp);
+    const float4* b = reinterpret_cast<const float4*>(P + (size_t)jj * ldp);
+    float acc = 0.f;
+    for (int k = 0; k < (ldp - 4) / 4; ++k) {
+      const float4 x = a[k], y = b[k];
+      acc = fmaf(x.x, y.x, acc); acc = fmaf(x.y, y.y, acc); acc = fmaf(x.z, y.z, acc); acc = fmaf(x.w, y.w, acc);
     }
-#pragma unroll
-    for (int i = 0; i < RT; ++i)
-#pragma unroll
-      for (int j = 0; j < RT; ++j) Ms[(ty + 16 * i) * LDM + tx + 16 * j] = acc[i][j];
+    Mp[i * LDM + jj] = acc;
+    Mp[jj * LDM + i] = acc;
   }
-  __syncthreads();
+  if constexpr (kCl > 1) cluster.sync(); else __syncthreads();     // every CTA's partial matrix is complete
+  for (int idx = tid; idx < 32 * LDM; idx += 256) {
+    float acc = 0.f;
+    if constexpr (kCl > 1) {
+#pragma unroll
+      for (int c = 0; c < kCl; ++c) acc += cluster.map_shared_rank(Mp, c)[idx];   // ascending CTA order in every CTA
+    } else {
+      acc = Mp[idx];
+    }
+    Ms[idx] = acc;
+  }
+  if constexpr (kCl > 1) cluster.sync(); else __syncthreads();     // nobody reads a peer's partial matrix after this
 
   // ---- how far from orthogonal is this panel?  (also collects the largest squared norm)
   {
     float worst = 0.f, big = 0.f;
     int rot = 0;
     for (int idx = tid; idx < PB * PB; idx += 256) {
-      int i = idx / PB, j = idx - i * PB;
-      float mii = Ms[i * LDM + i], mjj = Ms[j * LDM + j];
-      if (i == j) { big = fmaxf(big, mii); continue; }
-      if (i < j && mii > dead2 && mjj > dead2 && mii > 0.f && mjj > 0.f) {
-        float rel = fabsf(Ms[i * LDM + j]) / (sqrtf(mii) * sqrtf(mjj));
+      int i = idx / PB, jj = idx - i * PB;
+      float mii = Ms[i * LDM + i], mjj = Ms[jj * LDM + jj];
+      if (i == jj) { big = fmaxf(big, mii); continue; }
+      if (i < jj && mii > dead2 && mjj > dead2 && mii > 0.f && mjj > 0.f) {
+        float rel = fabsf(Ms[i * LDM + jj]) / (sqrtf(mii) * sqrtf(mjj));
         if (rel > tol) rot = 1;
         // rows far below the largest norm are rounding noise of the large ones: they are still
         // rotated, but the sweep counts as converged without them
@@ -296,32 +307,24 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
       worst = fmaxf(worst, __shfl_xor_sync(0xffffffffu, worst, o));
       big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, o));
     }
-    if ((tid & 31) == 0) {
+    if ((tid & 31) == 0 && crank == 0) {
       atomicMax(&st->off_bits, __float_as_uint(worst));
       atomicMax(&st->next_maxn2_bits, __float_as_uint(big));
     }
     if (rot) atomicExch(&any_rot, 1);
   }
   __syncthreads();
-  if (!any_rot) return;               // panel already orthogonal: nothing to write
+  if (!any_rot) return;               // panel already orthogonal: nothing to write (the same M in every CTA)
 
-  // ---- diagonalise M in warp 0 (the other warps wait at the barrier)
-  if (tid < 32) {
-    float y[32], q[32];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      y[j] = Ms[j * LDM + tid];
-      q[j] = (j == tid) ? 1.f : 0.f;
-    }
-    warp_eig32(y, q, 0.25f * tol, dead2, kInnerSweeps);
-    if (tid < PB) {
-#pragma unroll
-      for (int i = 0; i < PB; ++i) Qt[tid * LDQ + i] = q[i];
-    }
+  // ---- diagonalise M (all threads; the same arithmetic in every CTA of the cluster), then Qt[c][i] = Q[i][c]
+  cta_eig32(Ms, Qs, LDM, 0.25f * tol, dead2, kInnerSweeps, &eig_scratch);
+  for (int idx = tid; idx < PB * PB; idx += 256) {
+    const int c = idx / PB, i = idx - c * PB;
+    Qt[c * LDQ + i] = Qs[i * LDM + c];
   }
   __syncthreads();
 
-  // ---- rotate the panel of X, then the same rows of V^T
+  // ---- rotate this slice of the panel of X, then of the same rows of V^T
   apply_q();
   __syncthreads();
   store_panel(X);
@@ -333,10 +336,11 @@ jacobi_pair_kernel(float* __restrict__ Xall, float* __restrict__ Vall, int s, in
   store_panel(V);
 }
 
-template <int PB>
+template <int PB, int kCl>
 size_t jacobi_smem_bytes(int s) {
-  const int ldp = ((s + 3) & ~3) + 4;
-  return sizeof(float) * ((size_t)PB * ldp + 32 * 33 + 8 + (size_t)PB * (PB + 4));
+  const int s4 = (s + 3) >> 2;
+  const int ldp = (((s4 + kCl - 1) / kCl) * 4) + 4;
+  return sizeof(float) * ((size_t)PB * ldp + 3 * 32 * 33 + 8 + (size_t)PB * (PB + 4));
 }
 
 // lam[i] = |row i of X|, perm = indices by descending lam (ties by index).  One CTA per matrix.
@@ -598,24 +602,44 @@ Layout make_layout(const SvdItem* items, int L, void* ws) {
   return lo;
 }
 
-template <int PB>
-int run_jacobi(float* X, float* Vt, JState* st, int s, int nb, int count, cudaStream_t stream) {
-  const size_t smem = jacobi_smem_bytes<PB>(s);
+template <int PB, int CL>
+int run_jacobi_cl(float* X, float* Vt, JState* st, int s, int nb, int count, cudaStream_t stream) {
+  const size_t smem = jacobi_smem_bytes<PB, CL>(s);
   if (smem > 227 * 1024) return AB_ERR_UNSUPPORTED;
-  AB_CUDA_OK(cudaFuncSetAttribute(jacobi_pair_kernel<PB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  AB_CUDA_OK(cudaFuncSetAttribute(jacobi_pair_kernel<PB, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const int nbe = nb + (nb & 1);
   const int rounds = nbe > 2 ? nbe - 1 : 1;
   const float tol = jacobi_tol(s);
-  dim3 grid((unsigned)(nbe / 2), (unsigned)count);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(nbe / 2) * CL, (unsigned)count);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CL; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
   for (int sw = 0; sw < kMaxSweeps; ++sw) {
     for (int r = 0; r < rounds; ++r) {
-      jacobi_pair_kernel<PB><<<grid, 256, smem, stream>>>(X, Vt, s, nb, r, tol, st);
+      AB_CUDA_OK(cudaLaunchKernelEx(&cfg, jacobi_pair_kernel<PB, CL>, X, Vt, s, nb, r, tol, st));
     }
     sweep_end_kernel<<<(count + 127) / 128, 128, 0, stream>>>(st, count, tol);
   }
   count_launches((long long)kMaxSweeps * (rounds + 1) - 1);
   AB_LAUNCH_OK();
   return AB_OK;
+}
+
+// Clusters of 8 CTAs per block pair while that leaves the device room for every pair of a round (a lone matrix);
+// one CTA per pair for batches, whose pairs fill the device by themselves.
+template <int PB>
+int run_jacobi(float* X, float* Vt, JState* st, int s, int nb, int count, cudaStream_t stream) {
+  const int nbe = nb + (nb & 1);
+  const long long pairs = (long long)(nbe / 2) * count;
+  int sms = sm_count();
+  if (sms <= 0) sms = 1;
+  if (pairs * 8 <= 2LL * sms + 8) return run_jacobi_cl<PB, 8>(X, Vt, st, s, nb, count, stream);
+  return run_jacobi_cl<PB, 1>(X, Vt, st, s, nb, count, stream);
 }
 
 }  // namespace
