@@ -34,9 +34,9 @@ NOMINAL_BF16_TFLOPS = 2250.0
 R = 192
 LAYERS = ((3072, 768), (768, 3072))
 K_GROUPS = 4
-# dram__bytes_read.sum + dram__bytes_write.sum of one row_chain_units_kernel launch (forward, 50,432 rows),
-# from the ncu capture summarised under profiles/; None until the kernel of that capture is current.
-ROW_CHAIN_DRAM_BYTES_PER_LAUNCH = 349.8e6   # forward of W1: 79.4 MB read + 270.4 MB written (ncu capture under profiles/)
+# dram__bytes_read.sum + dram__bytes_write.sum of one chain_kernel launch (forward of W1, 50,432 rows), from the
+# ncu capture summarised under profiles/; None until the kernel of that capture is current.
+ROW_CHAIN_DRAM_BYTES_PER_LAUNCH = 352.5e6   # 79.5 MB read + 273.0 MB written
 
 
 def chain_flops(N, layers=LAYERS, r=R):
@@ -459,6 +459,42 @@ def training_cycle(ab, torch, N=256 * 197, n_ab=4, n_dense=1, K=K_GROUPS):
     return out
 
 
+def fused_mean_recombine(ab, torch, iters=10):
+    """Mean of K = 8 copies and W = Abar Bbar for one ViT-B/16 matrix of each shape: the one-kernel form (the mean
+    as the product's operand prologue, ab_recombine_mean) against the separate calls (ab_group_average twice,
+    then ab_recombine on the tensor cores)."""
+    out = {}
+    K, r = 8, 192
+    for (m, n) in ((768, 768), (3072, 768), (768, 3072)):
+        Ak = torch.randn((K, m, r), device="cuda")
+        Bk = torch.randn((K, r, n), device="cuda")
+        W = torch.empty((m, n), device="cuda")
+        Ab, Bb = torch.empty((m, r), device="cuda"), torch.empty((r, n), device="cuda")
+        ws = ab.workspace(ab.ab_workspace_bytes(ab.AB_OP_RECOMBINE, 0, m, n, r, 1, ab.AB_F32), "cuda")
+
+        def separate():
+            ab.ab_group_average(Ak, out=Ab)
+            ab.ab_group_average(Bk, out=Bb)
+            ab.ab_recombine(Ab, Bb, W=W, ws=ws)
+
+        def fused():
+            ab.ab_recombine_mean(Ak, Bk, W=W, Abar=Ab, Bbar=Bb)
+        res = {}
+        for name, fn in (("separate_us", separate), ("one_kernel_us", fused)):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(iters):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            res[name] = e0.elapsed_time(e1) / iters * 1e3
+        out[f"{m}x{n}"] = res
+    return out
+
+
 def dense_split_times(ab, torch, iters=3):
     """The decomposition Algorithm 1 runs after the full-rank rebound phase: W is dense and no longer of rank
     <= r, so the factored route does not apply.  ab_svd_split (r_max 192, fixed rank) of one matrix of each
@@ -704,7 +740,7 @@ def run_ours(args):
         h2d = sum(L["h"]["x"].numel() + L["h"]["dY"].numel() for L in layers) * 2
         d2h = sum(sum(L["hout"][k].numel() * L["hout"][k].element_size() for k in ("dA", "dB")) for L in layers)
         per_gpu = value / world
-        # dominant kernel of the chain: row_chain_kernel (every forward call is exactly one launch of
+        # dominant kernel of the chain: chain_kernel (every forward call is exactly one launch of
         # it; backward launches it once more).  Algorithmic work of a forward launch: 2 N r (m+n) FLOP
         # (both layers have m+n = 3840), 2 N (m+n) bytes.
         fwd_flops = 2.0 * N * R * 3840
@@ -715,7 +751,7 @@ def run_ours(args):
         # 0.1 ms at full clocks) or its intensity times the HBM peak
         hbm_ceiling_tflops = fwd_flops / fwd_bytes * pk["hbm"] / 1e3
         hbm_bound = hbm_ceiling_tflops < pk["tc_burst"]
-        kernel = "row_chain_units_kernel (one launch = ab_layer_forward of one layer at this size)"
+        kernel = "chain_kernel (one launch = ab_layer_forward of one layer at this size)"
         common = dict(kernel=kernel, traffic=ROW_CHAIN_DRAM_BYTES_PER_LAUNCH, us_per_launch=fwd_ms * 1e3,
                       tflops=fwd_tflops, algorithmic_gbs=fwd_gbs, hbm_peak_gbs=pk["hbm"], tensor_peak_tflops=pk["tc_burst"],
                       frac_of_tensor_burst=fwd_tflops / pk["tc_burst"], frac_of_hbm=fwd_gbs / pk["hbm"],
@@ -754,6 +790,7 @@ def run_ours(args):
             line["other_workloads"] = other_workloads(ab, torch)
             line["adamw_update_vit_factors"] = optimizer_step(ab, torch)
             line["dense_split_ms"] = dense_split_times(ab, torch)
+            line["fused_mean_recombine"] = fused_mean_recombine(ab, torch)
             line["implicit_conv"] = conv_workloads(ab, torch)
             torch.cuda.empty_cache()
             line["training_cycle"] = training_cycle(ab, torch)

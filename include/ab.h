@@ -232,6 +232,18 @@ int ab_recombine(const void* Abar, const void* Bbar, float* W, int m, int n, int
                  int ldA, int ldB, int dt, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The two all-reduces and the recombination of Algorithm 1 in ONE kernel: W = mean_k(A_k) mean_k(B_k), the mean
+ * taken in the product's operand loader (fp32, copies added in ascending k, times fl(1/K): the bits of
+ * ab_group_average); Abar [m,r] and Bbar [r,n], when not NULL, receive the averaged factors (written by the
+ * CTAs of the first tile column / row).  fp32 factors only (AB_ERR_UNSUPPORTED otherwise); product on the fp32
+ * pipes.  Every output tile re-reads the K copies of its operand panels, so for K > 1 this is slower than
+ * ab_group_average + ab_recombine on all but small matrices (measured: the bench line's fused_mean_recombine);
+ * it is here for callers who want one launch and no intermediate.
+ */
+int ab_recombine_mean(const void* A_copies, int64_t strideA, const void* B_copies, int64_t strideB, int K,
+                      float* W, float* Abar, float* Bbar, int m, int n, int r, int dt, void* cuda_stream);
+
+/*
  * Truncated SVD and split (Eq. 3 with the rank rule of the AB-decomposition phase):
  *   W = U S V^T;  r' = #{ i < r_cap : s_i >= sigma_cutoff * s_0 }, at least 1, where
  *   r_cap = min(r_max, m, n);  A = U_r' S_r'^(1/2),  B = S_r'^(1/2) V_r'^T.

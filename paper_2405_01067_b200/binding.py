@@ -27,7 +27,7 @@ EXPORTS = ["ab_status_string", "ab_version", "ab_launch_count", "ab_workspace_by
            "ab_layer_forward_static", "ab_static_scratch_elems", "ab_adamw_step", "ab_lr_rebound_factor", "ab_selftest_bounded_wait",
            "ab_selftest_chain_stall", "ab_selftest_chain_stall_workspace_bytes",
            "ab_dense_forward", "ab_dense_backward", "ab_conv3x3_forward", "ab_conv3x3_backward",
-           "ab_conv3x3_workspace_bytes"]
+           "ab_conv3x3_workspace_bytes", "ab_recombine_mean"]
 
 
 class AbError(RuntimeError):
@@ -98,6 +98,9 @@ def lib() -> ctypes.CDLL:
     L.ab_conv3x3_backward.argtypes = [c_void_p] * 8 + [c_int] * 9 + [c_void_p, c_size_t, c_void_p]
     L.ab_conv3x3_workspace_bytes.restype = c_size_t
     L.ab_conv3x3_workspace_bytes.argtypes = [c_int] * 6
+    L.ab_recombine_mean.restype = c_int
+    L.ab_recombine_mean.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_int, c_void_p, c_void_p, c_void_p,
+                                    c_int, c_int, c_int, c_int, c_void_p]
     _lib = L
     return L
 
@@ -340,6 +343,26 @@ def ab_recombine(Abar, Bbar, W=None, ws=None, stream=None):
                             _ptr(ws), ws.numel(), _stream(stream))
     _check(st, "ab_recombine")
     return W
+
+
+def ab_recombine_mean(A_copies, B_copies, W=None, Abar=None, Bbar=None, want_means=True, stream=None):
+    """W = mean_k(A_k) mean_k(B_k) in one kernel; A_copies (K, m, r), B_copies (K, r, n), fp32.
+    Returns (W, Abar, Bbar) (the means are None when want_means is False and none were passed)."""
+    _dev_ok(A_copies, B_copies, W, Abar, Bbar)
+    K, m, r = A_copies.shape
+    n = B_copies.shape[2]
+    dev = A_copies.device
+    if W is None:
+        W = torch.empty((m, n), dtype=torch.float32, device=dev)
+    if want_means and Abar is None:
+        Abar = torch.empty((m, r), dtype=torch.float32, device=dev)
+    if want_means and Bbar is None:
+        Bbar = torch.empty((r, n), dtype=torch.float32, device=dev)
+    st = lib().ab_recombine_mean(_ptr(A_copies), A_copies.stride(0) if K > 1 else m * r, _ptr(B_copies),
+                                 B_copies.stride(0) if K > 1 else r * n, K, _ptr(W), _ptr(Abar), _ptr(Bbar), m, n, r,
+                                 _dt(A_copies), _stream(stream))
+    _check(st, "ab_recombine_mean")
+    return W, Abar, Bbar
 
 
 def ab_svd_split(W, r_max, sigma_cutoff=0.0, out_dtype=None, ws=None, stream=None):

@@ -321,6 +321,17 @@ int ab_recombine(const void* Abar, const void* Bbar, float* W, int m, int n, int
   return gemm_tc_batched(&q, 1, w.table, w.status, st);
 }
 
+int ab_recombine_mean(const void* A_copies, int64_t strideA, const void* B_copies, int64_t strideB, int K,
+                      float* W, float* Abar, float* Bbar, int m, int n, int r, int dt, void* cuda_stream) {
+  if (!dtype_ok(dt) || m <= 0 || n <= 0 || r <= 0 || K < 1) return AB_ERR_INVALID_ARG;
+  if (!A_copies || !B_copies || !W) return AB_ERR_INVALID_ARG;
+  if (K > 1 && (strideA < (int64_t)m * r || strideB < (int64_t)r * n)) return AB_ERR_INVALID_ARG;
+  if (K > 64 || dt != AB_F32) return AB_ERR_UNSUPPORTED;
+  if (!have_device()) return AB_ERR_CUDA;
+  return recombine_mean_simt(static_cast<const float*>(A_copies), strideA, static_cast<const float*>(B_copies), strideB, K,
+                             W, Abar, Bbar, m, n, r, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int ab_svd_split(const void* W, int m, int n, int r_max, float sigma_cutoff,
                  void* A, void* B, float* sigma, int* r_out, int* dev_status,
                  int w_dt, int out_dt, void* ws, size_t ws_bytes, void* cuda_stream) {

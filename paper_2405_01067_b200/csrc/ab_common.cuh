@@ -90,8 +90,19 @@ struct GemmDesc {
   float thr;
   const int* live_rows; const int* live_cols;
   int upper_only;   // 1: tiles entirely below the diagonal are skipped (symmetric result, upper part used)
+  // Operand prologue that averages group copies (0 / 1 copies: plain operand).  Copy c of A starts a_cstride
+  // elements after copy c - 1; the loader adds the copies in ascending c in fp32 and scales by copy_inv, the
+  // arithmetic of the group mean.  The CTAs of the first tile column / row also write the averaged operand out.
+  int a_copies, b_copies;
+  int64_t a_cstride, b_cstride;
+  float copy_inv;
+  float* a_mean_out;   // optional, M x K row-major
+  float* b_mean_out;   // optional, K x N row-major
 };
 int gemm_simt_batched(const GemmDesc* d_descs, int count, int max_M, int max_N, cudaStream_t st);
+// W = mean_k(A_k) mean_k(B_k) in one kernel (the mean as the product's operand prologue); Abar, Bbar optional outputs.
+int recombine_mean_simt(const float* A_copies, int64_t strideA, const float* B_copies, int64_t strideB, int K,
+                        float* W, float* Abar, float* Bbar, int m, int n, int r, cudaStream_t st);
 
 // ---- general tensor-core GEMM (ab_gemm_tc.cu) --------------------------------------------------
 // C[M x N] = sum over terms of A_t B_t^T on the tensor cores; see the head of ab_gemm_tc.cu.

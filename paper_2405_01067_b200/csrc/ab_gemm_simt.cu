@@ -119,8 +119,23 @@ struct TileIo {
   const float* P;
   int64_t s_r, s_k;
   bool along_k, vec;
+  int copies; int64_t cstride; float cinv;      // group copies averaged on the way in (see GemmDesc)
+  __device__ __forceinline__ void add_copies(float (&t)[4], const float* p, bool as_vec, int64_t step, int valid) const {
+    for (int c = 1; c < copies; ++c) {
+      const float* q = p + c * cstride;
+      if (as_vec) {
+        const float4 v = *reinterpret_cast<const float4*>(q);
+        t[0] = __fadd_rn(t[0], v.x); t[1] = __fadd_rn(t[1], v.y); t[2] = __fadd_rn(t[2], v.z); t[3] = __fadd_rn(t[3], v.w);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) if (j < valid) t[j] = __fadd_rn(t[j], q[j * step]);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) t[j] = __fmul_rn(t[j], cinv);
+  }
   __device__ __forceinline__ void init(const float* p, int64_t sr, int64_t sk) {
-    P = p; s_r = sr; s_k = sk;
+    P = p; s_r = sr; s_k = sk; copies = 1; cstride = 0; cinv = 1.f;
     along_k = (sk == 1) || (sk < sr && sr != 1);
     const bool al = (reinterpret_cast<uintptr_t>(p) & 15u) == 0;
     vec = al && (along_k ? (sk == 1 && (sr & 3) == 0) : (sr == 1 && (sk & 3) == 0));
@@ -138,9 +153,11 @@ struct TileIo {
         if (vec && gr < R && gk + 3 < K) {
           const float4 q = *reinterpret_cast<const float4*>(p);
           t[0] = q.x; t[1] = q.y; t[2] = q.z; t[3] = q.w;
+          if (copies > 1) add_copies(t, p, true, 0, 4);
         } else {
 #pragma unroll
           for (int j = 0; j < 4; ++j) t[j] = (gr < R && gk + j < K) ? p[j * s_k] : 0.f;
+          if (copies > 1 && gr < R) add_copies(t, p, false, s_k, (int)(K - gk < 4 ? (K - gk < 0 ? 0 : K - gk) : 4));
         }
         if (kvec) {
 #pragma unroll
@@ -153,9 +170,11 @@ struct TileIo {
         if (vec && gr + 3 < R && gk < K) {
           const float4 q = *reinterpret_cast<const float4*>(p);
           t[0] = q.x; t[1] = q.y; t[2] = q.z; t[3] = q.w;
+          if (copies > 1) add_copies(t, p, true, 0, 4);
         } else {
 #pragma unroll
           for (int j = 0; j < 4; ++j) t[j] = (gr + j < R && gk < K) ? p[j * s_r] : 0.f;
+          if (copies > 1 && gk < K) add_copies(t, p, false, s_r, (int)(R - gr < 4 ? (R - gr < 0 ? 0 : R - gr) : 4));
         }
         if (kvec && gk < K) {
           const float sc = diag_scale(kvec, (int)gk, kmode, thr);
@@ -164,6 +183,26 @@ struct TileIo {
         }
       }
       v[e] = make_float4(t[0], t[1], t[2], t[3]);
+    }
+  }
+  // writes the fetched values to a dense copy of the operand: element (r, k) at out[r * o_r + k * o_k]
+  __device__ __forceinline__ void emit(float* out, int64_t o_r, int64_t o_k, const float4 (&v)[F], int64_t r0, int R,
+                                       int64_t k0, int K, int tid) const {
+#pragma unroll
+    for (int e = 0; e < F; ++e) {
+      const int f = tid + e * NT;
+      const float t[4] = {v[e].x, v[e].y, v[e].z, v[e].w};
+      if (along_k) {
+        const int k4 = f & 3, row = f >> 2;
+        const int64_t gr = r0 + row, gk = k0 + 4 * k4;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) if (gr < R && gk + j < K) out[gr * o_r + (gk + j) * o_k] = t[j];
+      } else {
+        const int r4 = f % (R_ / 4), kk = f / (R_ / 4);
+        const int64_t gr = r0 + 4 * r4, gk = k0 + kk;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) if (gr + j < R && gk < K) out[(gr + j) * o_r + gk * o_k] = t[j];
+      }
     }
   }
   __device__ __forceinline__ void stash(float (*S)[R_ + 4], const float4 (&v)[F], int tid) const {
@@ -196,6 +235,10 @@ __device__ __forceinline__ void gemm_tile_8x8(const GemmDesc& d) {
   TileIo<BN_, NT> ioB;
   ioA.init(d.A, d.sAm, d.sAk);
   ioB.init(d.B, d.sBn, d.sBk);
+  if (d.a_copies > 1) { ioA.copies = d.a_copies; ioA.cstride = d.a_cstride; ioA.cinv = d.copy_inv; }
+  if (d.b_copies > 1) { ioB.copies = d.b_copies; ioB.cstride = d.b_cstride; ioB.cinv = d.copy_inv; }
+  const bool emit_a = d.a_mean_out != nullptr && blockIdx.x == 0;     // first tile column writes Abar
+  const bool emit_b = d.b_mean_out != nullptr && blockIdx.y == 0;     // first tile row writes Bbar
   float4 va[TileIo<BM_, NT>::F], vb[TileIo<BN_, NT>::F];
   float acc[8][8];
 #pragma unroll
@@ -206,6 +249,8 @@ __device__ __forceinline__ void gemm_tile_8x8(const GemmDesc& d) {
   const int nk = (d.K + BK - 1) / BK;
   ioA.fetch(va, m0, d.M, 0, d.K, d.k_vec, d.k_mode, d.thr, tid);
   ioB.fetch(vb, n0, d.N, 0, d.K, nullptr, 0, 0.f, tid);
+  if (emit_a) ioA.emit(d.a_mean_out, d.K, 1, va, m0, d.M, 0, d.K, tid);
+  if (emit_b) ioB.emit(d.b_mean_out, 1, d.N, vb, n0, d.N, 0, d.K, tid);
   ioA.stash(As[0], va, tid);
   ioB.stash(Bs[0], vb, tid);
   __syncthreads();
@@ -215,6 +260,8 @@ __device__ __forceinline__ void gemm_tile_8x8(const GemmDesc& d) {
     if (more) {
       ioA.fetch(va, m0, d.M, (int64_t)(kt + 1) * BK, d.K, d.k_vec, d.k_mode, d.thr, tid);
       ioB.fetch(vb, n0, d.N, (int64_t)(kt + 1) * BK, d.K, nullptr, 0, 0.f, tid);
+      if (emit_a) ioA.emit(d.a_mean_out, d.K, 1, va, m0, d.M, (int64_t)(kt + 1) * BK, d.K, tid);
+      if (emit_b) ioB.emit(d.b_mean_out, 1, d.N, vb, n0, d.N, (int64_t)(kt + 1) * BK, d.K, tid);
     }
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
@@ -322,6 +369,26 @@ int gemm_simt_batched(const GemmDesc* d_descs, int count, int max_M, int max_N, 
   return launch_batched<64, 64>(d_descs, count, max_M, max_N, st);
 }
 
+int recombine_mean_simt(const float* A_copies, int64_t strideA, const float* B_copies, int64_t strideB, int K,
+                        float* W, float* Abar, float* Bbar, int m, int n, int r, cudaStream_t st) {
+  GemmDesc d;
+  d.A = A_copies; d.B = B_copies; d.C = W;
+  d.sAm = r; d.sAk = 1; d.sBk = n; d.sBn = 1; d.ldc = n;
+  d.M = m; d.N = n; d.K = r; d.c_bf16 = 0;
+  d.row_vec = d.col_vec = d.k_vec = nullptr;
+  d.row_mode = d.col_mode = d.k_mode = 0;
+  d.thr = 0.f;
+  d.live_rows = d.live_cols = nullptr;
+  d.upper_only = 0;
+  d.a_copies = d.b_copies = K; d.a_cstride = strideA; d.b_cstride = strideB; d.copy_inv = 1.0f / (float)K;
+  d.a_mean_out = Abar; d.b_mean_out = Bbar;
+  const bool bigM = m >= 512, bigN = n >= 512;
+  if (bigM && bigN) return launch_one<128, 128>(d, st);
+  if (bigM) return launch_one<128, 64>(d, st);
+  if (bigN) return launch_one<64, 128>(d, st);
+  return launch_one<64, 64>(d, st);
+}
+
 int gemm_simt(const void* A, int a_dt, int64_t sAm, int64_t sAk,
               const void* B, int b_dt, int64_t sBk, int64_t sBn,
               void* C, int c_dt, int64_t ldc,
@@ -341,6 +408,7 @@ int gemm_simt(const void* A, int a_dt, int64_t sAm, int64_t sAk,
     d.thr = 0.f;
     d.live_rows = d.live_cols = nullptr;
     d.upper_only = 0;
+    d.a_copies = d.b_copies = 1; d.a_cstride = d.b_cstride = 0; d.copy_inv = 1.f; d.a_mean_out = d.b_mean_out = nullptr;
     const bool bigM = M >= 512, bigN = N >= 512;
     if (bigM && bigN) return launch_one<128, 128>(d, st);
     if (bigM) return launch_one<128, 64>(d, st);

@@ -635,6 +635,7 @@ GemmDesc mk(const float* A, int64_t sAm, int64_t sAk, const float* B, int64_t sB
   g.thr = kEigThr;
   g.live_rows = g.live_cols = nullptr;
   g.upper_only = 0;
+  g.a_copies = g.b_copies = 1; g.a_cstride = g.b_cstride = 0; g.copy_inv = 1.f; g.a_mean_out = g.b_mean_out = nullptr;
   return g;
 }
 

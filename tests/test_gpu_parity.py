@@ -238,6 +238,24 @@ def test_recombine_bf16_factors(ab):
     assert orc.rel_frob(host(W), orc.recombine(A, B)) <= 1e-6
 
 
+@pytest.mark.parametrize("m,n,r,K", [(256, 512, 32, 2), (70, 130, 33, 3), (768, 768, 192, 8), (65, 63, 17, 1), (640, 200, 64, 4)])
+def test_recombine_mean_one_kernel(ab, m, n, r, K):
+    """Mean and recombination in one kernel: the averaged factors it writes have the bits of the fixed-order
+    fp32 mean, W matches the checker's product of those means."""
+    rng = np.random.default_rng(m + n + r + K)
+    Ak = rng.standard_normal((K, m, r)).astype(np.float32)
+    Bk = rng.standard_normal((K, r, n)).astype(np.float32)
+    W, Abar, Bbar = ab.ab_recombine_mean(dev(Ak), dev(Bk))
+    torch.cuda.synchronize()
+    Ar, Br = orc.group_average_f32(Ak), orc.group_average_f32(Bk)
+    assert np.array_equal(Abar.cpu().numpy().view(np.uint32), Ar.view(np.uint32))
+    assert np.array_equal(Bbar.cpu().numpy().view(np.uint32), Br.view(np.uint32))
+    assert orc.rel_frob(host(W), orc.recombine(Ar, Br)) <= 1e-6
+    W2, _, _ = ab.ab_recombine_mean(dev(Ak), dev(Bk), want_means=False)
+    torch.cuda.synchronize()
+    assert torch.equal(W, W2)
+
+
 # ------------------------------------------------------------------ SVD split
 
 def check_split(ab, W, r_max, cutoff, out_bf16=False):
