@@ -43,3 +43,32 @@ def test_two_ranks_on_gloo():
     assert t0 == t1 == [11.0, 5.0, 1.0, 4.0]          # MAX over ranks, identical on every rank
     import bench
     assert np.isclose(v0, 2 * bench.chain_flops(1024) * 3 / 5.0e-3 / 1e12) and v0 == v1
+
+
+def test_bench_starts_its_own_ranks(monkeypatch):
+    """`python bench.py --gpus N` outside torchrun re-launches itself under torch.distributed.run with one process
+    per GPU on 127.0.0.1 and hands back that launcher's exit status; under torchrun (WORLD_SIZE set) it does not."""
+    import subprocess
+    import bench
+    seen = {}
+
+    def fake_call(cmd):
+        seen["cmd"] = cmd
+        return 7
+
+    monkeypatch.setattr(subprocess, "call", fake_call)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4", "--steps", "3"])
+    assert bench.spawn_ranks(4) == 7
+    cmd = seen["cmd"]
+    assert cmd[1:3] == ["-m", "torch.distributed.run"]
+    assert "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert int(cmd[cmd.index("--master-port") + 1]) > 0
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "3"] and cmd[-5].endswith("bench.py")
+    # main() takes that route only when no launcher has set the world size
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    called = {}
+    monkeypatch.setattr(bench, "spawn_ranks", lambda n: called.setdefault("n", n) or 0)
+    with __import__("pytest").raises(SystemExit):
+        bench.main()
+    assert called["n"] == 4
