@@ -548,6 +548,13 @@ __global__ void fast_rank_rule_kernel(const float* const* __restrict__ sigma, co
   }
 }
 
+// A bounded wait that ran out inside one of the tensor-core launches of the call reaches every matrix's status.
+__global__ void fold_tc_status_kernel(const int* __restrict__ tc_status, int* __restrict__ dev_status, int L) {
+  const int bad = (tc_status[0] != AB_OK) ? tc_status[0] : (tc_status[1] != AB_OK) ? tc_status[1] : tc_status[2];
+  if (bad == AB_OK) return;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < L; i += gridDim.x * blockDim.x) dev_status[i] = bad;
+}
+
 // The long index of a Gram product is cut into slices of about kGramSlice (at most kGramMaxParts).
 constexpr int kGramSlice = 768, kGramMaxParts = 8;
 int gram_parts(int len) { return std::max(1, std::min(kGramMaxParts, (len + kGramSlice - 1) / kGramSlice)); }
@@ -903,6 +910,10 @@ int sync_factored(const ab_sync_desc* d, int L, int K, float sigma_cutoff, int d
   if (side) {
     if (side_rc == AB_OK && cudaStreamWaitEvent(st, join, 0) != cudaSuccess) side_rc = AB_ERR_CUDA;
     if (side_rc != AB_OK) { (void)cudaGetLastError(); return side_rc; }
+  }
+  if (use_tc && dev_status) {
+    fold_tc_status_kernel<<<1, 128, 0, st>>>(w.tc_status, dev_status, L);
+    AB_LAUNCH_OK();
   }
   return AB_OK;
 }
